@@ -1,0 +1,194 @@
+/*
+ * flashmesh.h -- C ABI of the speculative decode step of an hourglass mesh transformer
+ * (FlashMesh, arXiv 2511.15618), hand-written CUDA for sm_100a, one GPU.
+ *
+ * The paper states the problem as: given a condition c and the accepted prefix, every
+ * forward pass of the backbone yields one main token and the draft modules yield D draft
+ * tokens (Sec. 3.1); the drafts may be edited before they are fed back (Sec. 3.2); one
+ * forward pass with causal masking verifies main + drafts (Sec. 3.3); the main token and
+ * the drafts up to the first mismatch are accepted and decoding continues from the
+ * backbone's output at the last accepted token (Sec. 3.3).  The calls below are those
+ * stages.  The model is the hourglass of the supplement ("Hourglass Transformer": three
+ * coordinates form a vertex, three vertices a face; shortening and upsampling layers with
+ * residuals between levels) with a KV cache at each level.
+ *
+ * Conventions
+ *   - Every call returns FM_OK (0) or a negative FM_ERR_* code; nothing throws.  On an error
+ *     return no decoding state has been changed.
+ *   - Pointers are marked HOST or DEV.  DEV pointers are caller-owned device memory that must
+ *     stay valid until the work enqueued by the call has finished on the context's stream.
+ *   - All calls except fm_create / fm_destroy / fm_generate only enqueue work on the
+ *     context's stream and return; fm_generate polls a completion flag and returns when every
+ *     sequence has finished.
+ *   - The library allocates no device memory: the caller hands a workspace of
+ *     fm_workspace_bytes() bytes to fm_create, which carves weights (bfloat16), KV caches and
+ *     scratch out of it.  (fm_create allocates a few hundred bytes of pinned host memory.)
+ *   - Indexing: inputs u_0 = BOS, u_i = t_{i-1}; the row at position i predicts mesh token
+ *     t_i.  L = inputs consumed so far; the pending main token is t_{L-1}.  A verify pass
+ *     feeds positions L..L+D; accepting a tokens moves L to L+a.
+ *   - Token ids: [0, n_bins) coordinate bins, BOS = n_bins, EOS = n_bins+1, PAD = n_bins+2.
+ *     Emitted ids are always coordinate bins, or EOS at a face boundary when allow_eos != 0;
+ *     ties in an argmax go to the lowest id.
+ */
+#ifndef FLASHMESH_H
+#define FLASHMESH_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FM_OK                0
+#define FM_ERR_INVALID_ARG  -1   /* null pointer, size out of range, inconsistent config      */
+#define FM_ERR_BAD_STATE    -2   /* call out of order (e.g. fm_verify before fm_prefill)       */
+#define FM_ERR_CAPACITY     -3   /* batch > max_batch, prompt or run longer than max_tokens    */
+#define FM_ERR_CUDA         -4   /* a CUDA runtime call failed                                 */
+#define FM_ERR_TIMEOUT      -5   /* a bounded device-side wait gave up (see fm_device_status)  */
+#define FM_ERR_UNSUPPORTED  -6   /* shape outside what the kernels were built for              */
+
+#define FM_MAX_FACE_HEADS 4
+#define FM_MAX_DRAFT      24
+
+typedef struct fm_ctx fm_ctx;    /* opaque; owns nothing but pinned host flags */
+
+/* Model and capacity description (the hourglass of the supplement; every reading the paper
+ * leaves open is fixed in the oracle's header and repeated here where it shapes a field). */
+typedef struct fm_config {
+  int32_t d_model, n_heads, n_kv_heads, head_dim, d_ff;
+  int32_t layers[5];          /* coord_down, vertex_down, face, vertex_up, coord_up          */
+  int32_t n_bins;             /* vocabulary = n_bins + 3                                     */
+  int32_t n_prefix;           /* P conditioning vectors, held as prefix keys/values          */
+  int32_t window[3];          /* attention window per level (coordinate, vertex, face); 0 = full */
+  int32_t draft_len;          /* D, 0..FM_MAX_DRAFT                                          */
+  int32_t max_batch;
+  int32_t max_tokens;         /* capacity per sequence in coordinate positions (inputs)      */
+  float   rope_theta;         /* 0 = no positional encoding                                  */
+  float   norm_eps;
+  int32_t allow_eos;          /* 0: EOS is masked everywhere (fixed-length runs)             */
+} fm_config;
+
+/* HOST pointers to float32 matrices, row-major [out, in]; values are rounded to bfloat16
+ * (nearest-even) when fm_create copies them.  Gains stay float32. */
+typedef struct fm_layer_weights {
+  const float* g1;            /* [d]                          RMSNorm gain before attention   */
+  const float* Wqkv;          /* [(H + 2*Hkv)*dh, d]          rows: Q heads, K heads, V heads */
+  const float* Wo;            /* [d, H*dh]                                                    */
+  const float* g2;            /* [d]                          RMSNorm gain before the FFN     */
+  const float* W1;            /* [d_ff, d]                                                    */
+  const float* W2;            /* [d, d_ff]                                                    */
+} fm_layer_weights;
+
+typedef struct fm_weights {
+  const float* E;                         /* [V, d] token embedding                          */
+  const fm_layer_weights* stack[5];       /* stack[s][l], l < layers[s]                      */
+  const float* S_cv;                      /* [d, 3d] shorten coordinate -> vertex            */
+  const float* S_vf;                      /* [d, 3d] shorten vertex -> face                  */
+  const float* U_fv;                      /* [3d, d] upsample face -> 3 vertices             */
+  const float* U_vc;                      /* [3d, d] upsample vertex -> 3 coordinates        */
+  const float* g_out;                     /* [d]                                              */
+  const float* W_out;                     /* [V, d]                                           */
+  const float* head_c_g[2];  const float* head_c_A[2];   /* coordinate draft heads, A [d,d]  */
+  const float* head_v_g[2];  const float* head_v_A[2];   /* vertex (point) draft heads       */
+  const float* head_f_g[FM_MAX_FACE_HEADS]; const float* head_f_A[FM_MAX_FACE_HEADS]; /* ceil(D/9) used */
+} fm_weights;
+
+/* Optional device-side draft editor for fm_generate: the place where the paper's Correct
+ * stage sits (Sec. 3.2 edits drafts only, never the main token).  Used by the benchmark to
+ * pin the true acceptance length: draft j (1..keep) is replaced by the known continuation,
+ * draft keep+1 by a deliberately different coordinate id. */
+typedef struct fm_teacher {
+  const int32_t* truth;       /* DEV [batch, truth_stride]: mesh tokens t_0.. (prompt included) */
+  int32_t truth_stride;
+  const int32_t* keep;        /* DEV [n_sched, batch]: correct drafts wanted per step, 0..D  */
+  int32_t n_sched;            /* the schedule wraps around                                   */
+} fm_teacher;
+
+typedef struct fm_stats {
+  int64_t steps;                          /* draft+verify+accept passes executed             */
+  int64_t emitted;                        /* mesh tokens emitted, all sequences              */
+  int64_t accept_hist[FM_MAX_DRAFT + 2];  /* accept_hist[a] = passes that accepted a tokens  */
+  float   ms;                             /* device time of the decode loop (CUDA events)    */
+} fm_stats;
+
+/* Bytes of device workspace fm_create needs for this configuration (0 if it is invalid). */
+size_t fm_workspace_bytes(const fm_config* cfg /*HOST*/);
+
+/* Build a context inside `dev_workspace` (DEV, 256-byte aligned, >= fm_workspace_bytes):
+ * copies and rounds the weights, zeroes state.  `cuda_stream` is a cudaStream_t (NULL = the
+ * default stream); all later work of this context runs on it.  Synchronous.
+ * Errors: INVALID_ARG (null, bad config), CAPACITY (workspace too small), UNSUPPORTED
+ * (d_model not a multiple of 64, head_dim not 32/64/128, D > FM_MAX_DRAFT), CUDA. */
+int fm_create(const fm_config* cfg /*HOST*/, const fm_weights* w /*HOST*/, void* dev_workspace /*DEV*/,
+              size_t workspace_bytes, void* cuda_stream, fm_ctx** out /*HOST*/);
+int fm_destroy(fm_ctx* ctx);
+
+/* Start `batch` sequences.  cond: DEV float32 [batch, P, d] conditioning vectors, projected by
+ * every layer's own K/V matrices into prefix cache slots.  prompt: DEV int32, the sequences'
+ * mesh tokens concatenated; prompt_off: HOST int32 [batch+1] offsets into it (lengths must be
+ * multiples of 9).  Runs BOS + prompt through the multi-row forward in chunks of D+1 rows.
+ * Afterwards L[b] = 1 + prompt_len[b] and the first main token is pending.
+ * Errors: INVALID_ARG, CAPACITY. */
+int fm_prefill(fm_ctx* ctx, int32_t batch, const float* cond /*DEV*/, const int32_t* prompt /*DEV*/,
+               const int32_t* prompt_off /*HOST*/);
+
+/* Per-sequence limit: sequence b stops once 9*max_faces[b] tokens have been emitted after
+ * its prompt (or at EOS).  HOST int32 [batch].  Default: the cache capacity. */
+int fm_set_max_faces(fm_ctx* ctx, const int32_t* max_faces /*HOST*/);
+
+/* Predict (Sec. 3.1, supplement "Three-Level Speculative Decoding"): run the draft heads on
+ * the split-node hiddens stashed at the last accepted position.  cand: DEV int32 out
+ * [batch, D+1] = pending main token, then D drafts (PAD for finished sequences).
+ * draft_logits: DEV float32 out [batch, D, V] or NULL.  draft_margin: DEV float32 out
+ * [batch, D] (top-1 minus top-2 of the masked draft logits) or NULL. */
+int fm_draft(fm_ctx* ctx, int32_t* cand /*DEV*/, float* draft_logits /*DEV*/, float* draft_margin /*DEV*/);
+
+/* Verify (Sec. 3.3): one forward pass over main + D candidates, causal among themselves,
+ * through all five level stacks.  cand: DEV int32 in [batch, D+1]; cand[b][0] must be the
+ * pending main token.  Rows fed per sequence = min(D+1, tokens left).  argmax: DEV int32 out
+ * [batch, D+1] (masked argmax per row, -1 for rows not fed) or NULL; logits: DEV float32 out
+ * [batch, D+1, V] or NULL; margin: DEV float32 out [batch, D+1] or NULL.
+ * Writes keys/values beyond L (invisible until accepted); does not move L; calling it twice
+ * is legal and gives the same result. */
+int fm_verify(fm_ctx* ctx, const int32_t* cand /*DEV*/, int32_t* argmax /*DEV*/, float* logits /*DEV*/,
+              float* margin /*DEV*/);
+
+/* Accept (Sec. 3.3) and roll back: a = 1 + number of leading drafts that equal the backbone's
+ * argmax at the previous row; clipped to the rows fed and at an accepted EOS; L += a; the next
+ * main token is the argmax at row a-1.  force_tok: DEV int32 [batch, D+1] or NULL, replaces the
+ * stored argmax; force_len: DEV int32 [batch] or NULL, replaces a (values 1..D+1).
+ * n_acc: DEV int32 out [batch]; emitted: DEV int32 out [batch, D+1] (accepted ids, then -1);
+ * kv_len: DEV int32 out [batch, 3] = (L, ceil(L/3), ceil(L/9)).  Any output may be NULL.
+ * Errors: BAD_STATE if no fm_verify preceded it. */
+int fm_accept(fm_ctx* ctx, const int32_t* force_len /*DEV*/, const int32_t* force_tok /*DEV*/,
+              int32_t* n_acc /*DEV*/, int32_t* emitted /*DEV*/, int32_t* kv_len /*DEV*/);
+
+/* The whole loop (Sec. 3): draft -> (optional teacher edit) -> verify -> accept, until every
+ * sequence has emitted 9*max_faces tokens or EOS.  out_tok: DEV int32 [batch, out_stride]
+ * receives the emitted tokens (prompt not included), out_len: DEV int32 [batch].  teacher and
+ * stats may be NULL.  plain != 0 accepts only the main token every pass (the one-token-at-a-
+ * time baseline on the same kernels).  Synchronous (returns after the last pass).
+ * Errors: BAD_STATE, CAPACITY (prompt + 9*max_faces + D + 2 > max_tokens, or out_stride too small). */
+int fm_generate(fm_ctx* ctx, int32_t max_faces, int32_t* out_tok /*DEV*/, int32_t out_stride,
+                int32_t* out_len /*DEV*/, const fm_teacher* teacher /*HOST struct, DEV arrays*/,
+                int32_t plain, fm_stats* stats /*HOST*/);
+
+/* Algorithmic bytes one verify pass must move for the given per-sequence lengths (weights of
+ * the stacks that have rows, shorten/upsample, output matrix, K and V entries visible to the
+ * rows); kv_len HOST int32 [batch,3] as returned by fm_accept.  For roofline reports. */
+double fm_verify_bytes(const fm_ctx* ctx, int32_t batch, const int32_t* kv_len /*HOST*/);
+
+/* Number of kernels launched by this context since creation (for launch accounting). */
+int64_t fm_launch_count(const fm_ctx* ctx);
+
+const char* fm_strerror(int code);
+/* Device status word: 0, or FM_ERR_TIMEOUT if a bounded wait inside a kernel gave up, or
+ * FM_ERR_INVALID_ARG if a kernel met an out-of-range token id (it then used PAD).  Synchronises
+ * the stream. */
+int fm_device_status(fm_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLASHMESH_H */

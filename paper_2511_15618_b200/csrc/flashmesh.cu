@@ -1,0 +1,668 @@
+// C ABI and host orchestration of the speculative decode step (see include/flashmesh.h).
+// All arithmetic of the path runs in the kernels of this directory; the host only carves the
+// workspace, uploads weights and enqueues launches.
+#include "../../include/flashmesh.h"
+
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "fm_attention.cuh"
+#include "fm_common.cuh"
+#include "fm_gemm.cuh"
+#include "fm_kernels.cuh"
+
+namespace {
+
+constexpr int STACK_LEVEL[5] = {0, 1, 2, 1, 0};
+constexpr int PREFILL_CHUNK = 512;      // conditioning rows projected per launch group
+
+struct LayerDev {
+  bf16 *Wqkv, *Wo, *W1, *W2;
+  float *g1, *g2;
+  bf16 *K, *V;                          // [max_batch, Hkv, P + cap, dh]
+};
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int round_up(int v, int a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+
+struct fm_ctx {
+  fm_config cfg;
+  Dims dm;
+  cudaStream_t stream;
+  char* ws;
+  size_t ws_bytes;
+  // weights
+  bf16* E;
+  std::vector<LayerDev> layers[5];
+  bf16 *S_cv, *S_vf, *U_fv, *U_vc, *W_out, *headA;
+  float *g_out, *head_g;
+  double* inv_freq;
+  // state
+  SeqState st;
+  // activations
+  float *xc, *xv, *xf, *qkv, *qbuf, *logits, *tmp3d;
+  bf16 *a_norm, *a_cat, *a_attn, *a_ff;
+  float *hc_ring, *hv_ring, *trif_ring, *triv_ring, *zc, *zv, *zf;
+  // draft
+  bf16 *dh_a, *up_in_v, *up_in_f, *feat_n;
+  float *dh_y, *feat, *dlogits;
+  // prefill temporaries
+  bf16* pre_a;
+  float* pre_o;
+  int* prompt_off_dev;
+  // generate
+  GenOut* gen_dev;
+  long long* stats_dev;
+  int* host_done;       // pinned, mapped
+  int* host_done_dev;
+  int batch;
+  std::vector<int> plen_host;
+  int phase;            // 0 created, 1 prefilled / accepted, 2 verified
+  int64_t launches;
+};
+
+namespace {
+
+// ------------------------------------------------------------------------------------------
+// configuration checks and workspace layout
+// ------------------------------------------------------------------------------------------
+int check_config(const fm_config* c) {
+  if (c == nullptr) return FM_ERR_INVALID_ARG;
+  if (c->d_model <= 0 || c->n_heads <= 0 || c->n_kv_heads <= 0 || c->head_dim <= 0 || c->d_ff <= 0) return FM_ERR_INVALID_ARG;
+  if (c->n_heads % c->n_kv_heads != 0) return FM_ERR_INVALID_ARG;
+  if (c->n_bins <= 0 || c->n_prefix < 0 || c->max_batch <= 0 || c->max_tokens <= 0) return FM_ERR_INVALID_ARG;
+  if (c->draft_len < 0 || c->norm_eps < 0.f) return FM_ERR_INVALID_ARG;
+  for (int i = 0; i < 3; ++i) if (c->window[i] < 0) return FM_ERR_INVALID_ARG;
+  for (int i = 0; i < 5; ++i) if (c->layers[i] < 1) return FM_ERR_UNSUPPORTED;
+  if (c->draft_len > FM_MAX_DRAFT) return FM_ERR_UNSUPPORTED;
+  if (c->d_model % 64 != 0 || c->d_ff % 64 != 0 || (c->n_heads * c->head_dim) % 64 != 0) return FM_ERR_UNSUPPORTED;
+  if (c->head_dim != 32 && c->head_dim != 64 && c->head_dim != 128) return FM_ERR_UNSUPPORTED;
+  if ((c->draft_len + 8) / 9 > FM_MAX_FACE_HEADS) return FM_ERR_UNSUPPORTED;
+  if (c->max_tokens < c->draft_len + 2) return FM_ERR_INVALID_ARG;
+  return FM_OK;
+}
+
+Dims make_dims(const fm_config& c) {
+  Dims dm;
+  dm.d = c.d_model; dm.H = c.n_heads; dm.Hkv = c.n_kv_heads; dm.dh = c.head_dim; dm.dff = c.d_ff;
+  dm.n_bins = c.n_bins; dm.V = c.n_bins + 3; dm.Vpad = round_up(dm.V, 128); dm.P = c.n_prefix;
+  dm.D = c.draft_len; dm.R1 = dm.D + 1; dm.mv = (dm.R1 + 2) / 3; dm.mf = (dm.R1 + 8) / 9;
+  for (int l = 0; l < 3; ++l) {
+    dm.window[l] = c.window[l];
+    const int ratio = fm_ratio(l);
+    const int linear = (c.max_tokens + ratio - 1) / ratio + 1;
+    // a windowed level keeps a ring of window + rows of one pass (+ slack) slots
+    const int ring = c.window[l] > 0 ? c.window[l] + fm_rows_per_seq(dm, l) + 8 : linear;
+    dm.cap[l] = ring < linear ? ring : linear;
+  }
+  dm.max_batch = c.max_batch; dm.max_tokens = c.max_tokens; dm.allow_eos = c.allow_eos;
+  dm.eps = c.norm_eps; dm.theta = c.rope_theta;
+  dm.Ef = dm.D > 0 ? (dm.D + 8) / 9 : 1; dm.NH = 4 + dm.Ef;
+  return dm;
+}
+
+// bump allocator; with base == nullptr it only measures
+struct Carver {
+  char* base; size_t off;
+  template <typename T> T* take(size_t n) {
+    off = align_up(off, 256);
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += n * sizeof(T);
+    return p;
+  }
+};
+
+void carve(fm_ctx* c, Carver& cv) {
+  const Dims& dm = c->dm;
+  const size_t d = dm.d, B = dm.max_batch;
+  const size_t qkvw = (size_t)(dm.H + 2 * dm.Hkv) * dm.dh, hd = (size_t)dm.H * dm.dh;
+  c->E = cv.take<bf16>((size_t)dm.V * d);
+  for (int s = 0; s < 5; ++s) {
+    c->layers[s].resize(c->cfg.layers[s]);
+    const int lvl = STACK_LEVEL[s];
+    const size_t kvn = B * dm.Hkv * (size_t)(dm.P + dm.cap[lvl]) * dm.dh;
+    for (auto& L : c->layers[s]) {
+      L.Wqkv = cv.take<bf16>(align_up(qkvw, 128) * d);
+      L.Wo = cv.take<bf16>(align_up(d, 128) * hd);
+      L.W1 = cv.take<bf16>(align_up((size_t)dm.dff, 128) * d);
+      L.W2 = cv.take<bf16>(align_up(d, 128) * dm.dff);
+      L.g1 = cv.take<float>(d);
+      L.g2 = cv.take<float>(d);
+      L.K = cv.take<bf16>(kvn);
+      L.V = cv.take<bf16>(kvn);
+    }
+  }
+  c->S_cv = cv.take<bf16>(align_up(d, 128) * 3 * d);
+  c->S_vf = cv.take<bf16>(align_up(d, 128) * 3 * d);
+  c->U_fv = cv.take<bf16>(align_up(3 * d, 128) * d);
+  c->U_vc = cv.take<bf16>(align_up(3 * d, 128) * d);
+  c->W_out = cv.take<bf16>((size_t)dm.Vpad * d);
+  c->headA = cv.take<bf16>((size_t)dm.NH * align_up(d, 128) * d);
+  c->g_out = cv.take<float>(d);
+  c->head_g = cv.take<float>((size_t)dm.NH * d);
+  c->inv_freq = cv.take<double>(dm.dh / 2);
+  // state
+  c->st.L = cv.take<int>(B); c->st.nrow = cv.take<int>(B); c->st.main_tok = cv.take<int>(B);
+  c->st.done = cv.take<int>(B); c->st.t_end = cv.take<int>(B); c->st.plen = cv.take<int>(B);
+  c->st.cand = cv.take<int>(B * dm.R1); c->st.o = cv.take<int>(B * dm.R1);
+  c->st.margin = cv.take<float>(B * dm.R1);
+  c->st.status = cv.take<int>(1); c->st.n_active = cv.take<int>(4); c->st.step = cv.take<int>(1);
+  // activations (row counts padded to 16 so that later tiles never run off the end)
+  const size_t Rc = align_up(B * dm.R1, 16), Rv = align_up(B * dm.mv, 16), Rf = align_up(B * dm.mf, 16);
+  c->xc = cv.take<float>(Rc * d); c->xv = cv.take<float>(Rv * d); c->xf = cv.take<float>(Rf * d);
+  c->qkv = cv.take<float>(Rc * qkvw); c->qbuf = cv.take<float>(Rc * hd);
+  c->logits = cv.take<float>(Rc * dm.Vpad); c->tmp3d = cv.take<float>(Rv * 3 * d);
+  c->a_norm = cv.take<bf16>(Rc * d); c->a_cat = cv.take<bf16>(Rv * 3 * d);
+  c->a_attn = cv.take<bf16>(Rc * hd); c->a_ff = cv.take<bf16>(Rc * dm.dff);
+  c->hc_ring = cv.take<float>(B * FM_RING_C * d); c->hv_ring = cv.take<float>(B * FM_RING_V * d);
+  c->trif_ring = cv.take<float>(B * FM_RING_F * 3 * d); c->triv_ring = cv.take<float>(B * FM_RING_V * 3 * d);
+  c->zc = cv.take<float>(B * FM_RING_C * d); c->zv = cv.take<float>(B * FM_RING_V * d);
+  c->zf = cv.take<float>(B * FM_RING_F * d);
+  // draft
+  const size_t NF = 8 + 9 * (size_t)dm.Ef;
+  c->dh_a = cv.take<bf16>((size_t)dm.NH * B * d); c->dh_y = cv.take<float>((size_t)dm.NH * B * d);
+  c->up_in_v = cv.take<bf16>(align_up((2 + 3 * (size_t)dm.Ef) * B, 16) * d);
+  c->up_in_f = cv.take<bf16>(align_up((size_t)dm.Ef * B, 16) * d);
+  c->feat = cv.take<float>(align_up(NF * B, 16) * d); c->feat_n = cv.take<bf16>(align_up(NF * B, 16) * d);
+  c->dlogits = cv.take<float>(align_up(NF * B, 16) * dm.Vpad);
+  // prefill temporaries
+  c->pre_a = cv.take<bf16>((size_t)PREFILL_CHUNK * d);
+  c->pre_o = cv.take<float>((size_t)PREFILL_CHUNK * 2 * dm.Hkv * dm.dh);
+  c->prompt_off_dev = cv.take<int>(B + 1);
+  c->gen_dev = cv.take<GenOut>(1);
+  c->stats_dev = cv.take<long long>(FM_MAX_DRAFT + 4);
+  cv.off = align_up(cv.off, 256);
+}
+
+#define CUDA_OK(expr) do { if ((expr) != cudaSuccess) return FM_ERR_CUDA; } while (0)
+
+// fp32 host matrix [rows, cols] -> bf16 device rows (nearest-even), staged through `tmp`
+int upload_bf16(bf16* dst, const float* src, size_t n, std::vector<uint16_t>& tmp) {
+  if (src == nullptr) return FM_ERR_INVALID_ARG;
+  tmp.resize(n);
+  for (size_t i = 0; i < n; ++i) {
+    uint32_t u;
+    memcpy(&u, src + i, 4);
+    if ((u & 0x7fffffffu) > 0x7f800000u) { tmp[i] = 0x7fc0; continue; }     // NaN
+    u += 0x7fffu + ((u >> 16) & 1u);
+    tmp[i] = (uint16_t)(u >> 16);
+  }
+  CUDA_OK(cudaMemcpy(dst, tmp.data(), n * 2, cudaMemcpyHostToDevice));
+  return FM_OK;
+}
+int upload_f32(float* dst, const float* src, size_t n) {
+  if (src == nullptr) return FM_ERR_INVALID_ARG;
+  CUDA_OK(cudaMemcpy(dst, src, n * 4, cudaMemcpyHostToDevice));
+  return FM_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// launch helpers
+// ------------------------------------------------------------------------------------------
+#define LAUNCH(ctx, kern, grid, block, smem, ...)                        \
+  do {                                                                   \
+    kern<<<grid, block, smem, (ctx)->stream>>>(__VA_ARGS__);             \
+    (ctx)->launches++;                                                   \
+  } while (0)
+
+void gemm(fm_ctx* c, int mode, const bf16* W, const bf16* A, void* out, int M, int K, int R, int ldo,
+          const int* n_active, int nz = 1, long long sW = 0, long long sA = 0, long long sO = 0) {
+  if (R <= 0) return;
+  GemmArgs g{W, A, out, M, K, R, ldo, sW, sA, sO, n_active};
+  dim3 grid((M + 3) / 4, (R + 15) / 16, nz);
+  switch (mode) {
+    case GEMM_STORE_F32: LAUNCH(c, gemm_simt_kernel<GEMM_STORE_F32>, grid, 128, 0, g); break;
+    case GEMM_ADD_F32: LAUNCH(c, gemm_simt_kernel<GEMM_ADD_F32>, grid, 128, 0, g); break;
+    case GEMM_GELU_BF16: LAUNCH(c, gemm_simt_kernel<GEMM_GELU_BF16>, grid, 128, 0, g); break;
+    default: LAUNCH(c, gemm_simt_kernel<GEMM_STORE_BF16>, grid, 128, 0, g); break;
+  }
+}
+
+__global__ void to_bf16_kernel(const float* __restrict__ x, bf16* __restrict__ out, size_t n) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) out[i] = __float2bfloat16(x[i]);
+}
+
+// rows fed at each level in this pass (n_active[level]); n_active[3] = unfinished sequences
+__global__ void row_count_kernel(Dims dm, SeqState st, int batch) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  int cnt[3] = {0, 0, 0}, act = 0;
+  for (int b = 0; b < batch; ++b) {
+    const int n = st.nrow[b], L = st.L[b];
+    if (n <= 0) continue;
+    act++;
+    for (int l = 0; l < 3; ++l) {
+      const int r = fm_ratio(l);
+      cnt[l] += (L + n - 1) / r - (L + r - 1) / r + 1;
+    }
+  }
+  st.n_active[0] = cnt[0]; st.n_active[1] = cnt[1]; st.n_active[2] = cnt[2]; st.n_active[3] = act;
+}
+
+void attention(fm_ctx* c, int level, int rows, const LayerDev& L) {
+  const Dims& dm = c->dm;
+  dim3 grid(rows, dm.H);
+  if (dm.dh == 32) LAUNCH(c, attn_rows_kernel<32>, grid, 128, 0, dm, c->st, c->batch, level, c->qbuf, L.K, L.V, c->a_attn);
+  else if (dm.dh == 64) LAUNCH(c, attn_rows_kernel<64>, grid, 128, 0, dm, c->st, c->batch, level, c->qbuf, L.K, L.V, c->a_attn);
+  else LAUNCH(c, attn_rows_kernel<128>, grid, 128, 0, dm, c->st, c->batch, level, c->qbuf, L.K, L.V, c->a_attn);
+}
+
+// one stack of pre-norm blocks on the rows of its level (a2/a4/a6/a8/a10)
+void run_stack(fm_ctx* c, int s, float* x, float* stash_ring) {
+  const Dims& dm = c->dm;
+  const int level = STACK_LEVEL[s];
+  const int rows = c->batch * fm_rows_per_seq(dm, level);
+  const int qkvw = (dm.H + 2 * dm.Hkv) * dm.dh, hd = dm.H * dm.dh;
+  const int* na = c->st.n_active + level;
+  const int nl = (int)c->layers[s].size();
+  for (int l = 0; l < nl; ++l) {
+    const LayerDev& L = c->layers[s][l];
+    if (stash_ring != nullptr && l == nl - 1)
+      LAUNCH(c, ring_store_kernel, rows, 128, 0, dm, c->st, c->batch, level, x, stash_ring, dm.d);
+    LAUNCH(c, rmsnorm_kernel, rows, 256, 0, x, L.g1, c->a_norm, dm.d, dm.eps);
+    gemm(c, GEMM_STORE_F32, L.Wqkv, c->a_norm, c->qkv, qkvw, dm.d, rows, qkvw, na);
+    LAUNCH(c, rope_append_kernel, rows, 128, dm.dh * sizeof(float), dm, c->st, c->batch, level, c->qkv, c->inv_freq,
+           c->qbuf, L.K, L.V);
+    attention(c, level, rows, L);
+    gemm(c, GEMM_ADD_F32, L.Wo, c->a_attn, x, dm.d, hd, rows, dm.d, na);
+    LAUNCH(c, rmsnorm_kernel, rows, 256, 0, x, L.g2, c->a_norm, dm.d, dm.eps);
+    gemm(c, GEMM_GELU_BF16, L.W1, c->a_norm, c->a_ff, dm.dff, dm.d, rows, dm.dff, na);
+    gemm(c, GEMM_ADD_F32, L.W2, c->a_ff, x, dm.d, dm.dff, rows, dm.d, na);
+  }
+}
+
+// the verify forward pass over st.cand / st.nrow (a1..a11)
+void forward(fm_ctx* c, float* logits_out) {
+  const Dims& dm = c->dm;
+  const int B = c->batch, d = dm.d;
+  const int Rc = B * dm.R1, Rv = B * dm.mv, Rf = B * dm.mf;
+  const int* na = c->st.n_active;
+  LAUNCH(c, row_count_kernel, 1, 32, 0, dm, c->st, B);
+  LAUNCH(c, embed_kernel, Rc, 128, 0, dm, c->st, B, c->E, c->xc);
+  run_stack(c, 0, c->xc, nullptr);
+  LAUNCH(c, ring_store_kernel, Rc, 128, 0, dm, c->st, B, 0, c->xc, c->hc_ring, d);
+  LAUNCH(c, shorten_gather_kernel, Rv, 128, 0, dm, c->st, B, 1, c->hc_ring, c->a_cat);
+  gemm(c, GEMM_STORE_F32, c->S_cv, c->a_cat, c->xv, d, 3 * d, Rv, d, na + 1);
+  run_stack(c, 1, c->xv, nullptr);
+  LAUNCH(c, ring_store_kernel, Rv, 128, 0, dm, c->st, B, 1, c->xv, c->hv_ring, d);
+  LAUNCH(c, shorten_gather_kernel, Rf, 128, 0, dm, c->st, B, 2, c->hv_ring, c->a_cat);
+  gemm(c, GEMM_STORE_F32, c->S_vf, c->a_cat, c->xf, d, 3 * d, Rf, d, na + 2);
+  run_stack(c, 2, c->xf, c->zf);
+  LAUNCH(c, to_bf16_kernel, (Rf * d + 255) / 256, 256, 0, c->xf, c->a_norm, (size_t)Rf * d);
+  gemm(c, GEMM_STORE_F32, c->U_fv, c->a_norm, c->tmp3d, 3 * d, d, Rf, 3 * d, na + 2);
+  LAUNCH(c, ring_store_kernel, Rf, 128, 0, dm, c->st, B, 2, c->tmp3d, c->trif_ring, 3 * d);
+  LAUNCH(c, upsample_add_kernel, Rv, 128, 0, dm, c->st, B, 1, c->hv_ring, c->trif_ring, c->xv);
+  run_stack(c, 3, c->xv, c->zv);
+  LAUNCH(c, to_bf16_kernel, (Rv * d + 255) / 256, 256, 0, c->xv, c->a_norm, (size_t)Rv * d);
+  gemm(c, GEMM_STORE_F32, c->U_vc, c->a_norm, c->tmp3d, 3 * d, d, Rv, 3 * d, na + 1);
+  LAUNCH(c, ring_store_kernel, Rv, 128, 0, dm, c->st, B, 1, c->tmp3d, c->triv_ring, 3 * d);
+  LAUNCH(c, upsample_add_kernel, Rc, 128, 0, dm, c->st, B, 0, c->hc_ring, c->triv_ring, c->xc);
+  run_stack(c, 4, c->xc, c->zc);
+  LAUNCH(c, rmsnorm_kernel, Rc, 256, 0, c->xc, c->g_out, c->a_norm, d, dm.eps);
+  gemm(c, GEMM_STORE_F32, c->W_out, c->a_norm, c->logits, dm.V, d, Rc, dm.Vpad, na);
+  LAUNCH(c, verify_top2_kernel, Rc, 256, 0, dm, c->st, B, c->logits, logits_out);
+}
+
+// a13: draft heads on the stashed split-node hiddens
+void draft(fm_ctx* c, float* logits_out, float* margin_out) {
+  const Dims& dm = c->dm;
+  const int B = c->batch, d = dm.d;
+  if (dm.D > 0) {
+    const int dpad = round_up(d, 128);
+    const int NF = 8 + 9 * dm.Ef;
+    const int* na = c->st.n_active + 3;
+    LAUNCH(c, draft_prep_kernel, dim3(B, dm.NH), 256, 0, dm, c->st, B, c->zc, c->zv, c->zf, c->head_g, c->dh_a);
+    gemm(c, GEMM_STORE_F32, c->headA, c->dh_a, c->dh_y, d, d, B, d, na, dm.NH, (long long)dpad * d,
+         (long long)dm.max_batch * d, (long long)dm.max_batch * d);
+    LAUNCH(c, draft_residual_kernel, dim3(B, dm.NH), 128, 0, dm, c->st, B, c->zc, c->zv, c->zf, c->dh_y, c->feat,
+           c->up_in_v, c->up_in_f);
+    gemm(c, GEMM_STORE_BF16, c->U_fv, c->up_in_f, c->up_in_v + (size_t)2 * B * d, 3 * d, d, dm.Ef * B, 3 * d, na);
+    gemm(c, GEMM_STORE_F32, c->U_vc, c->up_in_v, c->feat + (size_t)2 * B * d, 3 * d, d, (2 + 3 * dm.Ef) * B, 3 * d, na);
+    LAUNCH(c, rmsnorm_kernel, NF * B, 256, 0, c->feat, c->g_out, c->feat_n, d, dm.eps);
+    gemm(c, GEMM_STORE_F32, c->W_out, c->feat_n, c->dlogits, dm.V, d, NF * B, dm.Vpad, na);
+  }
+  LAUNCH(c, draft_pick_kernel, dim3(B, dm.R1), 256, 0, dm, c->st, B, c->dlogits, logits_out, margin_out);
+}
+
+__global__ void verify_load_kernel(Dims dm, SeqState st, int batch, const int* __restrict__ cand) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= batch * dm.R1) return;
+  const int b = i / dm.R1, j = i - b * dm.R1;
+  const int t = cand[i];
+  if (j == 0 && st.nrow[b] > 0 && t != st.main_tok[b]) atomicExch(st.status, FM_ERR_INVALID_ARG);
+  st.cand[i] = t;
+}
+
+__global__ void init_state_kernel(Dims dm, SeqState st, int batch, const int* __restrict__ prompt_off) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= dm.max_batch) return;
+  st.L[b] = 0; st.nrow[b] = 0; st.main_tok[b] = dm.n_bins + 2; st.done[b] = b < batch ? 0 : 1;
+  st.plen[b] = b < batch ? prompt_off[b + 1] - prompt_off[b] : 0;
+  st.t_end[b] = dm.max_tokens - dm.D - 2;
+  if (b == 0) { *st.step = 0; }
+}
+
+__global__ void set_limits_kernel(Dims dm, SeqState st, int batch, const int* __restrict__ max_faces) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= batch) return;
+  const int cap = dm.max_tokens - dm.D - 2;
+  const long long want = (long long)st.plen[b] + 9ll * max_faces[b];
+  st.t_end[b] = want < cap ? (int)want : cap;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------
+// C ABI
+// ------------------------------------------------------------------------------------------
+extern "C" {
+
+const char* fm_strerror(int code) {
+  switch (code) {
+    case FM_OK: return "ok";
+    case FM_ERR_INVALID_ARG: return "invalid argument";
+    case FM_ERR_BAD_STATE: return "call out of order";
+    case FM_ERR_CAPACITY: return "capacity exceeded";
+    case FM_ERR_CUDA: return "CUDA runtime error";
+    case FM_ERR_TIMEOUT: return "device-side wait timed out";
+    case FM_ERR_UNSUPPORTED: return "unsupported shape";
+    default: return "unknown error";
+  }
+}
+
+size_t fm_workspace_bytes(const fm_config* cfg) {
+  if (check_config(cfg) != FM_OK) return 0;
+  fm_ctx tmp{};
+  tmp.cfg = *cfg;
+  tmp.dm = make_dims(*cfg);
+  Carver cv{nullptr, 0};
+  carve(&tmp, cv);
+  return cv.off;
+}
+
+int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, size_t workspace_bytes, void* cuda_stream,
+              fm_ctx** out) {
+  if (out == nullptr) return FM_ERR_INVALID_ARG;
+  *out = nullptr;
+  int rc = check_config(cfg);
+  if (rc != FM_OK) return rc;
+  if (w == nullptr || dev_workspace == nullptr) return FM_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(dev_workspace) & 255u) != 0) return FM_ERR_INVALID_ARG;
+  const size_t need = fm_workspace_bytes(cfg);
+  if (workspace_bytes < need) return FM_ERR_CAPACITY;
+  for (int s = 0; s < 5; ++s) if (w->stack[s] == nullptr) return FM_ERR_INVALID_ARG;
+
+  fm_ctx* c = new (std::nothrow) fm_ctx{};
+  if (c == nullptr) return FM_ERR_INVALID_ARG;
+  c->cfg = *cfg;
+  c->dm = make_dims(*cfg);
+  c->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  c->ws = static_cast<char*>(dev_workspace);
+  c->ws_bytes = need;
+  Carver cv{c->ws, 0};
+  carve(c, cv);
+  const Dims& dm = c->dm;
+  const size_t d = dm.d, qkvw = (size_t)(dm.H + 2 * dm.Hkv) * dm.dh, hd = (size_t)dm.H * dm.dh;
+
+#define TRY(expr) do { rc = (expr); if (rc != FM_OK) { delete c; return rc; } } while (0)
+#define TRYCUDA(expr) do { if ((expr) != cudaSuccess) { delete c; return FM_ERR_CUDA; } } while (0)
+  // everything that is not explicitly uploaded (row padding, caches, rings, state) starts at zero
+  TRYCUDA(cudaMemset(c->ws, 0, need));
+  std::vector<uint16_t> tmp;
+  TRY(upload_bf16(c->E, w->E, (size_t)dm.V * d, tmp));
+  for (int s = 0; s < 5; ++s)
+    for (size_t l = 0; l < c->layers[s].size(); ++l) {
+      const fm_layer_weights& hw = w->stack[s][l];
+      LayerDev& L = c->layers[s][l];
+      TRY(upload_bf16(L.Wqkv, hw.Wqkv, qkvw * d, tmp));
+      TRY(upload_bf16(L.Wo, hw.Wo, d * hd, tmp));
+      TRY(upload_bf16(L.W1, hw.W1, (size_t)dm.dff * d, tmp));
+      TRY(upload_bf16(L.W2, hw.W2, d * dm.dff, tmp));
+      TRY(upload_f32(L.g1, hw.g1, d));
+      TRY(upload_f32(L.g2, hw.g2, d));
+    }
+  TRY(upload_bf16(c->S_cv, w->S_cv, d * 3 * d, tmp));
+  TRY(upload_bf16(c->S_vf, w->S_vf, d * 3 * d, tmp));
+  TRY(upload_bf16(c->U_fv, w->U_fv, 3 * d * d, tmp));
+  TRY(upload_bf16(c->U_vc, w->U_vc, 3 * d * d, tmp));
+  TRY(upload_bf16(c->W_out, w->W_out, (size_t)dm.V * d, tmp));
+  TRY(upload_f32(c->g_out, w->g_out, d));
+  const size_t dpad = align_up(d, 128);
+  for (int h = 0; h < dm.NH; ++h) {
+    const float* A = h < 2 ? w->head_c_A[h] : h < 4 ? w->head_v_A[h - 2] : w->head_f_A[h - 4];
+    const float* g = h < 2 ? w->head_c_g[h] : h < 4 ? w->head_v_g[h - 2] : w->head_f_g[h - 4];
+    if (dm.D == 0 && (A == nullptr || g == nullptr)) continue;     // no drafts: heads are unused
+    TRY(upload_bf16(c->headA + (size_t)h * dpad * d, A, d * d, tmp));
+    TRY(upload_f32(c->head_g + (size_t)h * d, g, d));
+  }
+  std::vector<double> freq(dm.dh / 2);
+  for (int i = 0; i < dm.dh / 2; ++i)
+    freq[i] = dm.theta != 0.f ? pow((double)dm.theta, -2.0 * (double)i / (double)dm.dh) : 0.0;
+  TRYCUDA(cudaMemcpy(c->inv_freq, freq.data(), freq.size() * sizeof(double), cudaMemcpyHostToDevice));
+  TRYCUDA(cudaHostAlloc(reinterpret_cast<void**>(&c->host_done), 64, cudaHostAllocMapped));
+  *c->host_done = 0;
+  TRYCUDA(cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->host_done_dev), c->host_done, 0));
+  TRYCUDA(cudaDeviceSynchronize());
+#undef TRY
+#undef TRYCUDA
+  c->batch = 0;
+  c->phase = 0;
+  c->launches = 0;
+  *out = c;
+  return FM_OK;
+}
+
+int fm_destroy(fm_ctx* c) {
+  if (c == nullptr) return FM_ERR_INVALID_ARG;
+  cudaStreamSynchronize(c->stream);
+  if (c->host_done != nullptr) cudaFreeHost(c->host_done);
+  delete c;
+  return FM_OK;
+}
+
+int fm_prefill(fm_ctx* c, int32_t batch, const float* cond, const int32_t* prompt, const int32_t* prompt_off) {
+  if (c == nullptr || prompt_off == nullptr) return FM_ERR_INVALID_ARG;
+  const Dims& dm = c->dm;
+  if (batch < 1) return FM_ERR_INVALID_ARG;
+  if (batch > dm.max_batch) return FM_ERR_CAPACITY;
+  if (dm.P > 0 && cond == nullptr) return FM_ERR_INVALID_ARG;
+  int longest = 0;
+  for (int b = 0; b < batch; ++b) {
+    const int n = prompt_off[b + 1] - prompt_off[b];
+    if (n < 0 || n % 9 != 0) return FM_ERR_INVALID_ARG;
+    if (1 + n + dm.D + 2 > dm.max_tokens) return FM_ERR_CAPACITY;
+    longest = n > longest ? n : longest;
+  }
+  if (prompt_off[batch] > 0 && prompt == nullptr) return FM_ERR_INVALID_ARG;
+  c->batch = batch;
+  c->plen_host.assign(batch, 0);
+  for (int b = 0; b < batch; ++b) c->plen_host[b] = prompt_off[b + 1] - prompt_off[b];
+  CUDA_OK(cudaMemcpyAsync(c->prompt_off_dev, prompt_off, (batch + 1) * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  CUDA_OK(cudaStreamSynchronize(c->stream));       // prompt_off is caller memory: finish reading it now
+  LAUNCH(c, init_state_kernel, (dm.max_batch + 127) / 128, 128, 0, dm, c->st, batch, c->prompt_off_dev);
+  // per-layer prefix keys/values: K_pre = Wk rms(c, g1), V_pre = Wv rms(c, g1), no rotation
+  const int rows_total = batch * dm.P, kvw = 2 * dm.Hkv * dm.dh;
+  for (int r0 = 0; r0 < rows_total; r0 += PREFILL_CHUNK) {
+    const int rows = rows_total - r0 < PREFILL_CHUNK ? rows_total - r0 : PREFILL_CHUNK;
+    for (int s = 0; s < 5; ++s)
+      for (auto& L : c->layers[s]) {
+        LAUNCH(c, rmsnorm_kernel, rows, 256, 0, cond + (size_t)r0 * dm.d, L.g1, c->pre_a, dm.d, dm.eps);
+        gemm(c, GEMM_STORE_F32, L.Wqkv + (size_t)dm.H * dm.dh * dm.d, c->pre_a, c->pre_o, kvw, dm.d, rows, kvw, nullptr);
+        LAUNCH(c, prefix_store_kernel, rows, 128, 0, dm, STACK_LEVEL[s], r0, c->pre_o, L.K, L.V);
+      }
+  }
+  // BOS + prompt through the multi-row forward, D+1 rows per sequence and pass, all rows kept
+  const int passes = (1 + longest + dm.R1 - 1) / dm.R1;
+  for (int i = 0; i < passes; ++i) {
+    LAUNCH(c, prefill_feed_kernel, batch, 32, 0, dm, c->st, batch, prompt, c->prompt_off_dev);
+    forward(c, nullptr);
+    LAUNCH(c, prefill_advance_kernel, (batch + 127) / 128, 128, 0, dm, c->st, batch);
+  }
+  LAUNCH(c, arm_kernel, (batch + 127) / 128, 128, 0, dm, c->st, batch);
+  LAUNCH(c, row_count_kernel, 1, 32, 0, dm, c->st, batch);
+  CUDA_OK(cudaGetLastError());
+  c->phase = 1;
+  return FM_OK;
+}
+
+int fm_set_max_faces(fm_ctx* c, const int32_t* max_faces) {
+  if (c == nullptr || max_faces == nullptr) return FM_ERR_INVALID_ARG;
+  if (c->phase < 1) return FM_ERR_BAD_STATE;
+  for (int b = 0; b < c->batch; ++b) if (max_faces[b] < 0) return FM_ERR_INVALID_ARG;
+  int* tmp = reinterpret_cast<int*>(c->pre_o);       // scratch that no pass is using now
+  CUDA_OK(cudaMemcpyAsync(tmp, max_faces, c->batch * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  LAUNCH(c, set_limits_kernel, (c->batch + 127) / 128, 128, 0, c->dm, c->st, c->batch, tmp);
+  LAUNCH(c, arm_kernel, (c->batch + 127) / 128, 128, 0, c->dm, c->st, c->batch);
+  LAUNCH(c, row_count_kernel, 1, 32, 0, c->dm, c->st, c->batch);
+  CUDA_OK(cudaStreamSynchronize(c->stream));       // max_faces is caller memory
+  return FM_OK;
+}
+
+int fm_draft(fm_ctx* c, int32_t* cand, float* draft_logits, float* draft_margin) {
+  if (c == nullptr) return FM_ERR_INVALID_ARG;
+  if (c->phase < 1) return FM_ERR_BAD_STATE;
+  draft(c, draft_logits, draft_margin);
+  const int n = c->batch * c->dm.R1;
+  if (cand != nullptr) LAUNCH(c, copy_i32_kernel, (n + 127) / 128, 128, 0, c->st.cand, cand, n);
+  CUDA_OK(cudaGetLastError());
+  return FM_OK;
+}
+
+int fm_verify(fm_ctx* c, const int32_t* cand, int32_t* argmax, float* logits, float* margin) {
+  if (c == nullptr || cand == nullptr) return FM_ERR_INVALID_ARG;
+  if (c->phase < 1) return FM_ERR_BAD_STATE;
+  const int n = c->batch * c->dm.R1;
+  LAUNCH(c, verify_load_kernel, (n + 127) / 128, 128, 0, c->dm, c->st, c->batch, cand);
+  forward(c, logits);
+  if (argmax != nullptr) LAUNCH(c, copy_i32_kernel, (n + 127) / 128, 128, 0, c->st.o, argmax, n);
+  if (margin != nullptr) LAUNCH(c, copy_f32_kernel, (n + 127) / 128, 128, 0, c->st.margin, margin, n);
+  CUDA_OK(cudaGetLastError());
+  c->phase = 2;
+  return FM_OK;
+}
+
+int fm_accept(fm_ctx* c, const int32_t* force_len, const int32_t* force_tok, int32_t* n_acc, int32_t* emitted,
+              int32_t* kv_len) {
+  if (c == nullptr) return FM_ERR_INVALID_ARG;
+  if (c->phase != 2) return FM_ERR_BAD_STATE;
+  LAUNCH(c, accept_kernel, (c->batch * 32 + 127) / 128, 128, 0, c->dm, c->st, c->batch, force_len, force_tok, n_acc,
+         emitted, kv_len, (const GenOut*)nullptr);
+  LAUNCH(c, row_count_kernel, 1, 32, 0, c->dm, c->st, c->batch);
+  CUDA_OK(cudaGetLastError());
+  c->phase = 1;
+  return FM_OK;
+}
+
+int fm_generate(fm_ctx* c, int32_t max_faces, int32_t* out_tok, int32_t out_stride, int32_t* out_len,
+                const fm_teacher* teacher, int32_t plain, fm_stats* stats) {
+  if (c == nullptr || max_faces < 0) return FM_ERR_INVALID_ARG;
+  if (c->phase < 1) return FM_ERR_BAD_STATE;
+  const Dims& dm = c->dm;
+  if (out_tok != nullptr && (out_len == nullptr || out_stride < 9 * max_faces)) return FM_ERR_CAPACITY;
+  if (teacher != nullptr && (teacher->truth == nullptr || teacher->truth_stride <= 0 ||
+                             (teacher->keep != nullptr && teacher->n_sched <= 0))) return FM_ERR_INVALID_ARG;
+  for (int b = 0; b < c->batch; ++b)
+    if ((long long)c->plen_host[b] + 9ll * max_faces + dm.D + 2 > dm.max_tokens) return FM_ERR_CAPACITY;
+  std::vector<int> lim(c->batch, max_faces);
+  int rc = fm_set_max_faces(c, lim.data());
+  if (rc != FM_OK) return rc;
+  GenOut g{};
+  g.out_tok = out_tok; g.out_stride = out_stride; g.out_len = out_len;
+  if (teacher != nullptr) { g.truth = teacher->truth; g.truth_stride = teacher->truth_stride; g.keep = teacher->keep; g.n_sched = teacher->n_sched; }
+  g.plain = plain;
+  g.stats = c->stats_dev;
+  g.host_done = c->host_done_dev;
+  CUDA_OK(cudaMemcpyAsync(c->gen_dev, &g, sizeof(g), cudaMemcpyHostToDevice, c->stream));
+  CUDA_OK(cudaMemsetAsync(c->stats_dev, 0, (FM_MAX_DRAFT + 4) * sizeof(long long), c->stream));
+  if (out_len != nullptr) CUDA_OK(cudaMemsetAsync(out_len, 0, c->batch * sizeof(int), c->stream));
+  CUDA_OK(cudaStreamSynchronize(c->stream));       // `g` lives on this stack frame
+  cudaEvent_t e0, e1;
+  CUDA_OK(cudaEventCreate(&e0));
+  CUDA_OK(cudaEventCreate(&e1));
+  CUDA_OK(cudaEventRecord(e0, c->stream));
+  *c->host_done = c->batch;
+  // upper bound on passes: every pass emits at least one token per unfinished sequence
+  const long long max_steps = 9ll * max_faces + 1;
+  const int poll = 8;
+  long long steps = 0;
+  bool finished = false;
+  while (!finished && steps < max_steps + poll) {
+    for (int i = 0; i < poll; ++i) {
+      draft(c, nullptr, nullptr);
+      if (teacher != nullptr) LAUNCH(c, teacher_edit_kernel, c->batch, 32, 0, dm, c->st, c->batch, c->gen_dev);
+      forward(c, nullptr);
+      LAUNCH(c, accept_kernel, (c->batch * 32 + 127) / 128, 128, 0, dm, c->st, c->batch, (const int*)nullptr,
+             (const int*)nullptr, (int*)nullptr, (int*)nullptr, (int*)nullptr, (const GenOut*)c->gen_dev);
+      LAUNCH(c, row_count_kernel, 1, 32, 0, dm, c->st, c->batch);
+      LAUNCH(c, step_end_kernel, 1, 32, 0, c->st, (const GenOut*)c->gen_dev);
+      ++steps;
+    }
+    CUDA_OK(cudaStreamSynchronize(c->stream));
+    finished = *c->host_done == 0;
+  }
+  CUDA_OK(cudaEventRecord(e1, c->stream));
+  CUDA_OK(cudaEventSynchronize(e1));
+  float ms = 0.f;
+  cudaEventElapsedTime(&ms, e0, e1);
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  if (stats != nullptr) {
+    long long h[FM_MAX_DRAFT + 4];
+    CUDA_OK(cudaMemcpy(h, c->stats_dev, sizeof(h), cudaMemcpyDeviceToHost));
+    memset(stats, 0, sizeof(*stats));
+    stats->steps = h[0];
+    stats->emitted = h[1];
+    for (int a = 0; a < FM_MAX_DRAFT + 2; ++a) stats->accept_hist[a] = h[2 + a];
+    stats->ms = ms;
+  }
+  c->phase = 1;
+  return finished ? FM_OK : FM_ERR_TIMEOUT;
+}
+
+double fm_verify_bytes(const fm_ctx* c, int32_t batch, const int32_t* kv_len) {
+  if (c == nullptr || kv_len == nullptr || batch < 1) return 0.0;
+  const Dims& dm = c->dm;
+  const double d = dm.d;
+  const double layer_w = 2.0 * ((double)(dm.H + 2 * dm.Hkv) * dm.dh * d + d * dm.H * dm.dh + 2.0 * d * dm.dff);
+  bool has[3] = {false, false, false};
+  double kv[3] = {0, 0, 0};
+  for (int b = 0; b < batch; ++b) {
+    const int L = kv_len[b * 3];
+    for (int l = 0; l < 3; ++l) {
+      const int r = fm_ratio(l);
+      const int p0 = (L + r - 1) / r, p1 = (L + dm.D) / r;
+      if (p1 < p0) continue;
+      has[l] = true;
+      const int lo = dm.window[l] > 0 ? (p0 - dm.window[l] + 1 > 0 ? p0 - dm.window[l] + 1 : 0) : 0;
+      kv[l] += (double)(dm.P + p1 - lo + 1) * 2.0 * dm.Hkv * dm.dh * 2.0;     // K and V, bf16
+    }
+  }
+  double bytes = 2.0 * d * dm.V;                                              // output matrix
+  for (int s = 0; s < 5; ++s) {
+    const int l = STACK_LEVEL[s];
+    if (has[l]) bytes += c->cfg.layers[s] * (layer_w + kv[l]);
+  }
+  if (has[1]) bytes += 2.0 * 2.0 * 3.0 * d * d;                               // S_cv + U_vc
+  if (has[2]) bytes += 2.0 * 2.0 * 3.0 * d * d;                               // S_vf + U_fv
+  return bytes;
+}
+
+int64_t fm_launch_count(const fm_ctx* c) { return c ? c->launches : 0; }
+
+int fm_device_status(fm_ctx* c) {
+  if (c == nullptr) return FM_ERR_INVALID_ARG;
+  int s = 0;
+  if (cudaMemcpyAsync(&s, c->st.status, sizeof(int), cudaMemcpyDeviceToHost, c->stream) != cudaSuccess) return FM_ERR_CUDA;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return FM_ERR_CUDA;
+  return s;
+}
+
+}  // extern "C"

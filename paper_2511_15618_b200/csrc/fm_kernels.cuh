@@ -1,0 +1,447 @@
+// Element-wise, row-wise and bookkeeping kernels of the decode step.
+#pragma once
+#include "fm_common.cuh"
+
+// ------------------------------------------------------------------------------------------
+// block reductions (blockDim.x multiple of 32, <= 1024)
+// ------------------------------------------------------------------------------------------
+__device__ inline float block_sum(float v, float* sh) {
+  v = warp_sum(v);
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31, nw = blockDim.x >> 5;
+  __syncthreads();
+  if (l == 0) sh[w] = v;
+  __syncthreads();
+  float t = 0.f;
+  for (int i = 0; i < nw; ++i) t += sh[i];          // fixed order: same result in every thread
+  return t;
+}
+
+// ------------------------------------------------------------------------------------------
+// a1. candidate embedding: x[row] = E[cand[b][j]]  (zeros for rows that are not fed)
+// ------------------------------------------------------------------------------------------
+__global__ void embed_kernel(Dims dm, SeqState st, int batch, const bf16* __restrict__ E, float* __restrict__ x) {
+  const int row = blockIdx.x;
+  int b, p;
+  const bool valid = fm_row_map(dm, st, batch, 0, row, b, p);
+  int tok = 0;
+  if (valid) {
+    tok = st.cand[b * dm.R1 + (row - b * dm.R1)];
+    if (tok < 0 || tok >= dm.V) {                    // never index outside the table
+      if (threadIdx.x == 0) atomicExch(st.status, -1);
+      tok = dm.n_bins + 2;
+    }
+  }
+  for (int i = threadIdx.x; i < dm.d; i += blockDim.x)
+    x[(size_t)row * dm.d + i] = valid ? __bfloat162float(E[(size_t)tok * dm.d + i]) : 0.f;
+}
+
+// ------------------------------------------------------------------------------------------
+// RMSNorm of fp32 rows -> bf16 GEMM operand rows:  out = x / sqrt(mean(x^2)+eps) * g
+// ------------------------------------------------------------------------------------------
+__global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ g, bf16* __restrict__ out,
+                               int d, float eps) {
+  __shared__ float sh[32];
+  const float* xr = x + (size_t)blockIdx.x * d;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) { const float v = xr[i]; ss += v * v; }
+  ss = block_sum(ss, sh);
+  const float inv = rsqrtf(ss / (float)d + eps);
+  for (int i = threadIdx.x; i < d; i += blockDim.x)
+    out[(size_t)blockIdx.x * d + i] = __float2bfloat16(xr[i] * inv * g[i]);
+}
+
+// ------------------------------------------------------------------------------------------
+// RoPE on q and k (rotate-half pairs (i, i+dh/2), angle = pos * theta^(-2i/dh), evaluated in
+// double), then append k, v to the level's cache at slot P + pos % cap.
+// qkv: fp32 [rows, (H+2Hkv)*dh]; q_out: fp32 [rows, H*dh]; caches: bf16 [B, Hkv, slots, dh].
+// ------------------------------------------------------------------------------------------
+__global__ void rope_append_kernel(Dims dm, SeqState st, int batch, int level, const float* __restrict__ qkv,
+                                   const double* __restrict__ inv_freq, float* __restrict__ q_out,
+                                   bf16* __restrict__ Kc, bf16* __restrict__ Vc) {
+  const int row = blockIdx.x;
+  int b, p;
+  const bool valid = fm_row_map(dm, st, batch, level, row, b, p);
+  const int H = dm.H, Hkv = dm.Hkv, dh = dm.dh, half = dh / 2;
+  const int ldq = (H + 2 * Hkv) * dh;
+  const float* src = qkv + (size_t)row * ldq;
+  const int slots = dm.P + dm.cap[level];
+  const int slot = dm.P + (p % dm.cap[level]);
+  extern __shared__ float cs[];                     // cos[half], sin[half]
+  for (int i = threadIdx.x; i < half; i += blockDim.x) {
+    double s = 0.0, c = 1.0;
+    if (dm.theta != 0.f) sincos((double)p * inv_freq[i], &s, &c);
+    cs[i] = (float)c;
+    cs[half + i] = (float)s;
+  }
+  __syncthreads();
+  // q and k heads: one thread per rotation pair
+  const int pairs = (H + Hkv) * half;
+  for (int t = threadIdx.x; t < pairs; t += blockDim.x) {
+    const int head = t / half, i = t - head * half;
+    const float x1 = src[head * dh + i], x2 = src[head * dh + half + i];
+    const float c = cs[i], s = cs[half + i];
+    const float y1 = x1 * c - x2 * s, y2 = x2 * c + x1 * s;
+    if (head < H) {
+      q_out[(size_t)row * H * dh + head * dh + i] = valid ? y1 : 0.f;
+      q_out[(size_t)row * H * dh + head * dh + half + i] = valid ? y2 : 0.f;
+    } else if (valid) {
+      const int hk = head - H;
+      bf16* dst = Kc + (((size_t)b * Hkv + hk) * slots + slot) * dh;
+      dst[i] = __float2bfloat16(y1);
+      dst[half + i] = __float2bfloat16(y2);
+    }
+  }
+  if (valid) {
+    const float* vsrc = src + (H + Hkv) * dh;
+    for (int t = threadIdx.x; t < Hkv * dh; t += blockDim.x) {
+      const int hk = t / dh, i = t - hk * dh;
+      Vc[(((size_t)b * Hkv + hk) * slots + slot) * dh + i] = __float2bfloat16(vsrc[t]);
+    }
+  }
+}
+
+// prefix keys/values of one layer: kv fp32 [rows, 2*Hkv*dh] (rows = chunk of b*P+j) -> slots [0,P)
+__global__ void prefix_store_kernel(Dims dm, int level, int row0, const float* __restrict__ kv,
+                                    bf16* __restrict__ Kc, bf16* __restrict__ Vc) {
+  const int r = row0 + blockIdx.x;
+  const int b = r / dm.P, j = r - b * dm.P;
+  const int slots = dm.P + dm.cap[level];
+  const int n = dm.Hkv * dm.dh;
+  const float* src = kv + (size_t)blockIdx.x * 2 * n;
+  for (int t = threadIdx.x; t < n; t += blockDim.x) {
+    const int hk = t / dm.dh, i = t - hk * dm.dh;
+    const size_t o = (((size_t)b * dm.Hkv + hk) * slots + j) * dm.dh + i;
+    Kc[o] = __float2bfloat16(src[t]);
+    Vc[o] = __float2bfloat16(src[n + t]);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// hourglass carry rings
+// ------------------------------------------------------------------------------------------
+// ring[b][p % ring][:] = x[row][:] for rows that are fed (width = floats per entry)
+__global__ void ring_store_kernel(Dims dm, SeqState st, int batch, int level, const float* __restrict__ x,
+                                  float* __restrict__ ring, int width) {
+  const int row = blockIdx.x;
+  int b, p;
+  if (!fm_row_map(dm, st, batch, level, row, b, p)) return;
+  const int rs = fm_ring(level);
+  float* dst = ring + ((size_t)b * rs + (p % rs)) * width;
+  const float* src = x + (size_t)row * width;
+  for (int i = threadIdx.x; i < width; i += blockDim.x) dst[i] = src[i];
+}
+
+// a3/a5 shorten, gather half: row v of level `level_out` <- bf16 [h_{3v-2}; h_{3v-1}; h_{3v}] from
+// the ring of the level below (zeros for negative positions and for rows that are not fed)
+__global__ void shorten_gather_kernel(Dims dm, SeqState st, int batch, int level_out, const float* __restrict__ ring,
+                                      bf16* __restrict__ out) {
+  const int row = blockIdx.x;
+  int b, v;
+  const bool valid = fm_row_map(dm, st, batch, level_out, row, b, v);
+  const int rs = fm_ring(level_out - 1), d = dm.d;
+  for (int part = 0; part < 3; ++part) {
+    const int pos = 3 * v - 2 + part;
+    const bool ok = valid && pos >= 0;
+    const float* src = ring + ((size_t)b * rs + ((pos + rs) % rs)) * d;
+    for (int i = threadIdx.x; i < d; i += blockDim.x)
+      out[(size_t)row * 3 * d + part * d + i] = __float2bfloat16(ok ? src[i] : 0.f);
+  }
+}
+
+// a7/a9 upsample, residual half: x[row] = h_ring[b][p] + tri_ring[b][p/3][(p%3)*d ...]
+__global__ void upsample_add_kernel(Dims dm, SeqState st, int batch, int level, const float* __restrict__ h_ring,
+                                    const float* __restrict__ tri_ring, float* __restrict__ x) {
+  const int row = blockIdx.x;
+  int b, p;
+  const bool valid = fm_row_map(dm, st, batch, level, row, b, p);
+  const int rs = fm_ring(level), rsu = fm_ring(level + 1), d = dm.d;
+  const float* h = h_ring + ((size_t)b * rs + (p % rs)) * d;
+  const float* t = tri_ring + ((size_t)b * rsu + ((p / 3) % rsu)) * 3 * d + (p % 3) * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) x[(size_t)row * d + i] = valid ? h[i] + t[i] : 0.f;
+}
+
+// ------------------------------------------------------------------------------------------
+// a11. masked top-2 of the logits rows: ids >= n_bins forbidden, except EOS where a face
+// starts (target index % 9 == 0) when allowed; ties go to the lowest id.
+// ------------------------------------------------------------------------------------------
+struct Top2 { float v1; int i1; float v2; };
+__device__ inline void top2_push(Top2& t, float v, int i) {
+  if (v > t.v1 || (v == t.v1 && i < t.i1)) { t.v2 = t.v1; t.v1 = v; t.i1 = i; }
+  else if (v > t.v2) t.v2 = v;
+}
+__device__ inline void top2_merge(Top2& a, const Top2& b) {
+  if (b.i1 < 0) return;
+  if (a.i1 < 0) { a = b; return; }
+  if (b.v1 > a.v1 || (b.v1 == a.v1 && b.i1 < a.i1)) { const float lose = a.v1; a.v1 = b.v1; a.i1 = b.i1; a.v2 = fmaxf(fmaxf(a.v2, b.v2), lose); }
+  else a.v2 = fmaxf(fmaxf(a.v2, b.v2), b.v1);
+}
+__device__ inline Top2 block_top2(const float* __restrict__ z, const Dims& dm, int target_index) {
+  Top2 t{-INFINITY, -1, -INFINITY};
+  const bool eos_ok = dm.allow_eos && (target_index % 9 == 0);
+  const int n = dm.n_bins + (eos_ok ? 2 : 0);
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    if (i == dm.n_bins) continue;                    // BOS
+    top2_push(t, z[i], i);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    Top2 u;
+    u.v1 = __shfl_xor_sync(0xffffffffu, t.v1, o);
+    u.i1 = __shfl_xor_sync(0xffffffffu, t.i1, o);
+    u.v2 = __shfl_xor_sync(0xffffffffu, t.v2, o);
+    top2_merge(t, u);
+  }
+  __shared__ Top2 sh[32];
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31, nw = blockDim.x >> 5;
+  __syncthreads();
+  if (l == 0) sh[w] = t;
+  __syncthreads();
+  Top2 r = sh[0];
+  for (int i = 1; i < nw; ++i) top2_merge(r, sh[i]);
+  return r;
+}
+
+__global__ void verify_top2_kernel(Dims dm, SeqState st, int batch, const float* __restrict__ logits,
+                                   float* __restrict__ logits_out) {
+  const int row = blockIdx.x;
+  int b, p;
+  const bool valid = fm_row_map(dm, st, batch, 0, row, b, p);
+  const int j = row % dm.R1;
+  const int bb = row / dm.R1;
+  if (bb >= batch) return;
+  if (logits_out != nullptr)
+    for (int i = threadIdx.x; i < dm.V; i += blockDim.x)
+      logits_out[(size_t)row * dm.V + i] = valid ? logits[(size_t)row * dm.Vpad + i] : 0.f;
+  if (!valid) {
+    if (threadIdx.x == 0) { st.o[bb * dm.R1 + j] = -1; st.margin[bb * dm.R1 + j] = 0.f; }
+    return;
+  }
+  const Top2 t = block_top2(logits + (size_t)row * dm.Vpad, dm, p);
+  if (threadIdx.x == 0) { st.o[b * dm.R1 + j] = t.i1; st.margin[b * dm.R1 + j] = t.v1 - t.v2; }
+}
+
+// ------------------------------------------------------------------------------------------
+// a12. acceptance + rollback: one warp per sequence.
+// ------------------------------------------------------------------------------------------
+struct GenOut {            // where fm_generate collects tokens (device-resident parameter block)
+  int* out_tok; int out_stride; int* out_len;
+  const int* truth; int truth_stride; const int* keep; int n_sched;
+  int plain;
+  long long* stats;        // [0] steps, [1] emitted, [2..] accept histogram
+  volatile int* host_done; // mapped pinned flag: number of unfinished sequences
+};
+
+__global__ void accept_kernel(Dims dm, SeqState st, int batch, const int* __restrict__ force_len,
+                              const int* __restrict__ force_tok, int* __restrict__ n_acc, int* __restrict__ emitted,
+                              int* __restrict__ kv_len, const GenOut* __restrict__ gen) {
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  const int b = warp;
+  if (b >= batch) return;
+  const int R1 = dm.R1, eos = dm.n_bins + 1;
+  const int rows = st.nrow[b];
+  int a = 0;
+  int L = st.L[b];
+  const int* o = (force_tok != nullptr ? force_tok : st.o) + b * R1;
+  const int cand = lane < R1 ? st.cand[b * R1 + lane] : -1;
+  if (rows > 0 && !st.done[b]) {
+    // lane j holds candidate j; it matches if it is the main token or equals the argmax at row j-1
+    const bool match = lane < rows && (lane == 0 || cand == o[lane - 1]);
+    const unsigned mm = __ballot_sync(0xffffffffu, match);
+    a = __ffs(~mm) - 1;                              // length of the leading run of matches
+    if (gen != nullptr && gen->plain) a = 1;
+    if (force_len != nullptr) a = force_len[b];
+    a = max(1, min(a, rows));
+    const unsigned em = __ballot_sync(0xffffffffu, lane < a && cand == eos);
+    bool fin = false;
+    if (em) { a = __ffs(em); fin = true; }           // an accepted EOS ends the sequence
+    L += a;
+    if (L - 1 >= st.t_end[b]) fin = true;
+    if (gen != nullptr && gen->out_tok != nullptr && lane < a) {
+      const int at = gen->out_len[b] + lane;
+      if (at < gen->out_stride) gen->out_tok[(size_t)b * gen->out_stride + at] = cand;
+    }
+    __syncwarp();
+    if (lane == 0) {
+      st.L[b] = L;
+      st.main_tok[b] = o[a - 1];
+      st.done[b] = fin ? 1 : 0;
+      st.nrow[b] = fin ? 0 : min(R1, st.t_end[b] - (L - 1));
+      if (gen != nullptr) {
+        if (gen->out_len != nullptr) gen->out_len[b] += a;
+        if (gen->stats != nullptr) {
+          atomicAdd((unsigned long long*)&gen->stats[1], (unsigned long long)a);
+          atomicAdd((unsigned long long*)&gen->stats[2 + a], 1ull);
+        }
+      }
+    }
+  } else if (lane == 0) {
+    st.nrow[b] = 0;
+  }
+  if (n_acc != nullptr && lane == 0) n_acc[b] = a;
+  if (emitted != nullptr && lane < R1) emitted[b * R1 + lane] = lane < a ? cand : -1;
+  if (kv_len != nullptr && lane == 0) {
+    kv_len[b * 3 + 0] = L; kv_len[b * 3 + 1] = (L + 2) / 3; kv_len[b * 3 + 2] = (L + 8) / 9;
+  }
+}
+
+// after accept + row count of a generate pass: bump the step counter, tell the host how many
+// sequences are still running
+__global__ void step_end_kernel(SeqState st, const GenOut* __restrict__ gen) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  *st.step += 1;
+  if (gen->stats != nullptr) gen->stats[0] += 1;
+  if (gen->host_done != nullptr) { *gen->host_done = st.n_active[3]; __threadfence_system(); }
+}
+
+// ------------------------------------------------------------------------------------------
+// prefill helpers
+// ------------------------------------------------------------------------------------------
+// next chunk of BOS + prompt: cand[b][j] = u_{L+j}, nrow = min(R1, inputs left)
+__global__ void prefill_feed_kernel(Dims dm, SeqState st, int batch, const int* __restrict__ prompt,
+                                    const int* __restrict__ prompt_off) {
+  const int b = blockIdx.x;
+  if (b >= batch) return;
+  const int L = st.L[b], total = 1 + st.plen[b];
+  const int n = max(0, min(dm.R1, total - L));
+  for (int j = threadIdx.x; j < dm.R1; j += blockDim.x) {
+    const int pos = L + j;
+    int tok = dm.n_bins + 2;
+    if (j < n) tok = pos == 0 ? dm.n_bins : prompt[prompt_off[b] + pos - 1];
+    st.cand[b * dm.R1 + j] = tok;
+  }
+  if (threadIdx.x == 0) st.nrow[b] = n;
+}
+
+// all fed rows are accepted; when the prompt is used up the argmax of the last row is the main token
+__global__ void prefill_advance_kernel(Dims dm, SeqState st, int batch) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= batch) return;
+  const int n = st.nrow[b];
+  if (n <= 0) return;
+  const int L = st.L[b] + n;
+  st.L[b] = L;
+  if (L == 1 + st.plen[b]) st.main_tok[b] = st.o[b * dm.R1 + n - 1];
+}
+
+// set the rows of the first verify pass (and after fm_set_max_faces)
+__global__ void arm_kernel(Dims dm, SeqState st, int batch) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b < batch) {
+    const int L = st.L[b];
+    const bool fin = st.done[b] || (L - 1 >= st.t_end[b]);
+    st.done[b] = fin ? 1 : 0;
+    st.nrow[b] = fin ? 0 : min(dm.R1, st.t_end[b] - (L - 1));
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// a13. draft heads
+// ------------------------------------------------------------------------------------------
+// Head inputs.  Head index h: 0,1 coordinate; 2,3 vertex; 4.. face.  Row (h, b):
+// a[h][b] = bf16(rms(z) * g_h) with z the stashed split-node hidden of the pending position.
+__global__ void draft_prep_kernel(Dims dm, SeqState st, int batch, const float* __restrict__ zc, const float* __restrict__ zv,
+                                  const float* __restrict__ zf, const float* __restrict__ gains /*[NH,d]*/,
+                                  bf16* __restrict__ a /*[NH, max_batch, d]*/) {
+  __shared__ float sh[32];
+  const int h = blockIdx.y, b = blockIdx.x, d = dm.d;
+  if (b >= batch) return;
+  const int n = max(0, st.L[b] - 1);
+  const float* z = h < 2 ? zc + ((size_t)b * FM_RING_C + n % FM_RING_C) * d
+                 : h < 4 ? zv + ((size_t)b * FM_RING_V + (n / 3) % FM_RING_V) * d
+                         : zf + ((size_t)b * FM_RING_F + (n / 9) % FM_RING_F) * d;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) ss += z[i] * z[i];
+  ss = block_sum(ss, sh);
+  const float inv = rsqrtf(ss / (float)d + dm.eps);
+  bf16* dst = a + ((size_t)h * dm.max_batch + b) * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = __float2bfloat16(z[i] * inv * gains[(size_t)h * d + i]);
+}
+
+// y = z + A a  (Eq. 1 reduced to Linear + residual).  Coordinate-head features go straight to the
+// feature matrix (rows h*B+b); vertex/face head features become bf16 inputs of the upsample GEMMs.
+__global__ void draft_residual_kernel(Dims dm, SeqState st, int batch, const float* __restrict__ zc, const float* __restrict__ zv,
+                                      const float* __restrict__ zf, const float* __restrict__ y /*[NH,max_batch,d]*/,
+                                      float* __restrict__ feat /*[NF*B, d]*/, bf16* __restrict__ up_in_v /*[2B + 3*Ef*B, d]*/,
+                                      bf16* __restrict__ up_in_f /*[Ef*B, d]*/) {
+  const int h = blockIdx.y, b = blockIdx.x, d = dm.d;
+  if (b >= batch) return;
+  const int n = max(0, st.L[b] - 1);
+  const float* z = h < 2 ? zc + ((size_t)b * FM_RING_C + n % FM_RING_C) * d
+                 : h < 4 ? zv + ((size_t)b * FM_RING_V + (n / 3) % FM_RING_V) * d
+                         : zf + ((size_t)b * FM_RING_F + (n / 9) % FM_RING_F) * d;
+  const float* yr = y + ((size_t)h * dm.max_batch + b) * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    const float v = z[i] + yr[i];
+    if (h < 2) feat[((size_t)h * batch + b) * d + i] = v;
+    else if (h < 4) up_in_v[((size_t)(h - 2) * batch + b) * d + i] = __float2bfloat16(v);
+    else up_in_f[((size_t)(h - 4) * batch + b) * d + i] = __float2bfloat16(v);
+  }
+}
+
+// feature row that serves draft offset j of sequence b (single source per offset):
+// offsets 1,2 -> coordinate heads; later offsets in the current face -> vertex head
+// floor(p/3)-v*; offsets in a later face -> face head floor(p/9)-f*.
+__device__ inline int draft_feature_row(int n, int j, int b, int B) {
+  const int p = n + j;
+  if (j <= 2) return (j - 1) * B + b;
+  if (p / 9 == n / 9) {
+    const int e = p / 3 - n / 3;
+    return 2 * B + 3 * ((e - 1) * B + b) + p % 3;
+  }
+  const int e = p / 9 - n / 9, s = p % 9;
+  return 2 * B + 3 * (2 * B + 3 * ((e - 1) * B + b) + s / 3) + s % 3;
+}
+
+// masked argmax of the chosen feature's logits -> cand[b][j]; cand[b][0] = pending main token
+__global__ void draft_pick_kernel(Dims dm, SeqState st, int batch, const float* __restrict__ logits /*[NF*B, Vpad]*/,
+                                  float* __restrict__ logits_out, float* __restrict__ margin_out) {
+  const int b = blockIdx.x, j = blockIdx.y;        // j = 0..D
+  if (b >= batch) return;
+  const bool fin = st.done[b] != 0 || st.nrow[b] <= 0;
+  if (j == 0) {
+    if (threadIdx.x == 0) st.cand[b * dm.R1] = fin ? dm.n_bins + 2 : st.main_tok[b];
+    return;
+  }
+  if (fin) {
+    if (threadIdx.x == 0) { st.cand[b * dm.R1 + j] = dm.n_bins + 2; if (margin_out) margin_out[b * dm.D + j - 1] = 0.f; }
+    if (logits_out)
+      for (int i = threadIdx.x; i < dm.V; i += blockDim.x) logits_out[((size_t)b * dm.D + j - 1) * dm.V + i] = 0.f;
+    return;
+  }
+  const int n = st.L[b] - 1;
+  const float* z = logits + (size_t)draft_feature_row(n, j, b, batch) * dm.Vpad;
+  if (logits_out)
+    for (int i = threadIdx.x; i < dm.V; i += blockDim.x) logits_out[((size_t)b * dm.D + j - 1) * dm.V + i] = z[i];
+  const Top2 t = block_top2(z, dm, n + j);
+  if (threadIdx.x == 0) {
+    st.cand[b * dm.R1 + j] = t.i1;
+    if (margin_out) margin_out[b * dm.D + j - 1] = t.v1 - t.v2;
+  }
+}
+
+// teacher edit (benchmark stand-in for trained heads; sits where the Correct stage edits drafts):
+// drafts 1..keep <- known continuation, draft keep+1 <- a different coordinate id
+__global__ void teacher_edit_kernel(Dims dm, SeqState st, int batch, const GenOut* __restrict__ gen) {
+  const int b = blockIdx.x;
+  if (b >= batch || gen->truth == nullptr) return;
+  if (st.done[b] || st.nrow[b] <= 0) return;
+  const int n = st.L[b] - 1;
+  const int keep = gen->keep != nullptr ? gen->keep[(size_t)(*st.step % gen->n_sched) * batch + b] : dm.D;
+  for (int j = 1 + threadIdx.x; j <= dm.D; j += blockDim.x) {
+    const int idx = n + j;
+    if (idx >= gen->truth_stride) continue;
+    const int t = gen->truth[(size_t)b * gen->truth_stride + idx];
+    if (t < 0 || t >= dm.V) continue;
+    if (j <= keep) st.cand[b * dm.R1 + j] = t;
+    else if (j == keep + 1) st.cand[b * dm.R1 + j] = (t + 1) % dm.n_bins;
+  }
+}
+
+__global__ void copy_i32_kernel(const int* __restrict__ src, int* __restrict__ dst, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = src[i];
+}
+__global__ void copy_f32_kernel(const float* __restrict__ src, float* __restrict__ dst, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = src[i];
+}
