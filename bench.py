@@ -1,0 +1,364 @@
+#!/usr/bin/env python
+"""Benchmark of the speculative decode step (draft -> verify -> accept) on synthetic inputs.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload medium]
+
+A step is one pass of the whole hot path over the batch.  The metric is mesh tokens/s.  The
+timed region starts with the model, the KV caches (filled to the middle of the configured run)
+and the teacher schedule resident in HBM.  One JSON line is printed by rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import fm_synth as S  # noqa: E402
+
+METRIC = "mesh_tokens_per_s"
+MEAN_DRAFTS = 6.7          # accepted drafts per pass of the paper's 9-9 row (6.43 .. 6.97 of 9)
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def _fill_prompt(cfg, seq, n_faces):
+    """Seeded mesh tokens standing in for an already generated prefix: the sorted faces of a
+    twice-subdivided icosphere, repeated until n_faces faces."""
+    base = S.make_prompt(cfg.with_(prompt_faces=(320, 320), prompt_subdiv=2), seq)
+    reps = -(-n_faces * 9 // len(base))
+    return [int(t) for t in np.tile(base, reps)[:9 * n_faces]]
+
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=open(self.path, "w"),
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, reasons = [], set()
+        for ln in open(self.path):
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                out["sm_max_mhz"] = float(f[2])
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.path)
+        if sm:
+            out["sm_mhz"] = float(np.median(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# -------------------------------------------------------------------------------------------
+# our arm
+# -------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2511_15618_b200 import FlashMesh
+    from paper_2511_15618_b200.build import build
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    if rank == 0:
+        build()
+    if world > 1:
+        dist.barrier()
+    cfg = S.get_config(args.workload)
+    B, D = cfg.batch, cfg.draft_len
+    K, W = args.steps, args.warmup
+    start_faces = int(cfg.gen_faces * args.start_frac)
+    need_faces = -(-(K + W + 8) * (D + 1) // 9) + 1
+    max_tokens = 1 + 9 * (start_faces + cfg.prompt_faces[1] + need_faces) + D + 2
+    w = S.make_weights(cfg)
+    conds = np.stack([S.make_condition(cfg, rank * B + b) for b in range(B)])
+    rng = np.random.default_rng([cfg.seed, 77, rank])
+    prompts = []
+    for b in range(B):                    # ragged fills around the target (exact for batch 1)
+        f = start_faces if B == 1 else max(1, int(start_faces * rng.uniform(0.5, 1.0)))
+        prompts.append(_fill_prompt(cfg, rank * B + b, f))
+    dev = FlashMesh(cfg, w, device=f"cuda:{local}", max_tokens=max_tokens)
+    del w
+
+    # untimed set-up: the continuation the teacher drafts come from (plain decoding on the same kernels)
+    dev.prefill(conds, prompts)
+    plain_tok, plain_len, st_plain = dev.generate(need_faces, plain=True)
+    t_ori_ms = st_plain.ms / max(1, st_plain.steps)
+    truth = np.full((B, max(len(p) for p in prompts) + 9 * need_faces), 0, dtype=np.int32)
+    pt = plain_tok.cpu().numpy()
+    for b in range(B):
+        seq = np.concatenate([np.asarray(prompts[b], np.int32), pt[b]])
+        truth[b, :len(seq)] = seq
+    keep = (S.accept_schedule(cfg.seed + rank, B, 4096, D, MEAN_DRAFTS) - 1).astype(np.int32)
+    truth_d = torch.as_tensor(truth).cuda()
+    keep_d = torch.as_tensor(keep).cuda()
+
+    def sync_all():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- timed: K passes, inputs resident in HBM
+    dev.prefill(conds, prompts)
+    out = None
+    if W > 0:
+        tok, ln, _ = dev.generate(need_faces, truth=truth_d, keep=keep_d, max_steps=W)
+        out = (tok, ln)
+    sampler = ClockSampler(local)
+    sampler.start()
+    l0 = dev.launch_count()
+    sync_all()
+    tok, ln, st = dev.generate(need_faces, truth=truth_d, keep=keep_d, max_steps=K, out=out)
+    sync_all()
+    launches = dev.launch_count() - l0
+    clocks = sampler.stop()
+    ms, emitted, steps = float(st.ms), int(st.emitted), int(st.steps)
+    # generated tokens must be the plain-decoding continuation (teacher drafts change speed, not output)
+    got = tok.cpu().numpy()
+    n_chk = int(ln.cpu().numpy().min())
+    assert (got[:, :n_chk] == pt[:, :n_chk]).all(), "speculative output differs from plain decoding"
+
+    # ---- the same passes once more with per-kernel-class events (roofline of the dominant kernel)
+    dev.prefill(conds, prompts)
+    if W > 0:
+        dev.generate(need_faces, truth=truth_d, keep=keep_d, max_steps=W)
+    kv0 = None
+    dev.profile_begin()
+    _, _, stp = dev.generate(need_faces, truth=truth_d, keep=keep_d, max_steps=K)
+    prof = dev.profile_end()
+    # lengths at the end of the timed passes -> algorithmic bytes of a verify pass there
+    cand, _, _ = dev.draft()
+    dev.verify(cand)
+    _, _, kv = dev.accept()
+    kv_len = kv.cpu().numpy().tolist()
+    step_bytes = dev.verify_bytes(kv_len)
+
+    # ---- natural acceptance of the (random-weight) heads, same state
+    dev.prefill(conds, prompts)
+    _, _, st_nat = dev.generate(need_faces, max_steps=max(8, K // 4))
+
+    # ---- end to end: host in the loop (stepwise C ABI, pinned host buffers, copies inside the timing)
+    dev.prefill(conds, prompts)
+    e2e = run_e2e(dev, cfg, truth, keep, prompts, max(8, min(K, 64)))
+
+    peak, peak_kind = _peaks()
+    if world > 1:
+        t = torch.tensor([ms, float(emitted), float(launches)], dtype=torch.float64, device="cuda")
+        tmax = t.clone()
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        tsum = t.clone()
+        dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
+        ms, emitted, launches = float(tmax[0]), int(tsum[1]), int(tsum[2])
+        e = torch.tensor([e2e["tokens"], e2e["seconds"]], dtype=torch.float64, device="cuda")
+        emax, esum = e.clone(), e.clone()
+        dist.all_reduce(emax, op=dist.ReduceOp.MAX)
+        dist.all_reduce(esum, op=dist.ReduceOp.SUM)
+        e2e["tokens"], e2e["seconds"] = float(esum[0]), float(emax[1])
+    value = emitted / (ms * 1e-3)
+    gemm_gbs = prof.gemm_bytes / (prof.gemm_ms * 1e-3) / 1e9 if prof.gemm_ms > 0 else 0.0
+    step_ms = ms / max(1, steps)
+    line = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "batch_per_gpu": B, "draft_len": D,
+                   "kv_fill": f"prefix of {start_faces} faces per sequence already in the caches "
+                              f"(middle of the {cfg.gen_faces}-face run)",
+                   "acceptance": f"teacher drafts, seeded schedule, mean {MEAN_DRAFTS} drafts kept per pass",
+                   "l2": "weights streamed per pass exceed the 126 MB L2; no flush between passes",
+                   "parallelism": f"replicas x{world}"},
+        "mean_accept_len": emitted / max(1, steps * B * world),
+        "natural_accept_len": st_nat.emitted / max(1, st_nat.steps * B),
+        "natural_tokens_per_s": st_nat.emitted / (st_nat.ms * 1e-3),
+        "plain_tokens_per_s": B / (t_ori_ms * 1e-3), "plain_ms_per_step": t_ori_ms,
+        "clocks": clocks,
+        "e2e": {"value": e2e["tokens"] / e2e["seconds"], "unit": "tokens/s",
+                "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                "what": "stepwise fm_draft/fm_verify/fm_accept with the host in the loop: candidates from "
+                        "pinned host memory every pass, accepted tokens read back every pass"},
+        "gpu_launches": launches,
+        "roofline": {"bound": "hbm", "kernel": "weight-streaming GEMM (all launches of the timed passes)",
+                     "achieved": gemm_gbs, "peak": peak, "unit": "GB/s", "frac": gemm_gbs / peak,
+                     "peak_kind": peak_kind, "traffic": None,
+                     "launches": int(prof.gemm_launches), "ms_per_pass": prof.gemm_ms / max(1, stp.steps),
+                     "attention_ms_per_pass": prof.attn_ms / max(1, stp.steps)},
+        "verify_step": {"algorithmic_bytes": step_bytes, "ms": step_ms, "GB/s": step_bytes / (step_ms * 1e-3) / 1e9,
+                        "frac_of_hbm_peak": step_bytes / (step_ms * 1e-3) / 1e9 / peak, "kv_len": kv_len[0],
+                        "note": "whole pass (draft heads + verify + accept) against the verify bytes"},
+    }
+    if rank == 0:
+        if world == 1 and not args.no_cpu:
+            line["cpu_baseline"] = cpu_baseline(args.workload, budget_s=args.cpu_seconds)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def run_e2e(dev, cfg, truth, keep, prompts, steps):
+    """Host-in-the-loop decode through the stepwise C ABI: per pass the host builds the edited
+    candidates from the transcript (it knows L from the previous pass), copies them in from pinned
+    memory, and reads the accepted tokens back."""
+    import torch
+    B, D = len(prompts), cfg.draft_len
+    L = np.array([1 + len(p) for p in prompts])
+    cand_h = torch.empty((B, D + 1), dtype=torch.int32).pin_memory()
+    nacc_h = torch.empty((B,), dtype=torch.int32).pin_memory()
+    em_h = torch.empty((B, D + 1), dtype=torch.int32).pin_memory()
+    cand_d = torch.empty((B, D + 1), dtype=torch.int32, device="cuda")
+    tokens = 0
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for s in range(steps):
+        dev.draft()                                           # heads run; their drafts are replaced below
+        for b in range(B):
+            n = L[b] - 1
+            k = int(keep[s % keep.shape[0], b])
+            row = truth[b, n:n + D + 1].copy()
+            if k < D:
+                row[k + 1] = (row[k + 1] + 1) % cfg.n_bins
+            cand_h[b] = torch.from_numpy(row)
+        cand_d.copy_(cand_h, non_blocking=True)
+        dev.verify(cand_d)
+        n_acc, em, _ = dev.accept()
+        nacc_h.copy_(n_acc, non_blocking=True)
+        em_h.copy_(em, non_blocking=True)
+        torch.cuda.synchronize()
+        a = nacc_h.numpy()
+        L = L + a
+        tokens += int(a.sum())
+    dt = time.perf_counter() - t0
+    return {"tokens": float(tokens), "seconds": dt, "h2d": B * (D + 1) * 4, "d2h": B * (D + 2) * 4}
+
+
+# -------------------------------------------------------------------------------------------
+# the oracle as CPU baseline / reference arm
+# -------------------------------------------------------------------------------------------
+def _oracle_passes(workload, n_steps, budget_s):
+    """Time the oracle, as it stands, on a bounded sample: prefill of the workload's own short
+    prompt, then speculative passes with the seeded acceptance schedule (forced lengths)."""
+    from oracle.hourglass import OracleSeq
+    cfg = S.get_config(workload)
+    B, D = cfg.batch, cfg.draft_len
+    w = S.make_weights(cfg)
+    B_run = min(B, 2)
+    sched = S.accept_schedule(cfg.seed, B_run, 4096, D, MEAN_DRAFTS)
+    seqs = []
+    for b in range(B_run):
+        s = OracleSeq(cfg.with_(max_tokens=2048), w)
+        s.prefill(S.make_condition(cfg, b), [int(t) for t in S.make_prompt(cfg, b)], max_faces=200)
+        seqs.append(s)
+    t0 = time.perf_counter()
+    tokens = steps = 0
+    while steps < n_steps and time.perf_counter() - t0 < budget_s:
+        for b, s in enumerate(seqs):
+            cand, _, _ = s.draft()
+            s.verify(cand)
+            a, _, _ = s.accept(force_len=int(sched[steps % 4096, b]))
+            tokens += a
+        steps += 1
+    dt = time.perf_counter() - t0
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    return tokens, steps, dt, cores, B_run
+
+
+def cpu_baseline(workload, budget_s=20.0):
+    tokens, steps, dt, cores, b_run = _oracle_passes(workload, 10 ** 9, budget_s)
+    return {"value": tokens / dt, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+            "sample": f"{steps} speculative passes of {b_run} sequence(s) right after the prompt (short KV caches), "
+                      f"forced acceptance schedule with mean {MEAN_DRAFTS} drafts; numpy float64",
+            "ms_per_step": dt / max(1, steps) * 1e3}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    cfg = S.get_config(args.workload)
+    for _ in range(1):
+        _oracle_passes(args.workload, min(args.warmup, 1), 120.0)          # warm-up (weights cast, BLAS threads)
+    tokens, steps, dt, cores, b_run = _oracle_passes(args.workload, args.steps, 150.0)
+    value = tokens / dt
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world,
+            "steps": steps, "warmup": args.warmup, "ms_per_step": dt / max(1, steps) * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "batch_per_gpu": b_run, "draft_len": cfg.draft_len,
+                       "sample": "passes right after the prompt (short KV caches), forced acceptance schedule"},
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                             "sample": f"{steps} passes of {b_run} sequence(s), short KV caches"},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="medium", choices=list(S.CONFIGS))
+    ap.add_argument("--start-frac", type=float, default=0.5, help="fraction of the run already in the caches")
+    ap.add_argument("--cpu-seconds", type=float, default=20.0)
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(3, args.warmup) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -165,19 +165,32 @@ int fm_accept(fm_ctx* ctx, const int32_t* force_len /*DEV*/, const int32_t* forc
               int32_t* n_acc /*DEV*/, int32_t* emitted /*DEV*/, int32_t* kv_len /*DEV*/);
 
 /* The whole loop (Sec. 3): draft -> (optional teacher edit) -> verify -> accept, until every
- * sequence has emitted 9*max_faces tokens or EOS.  out_tok: DEV int32 [batch, out_stride]
- * receives the emitted tokens (prompt not included), out_len: DEV int32 [batch].  teacher and
- * stats may be NULL.  plain != 0 accepts only the main token every pass (the one-token-at-a-
- * time baseline on the same kernels).  Synchronous (returns after the last pass).
+ * sequence has emitted 9*max_faces tokens or EOS, or, when max_steps > 0, for exactly max_steps
+ * passes (a later call continues where this one stopped).  out_tok: DEV int32 [batch, out_stride]
+ * receives the emitted tokens (prompt not included), out_len: DEV int32 [batch], zeroed by the
+ * first call after fm_prefill and advanced by every call; both may be NULL.  teacher and stats may
+ * be NULL.  plain != 0 accepts only the main token every pass (the one-token-at-a-time baseline
+ * on the same kernels).  Synchronous (returns after the last pass).
  * Errors: BAD_STATE, CAPACITY (prompt + 9*max_faces + D + 2 > max_tokens, or out_stride too small). */
 int fm_generate(fm_ctx* ctx, int32_t max_faces, int32_t* out_tok /*DEV*/, int32_t out_stride,
                 int32_t* out_len /*DEV*/, const fm_teacher* teacher /*HOST struct, DEV arrays*/,
-                int32_t plain, fm_stats* stats /*HOST*/);
+                int32_t plain, int64_t max_steps, fm_stats* stats /*HOST*/);
 
 /* Algorithmic bytes one verify pass must move for the given per-sequence lengths (weights of
  * the stacks that have rows, shorten/upsample, output matrix, K and V entries visible to the
  * rows); kv_len HOST int32 [batch,3] as returned by fm_accept.  For roofline reports. */
 double fm_verify_bytes(const fm_ctx* ctx, int32_t batch, const int32_t* kv_len /*HOST*/);
+
+/* Per-kernel-class device timing for roofline reports (no counterpart in the paper).  Between
+ * fm_profile_begin and fm_profile_end every weight-streaming GEMM launch and every attention
+ * launch is bracketed by a CUDA event pair on the context's stream; fm_profile_end synchronises
+ * and sums them.  gemm_bytes counts each launch's weight matrix once (2*M*K bytes). */
+typedef struct fm_profile {
+  double gemm_ms, gemm_bytes; int64_t gemm_launches;
+  double attn_ms; int64_t attn_launches;
+} fm_profile;
+int fm_profile_begin(fm_ctx* ctx);
+int fm_profile_end(fm_ctx* ctx, fm_profile* out /*HOST*/);
 
 /* Number of kernels launched by this context since creation (for launch accounting). */
 int64_t fm_launch_count(const fm_ctx* ctx);

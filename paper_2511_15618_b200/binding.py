@@ -55,6 +55,11 @@ class FmStats(C.Structure):
                 ("ms", C.c_float)]
 
 
+class FmProfile(C.Structure):
+    _fields_ = [("gemm_ms", C.c_double), ("gemm_bytes", C.c_double), ("gemm_launches", C.c_int64),
+                ("attn_ms", C.c_double), ("attn_launches", C.c_int64)]
+
+
 def library_path() -> str:
     return os.path.join(_HERE, "libflashmesh.so")
 
@@ -87,9 +92,13 @@ def load_library():
     lib.fm_accept.restype = C.c_int
     lib.fm_accept.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.fm_generate.restype = C.c_int
-    lib.fm_generate.argtypes = [vp, i32, vp, i32, vp, C.POINTER(FmTeacher), i32, C.POINTER(FmStats)]
+    lib.fm_generate.argtypes = [vp, i32, vp, i32, vp, C.POINTER(FmTeacher), i32, C.c_int64, C.POINTER(FmStats)]
     lib.fm_verify_bytes.restype = C.c_double
     lib.fm_verify_bytes.argtypes = [vp, i32, C.POINTER(C.c_int32)]
+    lib.fm_profile_begin.restype = C.c_int
+    lib.fm_profile_begin.argtypes = [vp]
+    lib.fm_profile_end.restype = C.c_int
+    lib.fm_profile_end.argtypes = [vp, C.POINTER(FmProfile)]
     lib.fm_launch_count.restype = C.c_int64
     lib.fm_launch_count.argtypes = [vp]
     lib.fm_strerror.restype = C.c_char_p
@@ -144,15 +153,25 @@ def fm_accept(ctx, force_len_ptr=None, force_tok_ptr=None, n_acc_ptr=None, emitt
     return load_library().fm_accept(ctx, force_len_ptr, force_tok_ptr, n_acc_ptr, emitted_ptr, kv_len_ptr)
 
 
-def fm_generate(ctx, max_faces, out_tok_ptr, out_stride, out_len_ptr, teacher=None, plain=0, stats=None):
+def fm_generate(ctx, max_faces, out_tok_ptr, out_stride, out_len_ptr, teacher=None, plain=0, max_steps=0, stats=None):
     t = C.byref(teacher) if teacher is not None else None
     s = C.byref(stats) if stats is not None else None
-    return load_library().fm_generate(ctx, max_faces, out_tok_ptr, out_stride, out_len_ptr, t, plain, s)
+    return load_library().fm_generate(ctx, max_faces, out_tok_ptr, out_stride, out_len_ptr, t, plain, max_steps, s)
 
 
 def fm_verify_bytes(ctx, batch, kv_len):
     flat = [int(v) for row in kv_len for v in row]
     return float(load_library().fm_verify_bytes(ctx, batch, _i32_array(flat)))
+
+
+def fm_profile_begin(ctx):
+    return load_library().fm_profile_begin(ctx)
+
+
+def fm_profile_end(ctx):
+    p = FmProfile()
+    rc = load_library().fm_profile_end(ctx, C.byref(p))
+    return rc, p
 
 
 def fm_launch_count(ctx):
@@ -310,8 +329,9 @@ class FlashMesh:
                               kv.data_ptr()), "fm_accept")
         return n_acc, em, kv
 
-    def generate(self, max_faces, truth=None, keep=None, plain=False, out=None):
-        """Run the decode loop; returns (tokens [B, 9*max_faces] int32, lengths [B], FmStats)."""
+    def generate(self, max_faces, truth=None, keep=None, plain=False, out=None, max_steps=0):
+        """Run the decode loop; returns (tokens [B, 9*max_faces] int32, lengths [B], FmStats).
+        `out` = (tokens, lengths) of an earlier call continues appending to them."""
         t = self.torch
         B = self.batch
         stride = 9 * max_faces
@@ -328,11 +348,19 @@ class FlashMesh:
             teacher.n_sched = int(self._keep_sched.shape[0]) if self._keep_sched is not None else 0
         stats = FmStats()
         self._check(fm_generate(self.ctx, max_faces, out_tok.data_ptr(), stride, out_len.data_ptr(), teacher,
-                                1 if plain else 0, stats), "fm_generate")
+                                1 if plain else 0, max_steps, stats), "fm_generate")
         return out_tok, out_len, stats
 
     def verify_bytes(self, kv_len):
         return fm_verify_bytes(self.ctx, len(kv_len), kv_len)
+
+    def profile_begin(self):
+        self._check(fm_profile_begin(self.ctx), "fm_profile_begin")
+
+    def profile_end(self):
+        rc, p = fm_profile_end(self.ctx)
+        self._check(rc, "fm_profile_end")
+        return p
 
     def launch_count(self):
         return fm_launch_count(self.ctx)

@@ -63,7 +63,15 @@ struct fm_ctx {
   long long* stats_dev;
   int* host_done;       // pinned, mapped
   int* host_done_dev;
+  // optional per-kernel-class timing (fm_profile_begin / fm_profile_end)
+  bool prof_on;
+  std::vector<cudaEvent_t> prof_ev;     // pairs
+  std::vector<int> prof_cls;
+  size_t prof_used;
+  double prof_ms[3], prof_bytes[3];
+  long long prof_n[3];
   int batch;
+  bool gen_fresh;       // no fm_generate call since the last fm_prefill
   std::vector<int> plen_host;
   int phase;            // 0 created, 1 prefilled / accepted, 2 verified
   int64_t launches;
@@ -213,17 +221,46 @@ int upload_f32(float* dst, const float* src, size_t n) {
     (ctx)->launches++;                                                   \
   } while (0)
 
+enum ProfClass { PROF_GEMM = 0, PROF_ATTN = 1, PROF_OTHER = 2 };
+
+void prof_drain(fm_ctx* c) {
+  if (c->prof_used == 0) return;
+  cudaStreamSynchronize(c->stream);
+  for (size_t i = 0; i < c->prof_used; ++i) {
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, c->prof_ev[2 * i], c->prof_ev[2 * i + 1]);
+    c->prof_ms[c->prof_cls[i]] += ms;
+  }
+  c->prof_used = 0;
+}
+// bracket the launches issued between prof_open and prof_close with an event pair
+inline long prof_open(fm_ctx* c, int cls, double bytes) {
+  if (!c->prof_on) return -1;
+  if (c->prof_used == c->prof_cls.size()) prof_drain(c);
+  const size_t i = c->prof_used++;
+  c->prof_cls[i] = cls;
+  c->prof_bytes[cls] += bytes;
+  c->prof_n[cls] += 1;
+  cudaEventRecord(c->prof_ev[2 * i], c->stream);
+  return (long)i;
+}
+inline void prof_close(fm_ctx* c, long i) {
+  if (i >= 0) cudaEventRecord(c->prof_ev[2 * i + 1], c->stream);
+}
+
 void gemm(fm_ctx* c, int mode, const bf16* W, const bf16* A, void* out, int M, int K, int R, int ldo,
           const int* n_active, int nz = 1, long long sW = 0, long long sA = 0, long long sO = 0) {
   if (R <= 0) return;
   GemmArgs g{W, A, out, M, K, R, ldo, sW, sA, sO, n_active};
   dim3 grid((M + 3) / 4, (R + 15) / 16, nz);
+  const long pi = prof_open(c, PROF_GEMM, 2.0 * M * K * nz);       // algorithmic bytes: the weight matrix once
   switch (mode) {
     case GEMM_STORE_F32: LAUNCH(c, gemm_simt_kernel<GEMM_STORE_F32>, grid, 128, 0, g); break;
     case GEMM_ADD_F32: LAUNCH(c, gemm_simt_kernel<GEMM_ADD_F32>, grid, 128, 0, g); break;
     case GEMM_GELU_BF16: LAUNCH(c, gemm_simt_kernel<GEMM_GELU_BF16>, grid, 128, 0, g); break;
     default: LAUNCH(c, gemm_simt_kernel<GEMM_STORE_BF16>, grid, 128, 0, g); break;
   }
+  prof_close(c, pi);
 }
 
 __global__ void to_bf16_kernel(const float* __restrict__ x, bf16* __restrict__ out, size_t n) {
@@ -250,9 +287,11 @@ __global__ void row_count_kernel(Dims dm, SeqState st, int batch) {
 void attention(fm_ctx* c, int level, int rows, const LayerDev& L) {
   const Dims& dm = c->dm;
   dim3 grid(rows, dm.H);
+  const long pi = prof_open(c, PROF_ATTN, 0.0);
   if (dm.dh == 32) LAUNCH(c, attn_rows_kernel<32>, grid, 128, 0, dm, c->st, c->batch, level, c->qbuf, L.K, L.V, c->a_attn);
   else if (dm.dh == 64) LAUNCH(c, attn_rows_kernel<64>, grid, 128, 0, dm, c->st, c->batch, level, c->qbuf, L.K, L.V, c->a_attn);
   else LAUNCH(c, attn_rows_kernel<128>, grid, 128, 0, dm, c->st, c->batch, level, c->qbuf, L.K, L.V, c->a_attn);
+  prof_close(c, pi);
 }
 
 // one stack of pre-norm blocks on the rows of its level (a2/a4/a6/a8/a10)
@@ -460,9 +499,33 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
   return FM_OK;
 }
 
+int fm_profile_begin(fm_ctx* c) {
+  if (c == nullptr) return FM_ERR_INVALID_ARG;
+  if (c->prof_ev.empty()) {
+    const size_t pairs = 4096;
+    c->prof_ev.resize(2 * pairs);
+    c->prof_cls.assign(pairs, 0);
+    for (auto& e : c->prof_ev) CUDA_OK(cudaEventCreate(&e));
+  }
+  c->prof_used = 0;
+  for (int i = 0; i < 3; ++i) { c->prof_ms[i] = 0; c->prof_bytes[i] = 0; c->prof_n[i] = 0; }
+  c->prof_on = true;
+  return FM_OK;
+}
+
+int fm_profile_end(fm_ctx* c, fm_profile* out) {
+  if (c == nullptr || out == nullptr) return FM_ERR_INVALID_ARG;
+  prof_drain(c);
+  c->prof_on = false;
+  out->gemm_ms = c->prof_ms[PROF_GEMM]; out->gemm_bytes = c->prof_bytes[PROF_GEMM]; out->gemm_launches = c->prof_n[PROF_GEMM];
+  out->attn_ms = c->prof_ms[PROF_ATTN]; out->attn_launches = c->prof_n[PROF_ATTN];
+  return FM_OK;
+}
+
 int fm_destroy(fm_ctx* c) {
   if (c == nullptr) return FM_ERR_INVALID_ARG;
   cudaStreamSynchronize(c->stream);
+  for (auto& e : c->prof_ev) cudaEventDestroy(e);
   if (c->host_done != nullptr) cudaFreeHost(c->host_done);
   delete c;
   return FM_OK;
@@ -510,6 +573,7 @@ int fm_prefill(fm_ctx* c, int32_t batch, const float* cond, const int32_t* promp
   LAUNCH(c, row_count_kernel, 1, 32, 0, dm, c->st, batch);
   CUDA_OK(cudaGetLastError());
   c->phase = 1;
+  c->gen_fresh = true;
   return FM_OK;
 }
 
@@ -562,7 +626,7 @@ int fm_accept(fm_ctx* c, const int32_t* force_len, const int32_t* force_tok, int
 }
 
 int fm_generate(fm_ctx* c, int32_t max_faces, int32_t* out_tok, int32_t out_stride, int32_t* out_len,
-                const fm_teacher* teacher, int32_t plain, fm_stats* stats) {
+                const fm_teacher* teacher, int32_t plain, int64_t max_steps, fm_stats* stats) {
   if (c == nullptr || max_faces < 0) return FM_ERR_INVALID_ARG;
   if (c->phase < 1) return FM_ERR_BAD_STATE;
   const Dims& dm = c->dm;
@@ -582,7 +646,8 @@ int fm_generate(fm_ctx* c, int32_t max_faces, int32_t* out_tok, int32_t out_stri
   g.host_done = c->host_done_dev;
   CUDA_OK(cudaMemcpyAsync(c->gen_dev, &g, sizeof(g), cudaMemcpyHostToDevice, c->stream));
   CUDA_OK(cudaMemsetAsync(c->stats_dev, 0, (FM_MAX_DRAFT + 4) * sizeof(long long), c->stream));
-  if (out_len != nullptr) CUDA_OK(cudaMemsetAsync(out_len, 0, c->batch * sizeof(int), c->stream));
+  if (out_len != nullptr && c->gen_fresh) CUDA_OK(cudaMemsetAsync(out_len, 0, c->batch * sizeof(int), c->stream));
+  c->gen_fresh = false;
   CUDA_OK(cudaStreamSynchronize(c->stream));       // `g` lives on this stack frame
   cudaEvent_t e0, e1;
   CUDA_OK(cudaEventCreate(&e0));
@@ -590,12 +655,12 @@ int fm_generate(fm_ctx* c, int32_t max_faces, int32_t* out_tok, int32_t out_stri
   CUDA_OK(cudaEventRecord(e0, c->stream));
   *c->host_done = c->batch;
   // upper bound on passes: every pass emits at least one token per unfinished sequence
-  const long long max_steps = 9ll * max_faces + 1;
-  const int poll = 8;
+  const long long bound = max_steps > 0 ? max_steps : 9ll * max_faces + 8;
   long long steps = 0;
   bool finished = false;
-  while (!finished && steps < max_steps + poll) {
-    for (int i = 0; i < poll; ++i) {
+  while (!finished && steps < bound) {
+    const long long poll = max_steps > 0 ? bound : 8;
+    for (long long i = 0; i < poll; ++i) {
       draft(c, nullptr, nullptr);
       if (teacher != nullptr) LAUNCH(c, teacher_edit_kernel, c->batch, 32, 0, dm, c->st, c->batch, c->gen_dev);
       forward(c, nullptr);
@@ -606,7 +671,7 @@ int fm_generate(fm_ctx* c, int32_t max_faces, int32_t* out_tok, int32_t out_stri
       ++steps;
     }
     CUDA_OK(cudaStreamSynchronize(c->stream));
-    finished = *c->host_done == 0;
+    finished = *c->host_done == 0 || max_steps > 0;
   }
   CUDA_OK(cudaEventRecord(e1, c->stream));
   CUDA_OK(cudaEventSynchronize(e1));
