@@ -3,6 +3,7 @@
 // workspace, uploads weights and enqueues launches.
 #include "../../include/flashmesh.h"
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdio.h>
@@ -26,6 +27,7 @@ struct LayerDev {
   bf16 *Wqkv, *Wo, *W1, *W2;
   float *g1, *g2;
   bf16 *K, *V;                          // [max_batch, Hkv, P + cap, dh]
+  int tmK, tmV;                         // tensor-map indices
 };
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -54,6 +56,12 @@ struct fm_ctx {
   // draft
   bf16 *dh_a, *up_in_v, *up_in_f, *feat_n;
   float *dh_y, *feat, *dlogits;
+  // attention scratch and TMA descriptors
+  float* attn_part;
+  int* attn_ticket;
+  int attn_chunk, attn_max_chunks[3], attn_mrows[3];
+  CUtensorMap* tmaps;                    // device array
+  std::vector<CUtensorMap> tmaps_host;
   // prefill temporaries
   bf16* pre_a;
   float* pre_o;
@@ -92,7 +100,7 @@ int check_config(const fm_config* c) {
   for (int i = 0; i < 5; ++i) if (c->layers[i] < 1) return FM_ERR_UNSUPPORTED;
   if (c->draft_len > FM_MAX_DRAFT) return FM_ERR_UNSUPPORTED;
   if (c->d_model % 64 != 0 || c->d_ff % 64 != 0 || (c->n_heads * c->head_dim) % 64 != 0) return FM_ERR_UNSUPPORTED;
-  if (c->head_dim != 32 && c->head_dim != 64 && c->head_dim != 128) return FM_ERR_UNSUPPORTED;
+  if (c->head_dim != 64 && c->head_dim != 128) return FM_ERR_UNSUPPORTED;
   if ((c->draft_len + 8) / 9 > FM_MAX_FACE_HEADS) return FM_ERR_UNSUPPORTED;
   if (c->max_tokens < c->draft_len + 2) return FM_ERR_INVALID_ARG;
   return FM_OK;
@@ -181,6 +189,20 @@ void carve(fm_ctx* c, Carver& cv) {
   c->up_in_f = cv.take<bf16>(align_up((size_t)dm.Ef * B, 16) * d);
   c->feat = cv.take<float>(align_up(NF * B, 16) * d); c->feat_n = cv.take<bf16>(align_up(NF * B, 16) * d);
   c->dlogits = cv.take<float>(align_up(NF * B, 16) * dm.Vpad);
+  // attention: chunk partials (max over levels), tickets, tensor maps
+  c->attn_chunk = dm.dh == 64 ? 256 : 128;
+  size_t part_max = 0;
+  for (int l = 0; l < 3; ++l) {
+    c->attn_max_chunks[l] = (dm.P + dm.cap[l] + c->attn_chunk - 1) / c->attn_chunk;
+    c->attn_mrows[l] = round_up(fm_rows_per_seq(dm, l) * (dm.H / dm.Hkv), 16);
+    const size_t need = B * dm.Hkv * (size_t)c->attn_max_chunks[l] * c->attn_mrows[l] * (dm.dh + 2);
+    part_max = need > part_max ? need : part_max;
+  }
+  c->attn_part = cv.take<float>(part_max);
+  c->attn_ticket = cv.take<int>(B * dm.Hkv);
+  int n_layers = 0;
+  for (int s = 0; s < 5; ++s) n_layers += c->cfg.layers[s];
+  c->tmaps = cv.take<CUtensorMap>((size_t)2 * n_layers + 64);
   // prefill temporaries
   c->pre_a = cv.take<bf16>((size_t)PREFILL_CHUNK * d);
   c->pre_o = cv.take<float>((size_t)PREFILL_CHUNK * 2 * dm.Hkv * dm.dh);
@@ -284,14 +306,50 @@ __global__ void row_count_kernel(Dims dm, SeqState st, int batch) {
   st.n_active[0] = cnt[0]; st.n_active[1] = cnt[1]; st.n_active[2] = cnt[2]; st.n_active[3] = act;
 }
 
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// 2-D bf16 tensor [rows, cols] row-major, box [box_rows, 64 columns] (128 bytes), 128-byte swizzle.
+// Returns the index of the new map in ctx->tmaps_host, or -1.
+int add_tmap_bf16(fm_ctx* c, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (fn == nullptr) return -1;
+  CUtensorMap m;
+  const cuuint64_t gdim[2] = {cols, rows};
+  const cuuint64_t gstride[1] = {cols * 2};
+  const cuuint32_t box[2] = {64, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  if (fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return -1;
+  c->tmaps_host.push_back(m);
+  return (int)c->tmaps_host.size() - 1;
+}
+
 void attention(fm_ctx* c, int level, int rows, const LayerDev& L) {
   const Dims& dm = c->dm;
-  dim3 grid(rows, dm.H);
+  AttnArgs a{dm, c->st, c->batch, level, c->qbuf, c->tmaps + L.tmK, c->tmaps + L.tmV, c->attn_part, c->attn_ticket,
+             c->a_attn, c->attn_max_chunks[level], c->attn_mrows[level]};
+  dim3 grid(c->attn_max_chunks[level], dm.Hkv, c->batch);
   const long pi = prof_open(c, PROF_ATTN, 0.0);
-  if (dm.dh == 32) LAUNCH(c, attn_rows_kernel<32>, grid, 128, 0, dm, c->st, c->batch, level, c->qbuf, L.K, L.V, c->a_attn);
-  else if (dm.dh == 64) LAUNCH(c, attn_rows_kernel<64>, grid, 128, 0, dm, c->st, c->batch, level, c->qbuf, L.K, L.V, c->a_attn);
-  else LAUNCH(c, attn_rows_kernel<128>, grid, 128, 0, dm, c->st, c->batch, level, c->qbuf, L.K, L.V, c->a_attn);
+  if (dm.dh == 64) LAUNCH(c, (attn_split_kernel<64, 256>), grid, 128, (AttnSmem<64, 256>::BYTES), a);
+  else LAUNCH(c, (attn_split_kernel<128, 128>), grid, 128, (AttnSmem<128, 128>::BYTES), a);
   prof_close(c, pi);
+  (void)rows;
 }
 
 // one stack of pre-norm blocks on the rows of its level (a2/a4/a6/a8/a10)
@@ -482,6 +540,17 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
     TRY(upload_bf16(c->headA + (size_t)h * dpad * d, A, d * d, tmp));
     TRY(upload_f32(c->head_g + (size_t)h * d, g, d));
   }
+  // TMA descriptors of the KV caches: each cache is a 2-D [max_batch*Hkv*slots, dh] bf16 matrix
+  for (int s = 0; s < 5; ++s)
+    for (auto& L : c->layers[s]) {
+      const uint64_t rows = (uint64_t)dm.max_batch * dm.Hkv * (dm.P + dm.cap[STACK_LEVEL[s]]);
+      L.tmK = add_tmap_bf16(c, L.K, rows, dm.dh, 64);
+      L.tmV = add_tmap_bf16(c, L.V, rows, dm.dh, 64);
+      if (L.tmK < 0 || L.tmV < 0) { delete c; return FM_ERR_CUDA; }
+    }
+  TRYCUDA(cudaMemcpy(c->tmaps, c->tmaps_host.data(), c->tmaps_host.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice));
+  TRYCUDA(cudaFuncSetAttribute(attn_split_kernel<64, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<64, 256>::BYTES));
+  TRYCUDA(cudaFuncSetAttribute(attn_split_kernel<128, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<128, 128>::BYTES));
   std::vector<double> freq(dm.dh / 2);
   for (int i = 0; i < dm.dh / 2; ++i)
     freq[i] = dm.theta != 0.f ? pow((double)dm.theta, -2.0 * (double)i / (double)dm.dh) : 0.0;
