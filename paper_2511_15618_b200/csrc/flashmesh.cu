@@ -16,12 +16,13 @@
 #include "fm_attention.cuh"
 #include "fm_common.cuh"
 #include "fm_gemm.cuh"
+#include "fm_gemm_tc.cuh"
 #include "fm_kernels.cuh"
 
 namespace {
 
 constexpr int STACK_LEVEL[5] = {0, 1, 2, 1, 0};
-constexpr int PREFILL_CHUNK = 512;      // conditioning rows projected per launch group
+constexpr int PREFILL_CHUNK = 256;      // conditioning rows projected per launch group
 
 struct LayerDev {
   bf16 *Wqkv, *Wo, *W1, *W2;
@@ -50,7 +51,7 @@ struct fm_ctx {
   // state
   SeqState st;
   // activations
-  float *xc, *xv, *xf, *qkv, *qbuf, *logits, *tmp3d;
+  float *xc, *xv, *xf, *qbuf, *logits, *tmp3d;
   bf16 *a_norm, *a_cat, *a_attn, *a_ff;
   float *hc_ring, *hv_ring, *trif_ring, *triv_ring, *zc, *zv, *zf;
   // draft
@@ -62,6 +63,12 @@ struct fm_ctx {
   int attn_chunk, attn_max_chunks[3], attn_mrows[3];
   CUtensorMap* tmaps;                    // device array
   std::vector<CUtensorMap> tmaps_host;
+  struct TmapKey { const void* base; uint64_t rows, cols; uint32_t box_rows; };
+  std::vector<TmapKey> tmap_keys;
+  size_t tmaps_cap, tmaps_uploaded;
+  // split-K partial tiles of the GEMM in flight
+  float* gpart;
+  size_t gpart_floats;
   // prefill temporaries
   bf16* pre_a;
   float* pre_o;
@@ -78,6 +85,7 @@ struct fm_ctx {
   size_t prof_used;
   double prof_ms[3], prof_bytes[3];
   long long prof_n[3];
+  int launch_error;     // first error met while enqueueing (capacity, descriptor creation)
   int batch;
   bool gen_fresh;       // no fm_generate call since the last fm_prefill
   std::vector<int> plen_host;
@@ -174,7 +182,7 @@ void carve(fm_ctx* c, Carver& cv) {
   // activations (row counts padded to 16 so that later tiles never run off the end)
   const size_t Rc = align_up(B * dm.R1, 16), Rv = align_up(B * dm.mv, 16), Rf = align_up(B * dm.mf, 16);
   c->xc = cv.take<float>(Rc * d); c->xv = cv.take<float>(Rv * d); c->xf = cv.take<float>(Rf * d);
-  c->qkv = cv.take<float>(Rc * qkvw); c->qbuf = cv.take<float>(Rc * hd);
+  c->qbuf = cv.take<float>(Rc * hd);
   c->logits = cv.take<float>(Rc * dm.Vpad); c->tmp3d = cv.take<float>(Rv * 3 * d);
   c->a_norm = cv.take<bf16>(Rc * d); c->a_cat = cv.take<bf16>(Rv * 3 * d);
   c->a_attn = cv.take<bf16>(Rc * hd); c->a_ff = cv.take<bf16>(Rc * dm.dff);
@@ -184,7 +192,7 @@ void carve(fm_ctx* c, Carver& cv) {
   c->zf = cv.take<float>(B * FM_RING_F * d);
   // draft
   const size_t NF = 8 + 9 * (size_t)dm.Ef;
-  c->dh_a = cv.take<bf16>((size_t)dm.NH * B * d); c->dh_y = cv.take<float>((size_t)dm.NH * B * d);
+  c->dh_a = cv.take<bf16>(((size_t)dm.NH * B + 16) * d); c->dh_y = cv.take<float>((size_t)dm.NH * B * d);
   c->up_in_v = cv.take<bf16>(align_up((2 + 3 * (size_t)dm.Ef) * B, 16) * d);
   c->up_in_f = cv.take<bf16>(align_up((size_t)dm.Ef * B, 16) * d);
   c->feat = cv.take<float>(align_up(NF * B, 16) * d); c->feat_n = cv.take<bf16>(align_up(NF * B, 16) * d);
@@ -202,7 +210,17 @@ void carve(fm_ctx* c, Carver& cv) {
   c->attn_ticket = cv.take<int>(B * dm.Hkv);
   int n_layers = 0;
   for (int s = 0; s < 5; ++s) n_layers += c->cfg.layers[s];
-  c->tmaps = cv.take<CUtensorMap>((size_t)2 * n_layers + 64);
+  c->tmaps_cap = (size_t)6 * n_layers + 128;
+  c->tmaps = cv.take<CUtensorMap>(c->tmaps_cap);
+  {
+    // per row at most ~2 * 148 * 128 partial floats (split * padded M), see gemm()
+    size_t rows_max = align_up(B * dm.R1, 16);
+    const size_t nf_rows = align_up((8 + 9 * (size_t)dm.Ef) * B, 16);
+    rows_max = rows_max > nf_rows ? rows_max : nf_rows;
+    rows_max = rows_max > 256 ? rows_max : 256;
+    c->gpart_floats = rows_max * 40960;
+    c->gpart = cv.take<float>(c->gpart_floats);
+  }
   // prefill temporaries
   c->pre_a = cv.take<bf16>((size_t)PREFILL_CHUNK * d);
   c->pre_o = cv.take<float>((size_t)PREFILL_CHUNK * 2 * dm.Hkv * dm.dh);
@@ -270,42 +288,6 @@ inline void prof_close(fm_ctx* c, long i) {
   if (i >= 0) cudaEventRecord(c->prof_ev[2 * i + 1], c->stream);
 }
 
-void gemm(fm_ctx* c, int mode, const bf16* W, const bf16* A, void* out, int M, int K, int R, int ldo,
-          const int* n_active, int nz = 1, long long sW = 0, long long sA = 0, long long sO = 0) {
-  if (R <= 0) return;
-  GemmArgs g{W, A, out, M, K, R, ldo, sW, sA, sO, n_active};
-  dim3 grid((M + 3) / 4, (R + 15) / 16, nz);
-  const long pi = prof_open(c, PROF_GEMM, 2.0 * M * K * nz);       // algorithmic bytes: the weight matrix once
-  switch (mode) {
-    case GEMM_STORE_F32: LAUNCH(c, gemm_simt_kernel<GEMM_STORE_F32>, grid, 128, 0, g); break;
-    case GEMM_ADD_F32: LAUNCH(c, gemm_simt_kernel<GEMM_ADD_F32>, grid, 128, 0, g); break;
-    case GEMM_GELU_BF16: LAUNCH(c, gemm_simt_kernel<GEMM_GELU_BF16>, grid, 128, 0, g); break;
-    default: LAUNCH(c, gemm_simt_kernel<GEMM_STORE_BF16>, grid, 128, 0, g); break;
-  }
-  prof_close(c, pi);
-}
-
-__global__ void to_bf16_kernel(const float* __restrict__ x, bf16* __restrict__ out, size_t n) {
-  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) out[i] = __float2bfloat16(x[i]);
-}
-
-// rows fed at each level in this pass (n_active[level]); n_active[3] = unfinished sequences
-__global__ void row_count_kernel(Dims dm, SeqState st, int batch) {
-  if (threadIdx.x != 0 || blockIdx.x != 0) return;
-  int cnt[3] = {0, 0, 0}, act = 0;
-  for (int b = 0; b < batch; ++b) {
-    const int n = st.nrow[b], L = st.L[b];
-    if (n <= 0) continue;
-    act++;
-    for (int l = 0; l < 3; ++l) {
-      const int r = fm_ratio(l);
-      cnt[l] += (L + n - 1) / r - (L + r - 1) / r + 1;
-    }
-  }
-  st.n_active[0] = cnt[0]; st.n_active[1] = cnt[1]; st.n_active[2] = cnt[2]; st.n_active[3] = act;
-}
-
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -340,6 +322,83 @@ int add_tmap_bf16(fm_ctx* c, const void* base, uint64_t rows, uint64_t cols, uin
   return (int)c->tmaps_host.size() - 1;
 }
 
+// index of the tensor map for a bf16 matrix / box, created on first use (all call sites are
+// visited by the first pass, before any timing or capture)
+int tmap_for(fm_ctx* c, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  for (size_t i = 0; i < c->tmap_keys.size(); ++i) {
+    const auto& k = c->tmap_keys[i];
+    if (k.base == base && k.rows == rows && k.cols == cols && k.box_rows == box_rows) return (int)i;
+  }
+  if (c->tmaps_host.size() >= c->tmaps_cap) return -1;
+  const int idx = add_tmap_bf16(c, base, rows, cols, box_rows);
+  if (idx < 0) return -1;
+  c->tmap_keys.push_back({base, rows, cols, box_rows});
+  cudaMemcpyAsync(c->tmaps + idx, &c->tmaps_host[idx], sizeof(CUtensorMap), cudaMemcpyHostToDevice, c->stream);
+  cudaStreamSynchronize(c->stream);
+  return idx;
+}
+
+// part[z][n][m] = partial of W[w_row0 + m, :] . A[a_row0 + n, :] over K range z (see fm_gemm_tc.cuh).
+// W: [w_rows_alloc, K] bf16 (rows padded to 128), A: [a_rows_alloc, K] bf16 (rows padded to 16).
+// Returns the view the consumer kernel needs.  The K split depends on (M, K) only.
+PartView gemm(fm_ctx* c, const bf16* W, size_t w_rows_alloc, int w_row0, const bf16* A, size_t a_rows_alloc, int a_row0,
+              int M, int K, int R, const int* n_active) {
+  PartView pv{c->gpart, 0, 0, 0};
+  if (R <= 0) return pv;
+  const int tiles = (M + tc::BM - 1) / tc::BM, slabs = K / tc::BK;
+  int split = (148 + tiles / 2) / tiles;
+  split = split < 1 ? 1 : split;
+  split = split > slabs ? slabs : split;
+  split = split > 32 ? 32 : split;
+  const int ldm = tiles * tc::BM;
+  const int Rpad = round_up(R, 16);
+  pv.nsplit = split;
+  pv.ldm = ldm;
+  pv.split_stride = (long long)Rpad * ldm;
+  if ((size_t)split * Rpad * ldm > c->gpart_floats) { c->launch_error = FM_ERR_CAPACITY; return pv; }
+  const int tW = tmap_for(c, W, w_rows_alloc, K, tc::BM);
+  const long pi = prof_open(c, PROF_GEMM, 2.0 * M * K);            // algorithmic bytes: the weight matrix once
+  for (int n0 = 0; n0 < Rpad; n0 += 256) {                         // N tiles of at most 256 rows
+    const int N = Rpad - n0 < 256 ? Rpad - n0 : 256;
+    const int tA = tmap_for(c, A, a_rows_alloc, K, N);
+    if (tW < 0 || tA < 0) { c->launch_error = FM_ERR_CUDA; break; }
+    tc::Args g{c->tmaps + tW, c->tmaps + tA, c->gpart + (size_t)n0 * ldm, M, K, N, (R - n0 < N ? R - n0 : N), ldm,
+               pv.split_stride, split, w_row0, a_row0 + n0, n_active, c->st.status};
+    const int smem = tc::smem_bytes(N);
+    LAUNCH(c, tc::gemm_tc_kernel, dim3(tiles, split), 128, smem, g);
+  }
+  prof_close(c, pi);
+  return pv;
+}
+
+template <int MODE>
+void fold(fm_ctx* c, const PartView& pv, void* out, int ldo, int M, int R) {
+  if (R <= 0) return;
+  const int gy = (M + 1023) / 1024;
+  LAUNCH(c, fold_kernel<MODE>, dim3(R, gy), 256, 0, pv, out, ldo, M);
+}
+
+__global__ void to_bf16_kernel(const float* __restrict__ x, bf16* __restrict__ out, size_t n) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) out[i] = __float2bfloat16(x[i]);
+}
+
+// rows fed at each level in this pass (n_active[level]); n_active[3] = unfinished sequences
+__global__ void row_count_kernel(Dims dm, SeqState st, int batch) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  int cnt[3] = {0, 0, 0}, act = 0;
+  for (int b = 0; b < batch; ++b) {
+    const int n = st.nrow[b], L = st.L[b];
+    if (n <= 0) continue;
+    act++;
+    for (int l = 0; l < 3; ++l) {
+      const int r = fm_ratio(l);
+      cnt[l] += (L + n - 1) / r - (L + r - 1) / r + 1;
+    }
+  }
+  st.n_active[0] = cnt[0]; st.n_active[1] = cnt[1]; st.n_active[2] = cnt[2]; st.n_active[3] = act;
+}
+
 void attention(fm_ctx* c, int level, int rows, const LayerDev& L) {
   const Dims& dm = c->dm;
   AttnArgs a{dm, c->st, c->batch, level, c->qbuf, c->tmaps + L.tmK, c->tmaps + L.tmV, c->attn_part, c->attn_ticket,
@@ -352,28 +411,38 @@ void attention(fm_ctx* c, int level, int rows, const LayerDev& L) {
   (void)rows;
 }
 
-// one stack of pre-norm blocks on the rows of its level (a2/a4/a6/a8/a10)
-void run_stack(fm_ctx* c, int s, float* x, float* stash_ring) {
+inline size_t pad128(size_t v) { return align_up(v, 128); }
+
+// one stack of pre-norm blocks on the rows of its level (a2/a4/a6/a8/a10).  `pend` holds GEMM
+// partials that still have to be folded into x (mode 1: add, 2: store) by the first norm kernel.
+void run_stack(fm_ctx* c, int s, float* x, size_t x_rows_alloc, float* stash_ring, PartView pend, int pend_mode) {
   const Dims& dm = c->dm;
   const int level = STACK_LEVEL[s];
   const int rows = c->batch * fm_rows_per_seq(dm, level);
-  const int qkvw = (dm.H + 2 * dm.Hkv) * dm.dh, hd = dm.H * dm.dh;
+  const int qkvw = (dm.H + 2 * dm.Hkv) * dm.dh, hd = dm.H * dm.dh, d = dm.d;
+  const size_t Rc_alloc = align_up((size_t)dm.max_batch * dm.R1, 16);
   const int* na = c->st.n_active + level;
   const int nl = (int)c->layers[s].size();
+  (void)x_rows_alloc;
   for (int l = 0; l < nl; ++l) {
     const LayerDev& L = c->layers[s][l];
+    LAUNCH(c, resid_norm_kernel, rows, 256, d * sizeof(float), x, pend, pend_mode, L.g1, c->a_norm, d, dm.eps);
     if (stash_ring != nullptr && l == nl - 1)
-      LAUNCH(c, ring_store_kernel, rows, 128, 0, dm, c->st, c->batch, level, x, stash_ring, dm.d);
-    LAUNCH(c, rmsnorm_kernel, rows, 256, 0, x, L.g1, c->a_norm, dm.d, dm.eps);
-    gemm(c, GEMM_STORE_F32, L.Wqkv, c->a_norm, c->qkv, qkvw, dm.d, rows, qkvw, na);
-    LAUNCH(c, rope_append_kernel, rows, 128, dm.dh * sizeof(float), dm, c->st, c->batch, level, c->qkv, c->inv_freq,
+      LAUNCH(c, ring_store_kernel, rows, 128, 0, dm, c->st, c->batch, level, x, stash_ring, d);
+    PartView pq = gemm(c, L.Wqkv, pad128(qkvw), 0, c->a_norm, Rc_alloc, 0, qkvw, d, rows, na);
+    LAUNCH(c, rope_append_kernel, rows, 128, dm.dh * sizeof(float), dm, c->st, c->batch, level, pq, c->inv_freq,
            c->qbuf, L.K, L.V);
     attention(c, level, rows, L);
-    gemm(c, GEMM_ADD_F32, L.Wo, c->a_attn, x, dm.d, hd, rows, dm.d, na);
-    LAUNCH(c, rmsnorm_kernel, rows, 256, 0, x, L.g2, c->a_norm, dm.d, dm.eps);
-    gemm(c, GEMM_GELU_BF16, L.W1, c->a_norm, c->a_ff, dm.dff, dm.d, rows, dm.dff, na);
-    gemm(c, GEMM_ADD_F32, L.W2, c->a_ff, x, dm.d, dm.dff, rows, dm.d, na);
+    PartView po = gemm(c, L.Wo, pad128(d), 0, c->a_attn, Rc_alloc, 0, d, hd, rows, na);
+    LAUNCH(c, resid_norm_kernel, rows, 256, d * sizeof(float), x, po, 1, L.g2, c->a_norm, d, dm.eps);
+    PartView p1 = gemm(c, L.W1, pad128(dm.dff), 0, c->a_norm, Rc_alloc, 0, dm.dff, d, rows, na);
+    fold<FOLD_GELU_BF16>(c, p1, c->a_ff, dm.dff, dm.dff, rows);
+    pend = gemm(c, L.W2, pad128(d), 0, c->a_ff, Rc_alloc, 0, d, dm.dff, rows, na);
+    pend_mode = 1;
   }
+  // fold the last FFN output into the residual stream (no norm)
+  LAUNCH(c, resid_norm_kernel, rows, 256, d * sizeof(float), x, pend, pend_mode, (const float*)nullptr, (bf16*)nullptr, d,
+         dm.eps);
 }
 
 // the verify forward pass over st.cand / st.nrow (a1..a11)
@@ -381,30 +450,35 @@ void forward(fm_ctx* c, float* logits_out) {
   const Dims& dm = c->dm;
   const int B = c->batch, d = dm.d;
   const int Rc = B * dm.R1, Rv = B * dm.mv, Rf = B * dm.mf;
+  const size_t Rc_alloc = align_up((size_t)dm.max_batch * dm.R1, 16), Rv_alloc = align_up((size_t)dm.max_batch * dm.mv, 16);
   const int* na = c->st.n_active;
+  const PartView none{nullptr, 0, 0, 0};
   LAUNCH(c, row_count_kernel, 1, 32, 0, dm, c->st, B);
   LAUNCH(c, embed_kernel, Rc, 128, 0, dm, c->st, B, c->E, c->xc);
-  run_stack(c, 0, c->xc, nullptr);
+  run_stack(c, 0, c->xc, Rc_alloc, nullptr, none, 0);
   LAUNCH(c, ring_store_kernel, Rc, 128, 0, dm, c->st, B, 0, c->xc, c->hc_ring, d);
   LAUNCH(c, shorten_gather_kernel, Rv, 128, 0, dm, c->st, B, 1, c->hc_ring, c->a_cat);
-  gemm(c, GEMM_STORE_F32, c->S_cv, c->a_cat, c->xv, d, 3 * d, Rv, d, na + 1);
-  run_stack(c, 1, c->xv, nullptr);
+  PartView pv = gemm(c, c->S_cv, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rv, na + 1);
+  run_stack(c, 1, c->xv, Rv_alloc, nullptr, pv, 2);
   LAUNCH(c, ring_store_kernel, Rv, 128, 0, dm, c->st, B, 1, c->xv, c->hv_ring, d);
   LAUNCH(c, shorten_gather_kernel, Rf, 128, 0, dm, c->st, B, 2, c->hv_ring, c->a_cat);
-  gemm(c, GEMM_STORE_F32, c->S_vf, c->a_cat, c->xf, d, 3 * d, Rf, d, na + 2);
-  run_stack(c, 2, c->xf, c->zf);
+  pv = gemm(c, c->S_vf, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rf, na + 2);
+  run_stack(c, 2, c->xf, 0, c->zf, pv, 2);
   LAUNCH(c, to_bf16_kernel, (Rf * d + 255) / 256, 256, 0, c->xf, c->a_norm, (size_t)Rf * d);
-  gemm(c, GEMM_STORE_F32, c->U_fv, c->a_norm, c->tmp3d, 3 * d, d, Rf, 3 * d, na + 2);
+  pv = gemm(c, c->U_fv, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rf, na + 2);
+  fold<FOLD_F32>(c, pv, c->tmp3d, 3 * d, 3 * d, Rf);
   LAUNCH(c, ring_store_kernel, Rf, 128, 0, dm, c->st, B, 2, c->tmp3d, c->trif_ring, 3 * d);
   LAUNCH(c, upsample_add_kernel, Rv, 128, 0, dm, c->st, B, 1, c->hv_ring, c->trif_ring, c->xv);
-  run_stack(c, 3, c->xv, c->zv);
+  run_stack(c, 3, c->xv, Rv_alloc, c->zv, none, 0);
   LAUNCH(c, to_bf16_kernel, (Rv * d + 255) / 256, 256, 0, c->xv, c->a_norm, (size_t)Rv * d);
-  gemm(c, GEMM_STORE_F32, c->U_vc, c->a_norm, c->tmp3d, 3 * d, d, Rv, 3 * d, na + 1);
+  pv = gemm(c, c->U_vc, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rv, na + 1);
+  fold<FOLD_F32>(c, pv, c->tmp3d, 3 * d, 3 * d, Rv);
   LAUNCH(c, ring_store_kernel, Rv, 128, 0, dm, c->st, B, 1, c->tmp3d, c->triv_ring, 3 * d);
   LAUNCH(c, upsample_add_kernel, Rc, 128, 0, dm, c->st, B, 0, c->hc_ring, c->triv_ring, c->xc);
-  run_stack(c, 4, c->xc, c->zc);
+  run_stack(c, 4, c->xc, Rc_alloc, c->zc, none, 0);
   LAUNCH(c, rmsnorm_kernel, Rc, 256, 0, c->xc, c->g_out, c->a_norm, d, dm.eps);
-  gemm(c, GEMM_STORE_F32, c->W_out, c->a_norm, c->logits, dm.V, d, Rc, dm.Vpad, na);
+  pv = gemm(c, c->W_out, dm.Vpad, 0, c->a_norm, Rc_alloc, 0, dm.V, d, Rc, na);
+  fold<FOLD_F32>(c, pv, c->logits, dm.Vpad, dm.V, Rc);
   LAUNCH(c, verify_top2_kernel, Rc, 256, 0, dm, c->st, B, c->logits, logits_out);
 }
 
@@ -416,15 +490,22 @@ void draft(fm_ctx* c, float* logits_out, float* margin_out) {
     const int dpad = round_up(d, 128);
     const int NF = 8 + 9 * dm.Ef;
     const int* na = c->st.n_active + 3;
+    const size_t MB = dm.max_batch;
     LAUNCH(c, draft_prep_kernel, dim3(B, dm.NH), 256, 0, dm, c->st, B, c->zc, c->zv, c->zf, c->head_g, c->dh_a);
-    gemm(c, GEMM_STORE_F32, c->headA, c->dh_a, c->dh_y, d, d, B, d, na, dm.NH, (long long)dpad * d,
-         (long long)dm.max_batch * d, (long long)dm.max_batch * d);
+    for (int h = 0; h < dm.NH; ++h) {
+      PartView ph = gemm(c, c->headA, (size_t)dm.NH * dpad, h * dpad, c->dh_a, (size_t)dm.NH * MB + 16, h * (int)MB, d, d, B, na);
+      fold<FOLD_F32>(c, ph, c->dh_y + (size_t)h * MB * d, d, d, B);
+    }
     LAUNCH(c, draft_residual_kernel, dim3(B, dm.NH), 128, 0, dm, c->st, B, c->zc, c->zv, c->zf, c->dh_y, c->feat,
            c->up_in_v, c->up_in_f);
-    gemm(c, GEMM_STORE_BF16, c->U_fv, c->up_in_f, c->up_in_v + (size_t)2 * B * d, 3 * d, d, dm.Ef * B, 3 * d, na);
-    gemm(c, GEMM_STORE_F32, c->U_vc, c->up_in_v, c->feat + (size_t)2 * B * d, 3 * d, d, (2 + 3 * dm.Ef) * B, 3 * d, na);
+    PartView pf = gemm(c, c->U_fv, pad128(3 * d), 0, c->up_in_f, align_up((size_t)dm.Ef * MB, 16), 0, 3 * d, d, dm.Ef * B, na);
+    fold<FOLD_BF16>(c, pf, c->up_in_v + (size_t)2 * B * d, 3 * d, 3 * d, dm.Ef * B);
+    PartView pu = gemm(c, c->U_vc, pad128(3 * d), 0, c->up_in_v, align_up((2 + 3 * (size_t)dm.Ef) * MB, 16), 0, 3 * d, d,
+                       (2 + 3 * dm.Ef) * B, na);
+    fold<FOLD_F32>(c, pu, c->feat + (size_t)2 * B * d, 3 * d, 3 * d, (2 + 3 * dm.Ef) * B);
     LAUNCH(c, rmsnorm_kernel, NF * B, 256, 0, c->feat, c->g_out, c->feat_n, d, dm.eps);
-    gemm(c, GEMM_STORE_F32, c->W_out, c->feat_n, c->dlogits, dm.V, d, NF * B, dm.Vpad, na);
+    PartView pl = gemm(c, c->W_out, dm.Vpad, 0, c->feat_n, align_up((size_t)NF * MB, 16), 0, dm.V, d, NF * B, na);
+    fold<FOLD_F32>(c, pl, c->dlogits, dm.Vpad, dm.V, NF * B);
   }
   LAUNCH(c, draft_pick_kernel, dim3(B, dm.R1), 256, 0, dm, c->st, B, c->dlogits, logits_out, margin_out);
 }
@@ -545,10 +626,13 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
     for (auto& L : c->layers[s]) {
       const uint64_t rows = (uint64_t)dm.max_batch * dm.Hkv * (dm.P + dm.cap[STACK_LEVEL[s]]);
       L.tmK = add_tmap_bf16(c, L.K, rows, dm.dh, 64);
+      c->tmap_keys.push_back({L.K, rows, (uint64_t)dm.dh, 64u});
       L.tmV = add_tmap_bf16(c, L.V, rows, dm.dh, 64);
+      c->tmap_keys.push_back({L.V, rows, (uint64_t)dm.dh, 64u});
       if (L.tmK < 0 || L.tmV < 0) { delete c; return FM_ERR_CUDA; }
     }
   TRYCUDA(cudaMemcpy(c->tmaps, c->tmaps_host.data(), c->tmaps_host.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(256)));
   TRYCUDA(cudaFuncSetAttribute(attn_split_kernel<64, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<64, 256>::BYTES));
   TRYCUDA(cudaFuncSetAttribute(attn_split_kernel<128, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<128, 128>::BYTES));
   std::vector<double> freq(dm.dh / 2);
@@ -627,7 +711,9 @@ int fm_prefill(fm_ctx* c, int32_t batch, const float* cond, const int32_t* promp
     for (int s = 0; s < 5; ++s)
       for (auto& L : c->layers[s]) {
         LAUNCH(c, rmsnorm_kernel, rows, 256, 0, cond + (size_t)r0 * dm.d, L.g1, c->pre_a, dm.d, dm.eps);
-        gemm(c, GEMM_STORE_F32, L.Wqkv + (size_t)dm.H * dm.dh * dm.d, c->pre_a, c->pre_o, kvw, dm.d, rows, kvw, nullptr);
+        PartView pk = gemm(c, L.Wqkv, pad128((size_t)(dm.H + 2 * dm.Hkv) * dm.dh), dm.H * dm.dh, c->pre_a, PREFILL_CHUNK, 0,
+                           kvw, dm.d, rows, nullptr);
+        fold<FOLD_F32>(c, pk, c->pre_o, kvw, kvw, rows);
         LAUNCH(c, prefix_store_kernel, rows, 128, 0, dm, STACK_LEVEL[s], r0, c->pre_o, L.K, L.V);
       }
   }
@@ -641,6 +727,7 @@ int fm_prefill(fm_ctx* c, int32_t batch, const float* cond, const int32_t* promp
   LAUNCH(c, arm_kernel, (batch + 127) / 128, 128, 0, dm, c->st, batch);
   LAUNCH(c, row_count_kernel, 1, 32, 0, dm, c->st, batch);
   CUDA_OK(cudaGetLastError());
+  if (c->launch_error != FM_OK) return c->launch_error;
   c->phase = 1;
   c->gen_fresh = true;
   return FM_OK;
@@ -666,6 +753,7 @@ int fm_draft(fm_ctx* c, int32_t* cand, float* draft_logits, float* draft_margin)
   const int n = c->batch * c->dm.R1;
   if (cand != nullptr) LAUNCH(c, copy_i32_kernel, (n + 127) / 128, 128, 0, c->st.cand, cand, n);
   CUDA_OK(cudaGetLastError());
+  if (c->launch_error != FM_OK) return c->launch_error;
   return FM_OK;
 }
 
@@ -678,6 +766,7 @@ int fm_verify(fm_ctx* c, const int32_t* cand, int32_t* argmax, float* logits, fl
   if (argmax != nullptr) LAUNCH(c, copy_i32_kernel, (n + 127) / 128, 128, 0, c->st.o, argmax, n);
   if (margin != nullptr) LAUNCH(c, copy_f32_kernel, (n + 127) / 128, 128, 0, c->st.margin, margin, n);
   CUDA_OK(cudaGetLastError());
+  if (c->launch_error != FM_OK) return c->launch_error;
   c->phase = 2;
   return FM_OK;
 }
@@ -690,6 +779,7 @@ int fm_accept(fm_ctx* c, const int32_t* force_len, const int32_t* force_tok, int
          emitted, kv_len, (const GenOut*)nullptr);
   LAUNCH(c, row_count_kernel, 1, 32, 0, c->dm, c->st, c->batch);
   CUDA_OK(cudaGetLastError());
+  if (c->launch_error != FM_OK) return c->launch_error;
   c->phase = 1;
   return FM_OK;
 }

@@ -1,67 +1,34 @@
-// Skinny weight-streaming GEMM: out[r, m] = sum_k A[r, k] * W[m, k]  (bf16 operands, fp32 sums).
+// Row-wise consumers of the split-K partial tiles written by the tensor-core GEMM:
+// part[z][row][m], z < nsplit, summed in split order (a fixed order).
 #pragma once
 #include "fm_common.cuh"
 
-enum GemmMode { GEMM_STORE_F32 = 0, GEMM_ADD_F32 = 1, GEMM_GELU_BF16 = 2, GEMM_STORE_BF16 = 3 };
-
-struct GemmArgs {
-  const bf16* W;      // [M(pad), K] row-major
-  const bf16* A;      // [R, K] row-major
-  void* out;          // [R, ldo] fp32 or bf16
-  int M, K, R, ldo;
-  long long strideW, strideA, strideO;   // per blockIdx.z (elements)
-  const int* n_active;                   // skip all work when *n_active == 0 (may be null)
+struct PartView {
+  const float* part;      // null: nothing pending
+  int nsplit;
+  long long split_stride; // elements between splits
+  int ldm;                // elements between rows
 };
+
+__device__ inline float part_sum(const PartView& pv, int row, int m) {
+  const float* p = pv.part + (size_t)row * pv.ldm + m;
+  float v = 0.f;
+  for (int z = 0; z < pv.nsplit; ++z) v += __ldcg(p + (size_t)z * pv.split_stride);
+  return v;
+}
 
 __device__ inline float gelu_erf(float x) { return 0.5f * x * (1.f + erff(x * 0.70710678118654752f)); }
 
-template <int MODE>
-__device__ inline void gemm_store(void* out, size_t idx, float v) {
-  if (MODE == GEMM_STORE_F32) reinterpret_cast<float*>(out)[idx] = v;
-  else if (MODE == GEMM_ADD_F32) reinterpret_cast<float*>(out)[idx] += v;
-  else if (MODE == GEMM_GELU_BF16) reinterpret_cast<bf16*>(out)[idx] = __float2bfloat16(gelu_erf(v));
-  else reinterpret_cast<bf16*>(out)[idx] = __float2bfloat16(v);
-}
+enum FoldMode { FOLD_F32 = 0, FOLD_BF16 = 1, FOLD_GELU_BF16 = 2 };
 
-// CUDA-core version: one warp per output feature, a tile of 16 rows, lanes stride over K in
-// 16-byte pieces; the warp sum has a fixed shuffle order, so results do not depend on R.
+// out[row][m] = f(sum of partials); grid (rows, ceil(M / (4*256))), block 256
 template <int MODE>
-__global__ void __launch_bounds__(128) gemm_simt_kernel(GemmArgs g) {
-  if (g.n_active != nullptr && *g.n_active == 0) return;
-  constexpr int TR = 16;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m = blockIdx.x * 4 + warp;
-  const int r0 = blockIdx.y * TR;
-  if (m >= g.M) return;
-  const bf16* W = g.W + blockIdx.z * g.strideW + (size_t)m * g.K;
-  const bf16* A = g.A + blockIdx.z * g.strideA;
-  float acc[TR];
-#pragma unroll
-  for (int r = 0; r < TR; ++r) acc[r] = 0.f;
-  const int nr = min(TR, g.R - r0);
-  for (int k = lane * 8; k < g.K; k += 256) {
-    const uint4 wu = *reinterpret_cast<const uint4*>(W + k);
-    const __nv_bfloat162* w2 = reinterpret_cast<const __nv_bfloat162*>(&wu);
-    float wf[8];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) { const float2 f = __bfloat1622float2(w2[e]); wf[2 * e] = f.x; wf[2 * e + 1] = f.y; }
-#pragma unroll
-    for (int r = 0; r < TR; ++r) {
-      if (r < nr) {
-        const uint4 au = *reinterpret_cast<const uint4*>(A + (size_t)(r0 + r) * g.K + k);
-        const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&au);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float2 f = __bfloat1622float2(a2[e]);
-          acc[r] = fmaf(wf[2 * e], f.x, acc[r]);
-          acc[r] = fmaf(wf[2 * e + 1], f.y, acc[r]);
-        }
-      }
-    }
-  }
-#pragma unroll
-  for (int r = 0; r < TR; ++r) {
-    const float v = warp_sum(acc[r]);
-    if (lane == 0 && r < nr) gemm_store<MODE>(g.out, blockIdx.z * g.strideO + (size_t)(r0 + r) * g.ldo + m, v);
+__global__ void fold_kernel(PartView pv, void* __restrict__ out, int ldo, int M) {
+  const int row = blockIdx.x;
+  for (int m = blockIdx.y * blockDim.x + threadIdx.x; m < M; m += gridDim.y * blockDim.x) {
+    const float v = part_sum(pv, row, m);
+    if (MODE == FOLD_F32) reinterpret_cast<float*>(out)[(size_t)row * ldo + m] = v;
+    else if (MODE == FOLD_BF16) reinterpret_cast<bf16*>(out)[(size_t)row * ldo + m] = __float2bfloat16(v);
+    else reinterpret_cast<bf16*>(out)[(size_t)row * ldo + m] = __float2bfloat16(gelu_erf(v));
   }
 }

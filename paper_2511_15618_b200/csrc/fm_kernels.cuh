@@ -1,6 +1,7 @@
 // Element-wise, row-wise and bookkeeping kernels of the decode step.
 #pragma once
 #include "fm_common.cuh"
+#include "fm_gemm.cuh"
 
 // ------------------------------------------------------------------------------------------
 // block reductions (blockDim.x multiple of 32, <= 1024)
@@ -36,8 +37,30 @@ __global__ void embed_kernel(Dims dm, SeqState st, int batch, const bf16* __rest
 }
 
 // ------------------------------------------------------------------------------------------
-// RMSNorm of fp32 rows -> bf16 GEMM operand rows:  out = x / sqrt(mean(x^2)+eps) * g
+// Residual fold + RMSNorm: first x[row] (+)= sum of the pending GEMM partials (mode 1 adds them
+// to the residual stream, mode 2 replaces it, mode 0 leaves x alone), then, if a gain is given,
+// out = bf16(x / sqrt(mean(x^2)+eps) * g), the next GEMM's operand row.  One CTA per row.
 // ------------------------------------------------------------------------------------------
+__global__ void resid_norm_kernel(float* __restrict__ x, PartView pv, int mode, const float* __restrict__ g,
+                                  bf16* __restrict__ out, int d, float eps) {
+  __shared__ float sh[32];
+  extern __shared__ float xrow[];                   // d floats
+  float* xr = x + (size_t)blockIdx.x * d;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    float v = mode == 2 ? 0.f : xr[i];
+    if (mode != 0) { v += part_sum(pv, blockIdx.x, i); xr[i] = v; }
+    xrow[i] = v;
+    ss += v * v;
+  }
+  if (g == nullptr) return;
+  ss = block_sum(ss, sh);
+  const float inv = rsqrtf(ss / (float)d + eps);
+  for (int i = threadIdx.x; i < d; i += blockDim.x)
+    out[(size_t)blockIdx.x * d + i] = __float2bfloat16(xrow[i] * inv * g[i]);
+}
+
+// RMSNorm of read-only fp32 rows (conditioning vectors, draft features) -> bf16 operand rows
 __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ g, bf16* __restrict__ out,
                                int d, float eps) {
   __shared__ float sh[32];
@@ -53,17 +76,15 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
 // ------------------------------------------------------------------------------------------
 // RoPE on q and k (rotate-half pairs (i, i+dh/2), angle = pos * theta^(-2i/dh), evaluated in
 // double), then append k, v to the level's cache at slot P + pos % cap.
-// qkv: fp32 [rows, (H+2Hkv)*dh]; q_out: fp32 [rows, H*dh]; caches: bf16 [B, Hkv, slots, dh].
+// qkv: split-K partials of [rows, (H+2Hkv)*dh]; q_out: fp32 [rows, H*dh]; caches: bf16 [B, Hkv, slots, dh].
 // ------------------------------------------------------------------------------------------
-__global__ void rope_append_kernel(Dims dm, SeqState st, int batch, int level, const float* __restrict__ qkv,
+__global__ void rope_append_kernel(Dims dm, SeqState st, int batch, int level, PartView qkv,
                                    const double* __restrict__ inv_freq, float* __restrict__ q_out,
                                    bf16* __restrict__ Kc, bf16* __restrict__ Vc) {
   const int row = blockIdx.x;
   int b, p;
   const bool valid = fm_row_map(dm, st, batch, level, row, b, p);
   const int H = dm.H, Hkv = dm.Hkv, dh = dm.dh, half = dh / 2;
-  const int ldq = (H + 2 * Hkv) * dh;
-  const float* src = qkv + (size_t)row * ldq;
   const int slots = dm.P + dm.cap[level];
   const int slot = dm.P + (p % dm.cap[level]);
   extern __shared__ float cs[];                     // cos[half], sin[half]
@@ -78,7 +99,7 @@ __global__ void rope_append_kernel(Dims dm, SeqState st, int batch, int level, c
   const int pairs = (H + Hkv) * half;
   for (int t = threadIdx.x; t < pairs; t += blockDim.x) {
     const int head = t / half, i = t - head * half;
-    const float x1 = src[head * dh + i], x2 = src[head * dh + half + i];
+    const float x1 = part_sum(qkv, row, head * dh + i), x2 = part_sum(qkv, row, head * dh + half + i);
     const float c = cs[i], s = cs[half + i];
     const float y1 = x1 * c - x2 * s, y2 = x2 * c + x1 * s;
     if (head < H) {
@@ -92,10 +113,9 @@ __global__ void rope_append_kernel(Dims dm, SeqState st, int batch, int level, c
     }
   }
   if (valid) {
-    const float* vsrc = src + (H + Hkv) * dh;
     for (int t = threadIdx.x; t < Hkv * dh; t += blockDim.x) {
       const int hk = t / dh, i = t - hk * dh;
-      Vc[(((size_t)b * Hkv + hk) * slots + slot) * dh + i] = __float2bfloat16(vsrc[t]);
+      Vc[(((size_t)b * Hkv + hk) * slots + slot) * dh + i] = __float2bfloat16(part_sum(qkv, row, (H + Hkv) * dh + t));
     }
   }
 }

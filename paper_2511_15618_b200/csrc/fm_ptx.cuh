@@ -31,12 +31,14 @@ __device__ inline bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after `limit` polls (each poll itself blocks for a hardware time slice)
-// and returns false; the caller records the timeout and leaves without touching the data.
-__device__ inline bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t limit = 4000000u) {
-  for (uint32_t i = 0; i < limit; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  return false;
+// Bounded wait: gives up after about a tenth of a second of polling and returns false; the caller records
+// the timeout and leaves without touching the data.
+__device__ inline bool mbar_wait(uint64_t* bar, uint32_t parity, long long limit_cycles = 200000000ll) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity))
+    if (clock64() - t0 > limit_cycles) return false;
+  return true;
 }
 
 // ---------------------------------------------------------------- TMA
