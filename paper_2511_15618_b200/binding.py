@@ -246,7 +246,8 @@ class FlashMesh:
         with torch.cuda.device(self.device):
             self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
             base = (self.workspace.data_ptr() + 255) // 256 * 256
-            self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+            # a stream of its own: the legacy default stream cannot be captured into a CUDA graph
+            self.stream = stream if stream is not None else torch.cuda.Stream(self.device)
             fw, self._keep = make_weights(weights, (self.D + 8) // 9 if self.D else 0)
             rc, self.ctx = fm_create(self.cfg, fw, base, nbytes, self.stream.cuda_stream)
         if rc != 0:
@@ -269,6 +270,18 @@ class FlashMesh:
         if rc != 0:
             raise FmError(rc, where)
 
+    def _before(self):
+        """Order the context's stream after the caller's current stream (inputs are ready)."""
+        self.stream.wait_stream(self.torch.cuda.current_stream(self.device))
+
+    def _after(self, *tensors):
+        """Order the caller's current stream after the context's stream (outputs are ready)."""
+        cur = self.torch.cuda.current_stream(self.device)
+        cur.wait_stream(self.stream)
+        for t in tensors:
+            if t is not None:
+                t.record_stream(self.stream)
+
     def _dev(self, x, dtype):
         t = self.torch
         if isinstance(x, t.Tensor):
@@ -289,11 +302,15 @@ class FlashMesh:
         flat = np.concatenate([np.asarray(p, dtype=np.int32) for p in prompts] + [np.zeros(1, np.int32)])
         self._cond = self._dev(cond, t.float32)
         self._prompt = self._dev(flat, t.int32)
+        self._before()
         self._check(fm_prefill(self.ctx, B, self._cond.data_ptr(), self._prompt.data_ptr(), off), "fm_prefill")
+        self._after()
         self.batch = B
 
     def set_max_faces(self, max_faces):
+        self._before()
         self._check(fm_set_max_faces(self.ctx, list(max_faces)), "fm_set_max_faces")
+        self._after()
 
     def draft(self, want_logits=False):
         t = self.torch
@@ -301,8 +318,10 @@ class FlashMesh:
         cand = self._empty((B, D + 1), t.int32)
         dl = self._empty((B, D, self.V), t.float32) if want_logits else None
         dm = self._empty((B, max(D, 1)), t.float32)[:, :D].contiguous() if want_logits else None
+        self._before()
         self._check(fm_draft(self.ctx, cand.data_ptr(), dl.data_ptr() if dl is not None else None,
                              dm.data_ptr() if dm is not None and D > 0 else None), "fm_draft")
+        self._after(cand, dl, dm)
         return cand, dl, dm
 
     def verify(self, cand, want_logits=False):
@@ -312,8 +331,10 @@ class FlashMesh:
         o = self._empty((B, D + 1), t.int32)
         mg = self._empty((B, D + 1), t.float32)
         lg = self._empty((B, D + 1, self.V), t.float32) if want_logits else None
+        self._before()
         self._check(fm_verify(self.ctx, cand.data_ptr(), o.data_ptr(), lg.data_ptr() if lg is not None else None,
                               mg.data_ptr()), "fm_verify")
+        self._after(cand, o, lg, mg)
         return o, lg, mg
 
     def accept(self, force_len=None, force_tok=None):
@@ -324,9 +345,11 @@ class FlashMesh:
         n_acc = self._empty((B,), t.int32)
         em = self._empty((B, D + 1), t.int32)
         kv = self._empty((B, 3), t.int32)
+        self._before()
         self._check(fm_accept(self.ctx, fl.data_ptr() if fl is not None else None,
                               ft.data_ptr() if ft is not None else None, n_acc.data_ptr(), em.data_ptr(),
                               kv.data_ptr()), "fm_accept")
+        self._after(fl, ft, n_acc, em, kv)
         return n_acc, em, kv
 
     def generate(self, max_faces, truth=None, keep=None, plain=False, out=None, max_steps=0):
@@ -347,8 +370,10 @@ class FlashMesh:
             teacher.keep = self._keep_sched.data_ptr() if self._keep_sched is not None else None
             teacher.n_sched = int(self._keep_sched.shape[0]) if self._keep_sched is not None else 0
         stats = FmStats()
+        self._before()
         self._check(fm_generate(self.ctx, max_faces, out_tok.data_ptr(), stride, out_len.data_ptr(), teacher,
                                 1 if plain else 0, max_steps, stats), "fm_generate")
+        self._after(out_tok, out_len)
         return out_tok, out_len, stats
 
     def verify_bytes(self, kv_len):

@@ -48,6 +48,7 @@ struct fm_ctx {
   bf16 *S_cv, *S_vf, *U_fv, *U_vc, *W_out, *headA;
   float *g_out, *head_g;
   double* inv_freq;
+  float2* rope_tab;                      // [max level positions][dh/2] (cos, sin)
   // state
   SeqState st;
   // activations
@@ -86,6 +87,12 @@ struct fm_ctx {
   double prof_ms[3], prof_bytes[3];
   long long prof_n[3];
   int launch_error;     // first error met while enqueueing (capacity, descriptor creation)
+  // one decode pass (draft, teacher edit, verify, accept) captured as a CUDA graph
+  cudaGraph_t graph;
+  cudaGraphExec_t graph_exec;
+  int graph_batch;
+  int64_t graph_launches;
+  bool capturing, graph_unavailable;
   int batch;
   bool gen_fresh;       // no fm_generate call since the last fm_prefill
   std::vector<int> plen_host;
@@ -173,6 +180,7 @@ void carve(fm_ctx* c, Carver& cv) {
   c->g_out = cv.take<float>(d);
   c->head_g = cv.take<float>((size_t)dm.NH * d);
   c->inv_freq = cv.take<double>(dm.dh / 2);
+  c->rope_tab = cv.take<float2>((size_t)(dm.max_tokens + 1) * (dm.dh / 2));
   // state
   c->st.L = cv.take<int>(B); c->st.nrow = cv.take<int>(B); c->st.main_tok = cv.take<int>(B);
   c->st.done = cv.take<int>(B); c->st.t_end = cv.take<int>(B); c->st.plen = cv.take<int>(B);
@@ -329,7 +337,7 @@ int tmap_for(fm_ctx* c, const void* base, uint64_t rows, uint64_t cols, uint32_t
     const auto& k = c->tmap_keys[i];
     if (k.base == base && k.rows == rows && k.cols == cols && k.box_rows == box_rows) return (int)i;
   }
-  if (c->tmaps_host.size() >= c->tmaps_cap) return -1;
+  if (c->tmaps_host.size() >= c->tmaps_cap || c->capturing) return -1;   // descriptors are made before capture
   const int idx = add_tmap_bf16(c, base, rows, cols, box_rows);
   if (idx < 0) return -1;
   c->tmap_keys.push_back({base, rows, cols, box_rows});
@@ -374,7 +382,7 @@ PartView gemm(fm_ctx* c, const bf16* W, size_t w_rows_alloc, int w_row0, const b
 template <int MODE>
 void fold(fm_ctx* c, const PartView& pv, void* out, int ldo, int M, int R) {
   if (R <= 0) return;
-  const int gy = (M + 1023) / 1024;
+  const int gy = (M + 255) / 256;
   LAUNCH(c, fold_kernel<MODE>, dim3(R, gy), 256, 0, pv, out, ldo, M);
 }
 
@@ -426,22 +434,22 @@ void run_stack(fm_ctx* c, int s, float* x, size_t x_rows_alloc, float* stash_rin
   (void)x_rows_alloc;
   for (int l = 0; l < nl; ++l) {
     const LayerDev& L = c->layers[s][l];
-    LAUNCH(c, resid_norm_kernel, rows, 256, d * sizeof(float), x, pend, pend_mode, L.g1, c->a_norm, d, dm.eps);
+    LAUNCH(c, resid_norm_kernel, rows, (d >= 1024 ? 1024 : 256), d * sizeof(float), x, pend, pend_mode, L.g1, c->a_norm, d, dm.eps);
     if (stash_ring != nullptr && l == nl - 1)
       LAUNCH(c, ring_store_kernel, rows, 128, 0, dm, c->st, c->batch, level, x, stash_ring, d);
     PartView pq = gemm(c, L.Wqkv, pad128(qkvw), 0, c->a_norm, Rc_alloc, 0, qkvw, d, rows, na);
-    LAUNCH(c, rope_append_kernel, rows, 128, dm.dh * sizeof(float), dm, c->st, c->batch, level, pq, c->inv_freq,
-           c->qbuf, L.K, L.V);
+    LAUNCH(c, rope_append_kernel, dim3(rows, (dm.H + 2 * dm.Hkv + 1) / 2), dm.dh, 0, dm, c->st, c->batch, level, pq,
+           c->rope_tab, c->qbuf, L.K, L.V);
     attention(c, level, rows, L);
     PartView po = gemm(c, L.Wo, pad128(d), 0, c->a_attn, Rc_alloc, 0, d, hd, rows, na);
-    LAUNCH(c, resid_norm_kernel, rows, 256, d * sizeof(float), x, po, 1, L.g2, c->a_norm, d, dm.eps);
+    LAUNCH(c, resid_norm_kernel, rows, (d >= 1024 ? 1024 : 256), d * sizeof(float), x, po, 1, L.g2, c->a_norm, d, dm.eps);
     PartView p1 = gemm(c, L.W1, pad128(dm.dff), 0, c->a_norm, Rc_alloc, 0, dm.dff, d, rows, na);
     fold<FOLD_GELU_BF16>(c, p1, c->a_ff, dm.dff, dm.dff, rows);
     pend = gemm(c, L.W2, pad128(d), 0, c->a_ff, Rc_alloc, 0, d, dm.dff, rows, na);
     pend_mode = 1;
   }
   // fold the last FFN output into the residual stream (no norm)
-  LAUNCH(c, resid_norm_kernel, rows, 256, d * sizeof(float), x, pend, pend_mode, (const float*)nullptr, (bf16*)nullptr, d,
+  LAUNCH(c, resid_norm_kernel, rows, (d >= 1024 ? 1024 : 256), d * sizeof(float), x, pend, pend_mode, (const float*)nullptr, (bf16*)nullptr, d,
          dm.eps);
 }
 
@@ -534,6 +542,62 @@ __global__ void set_limits_kernel(Dims dm, SeqState st, int batch, const int* __
   const int cap = dm.max_tokens - dm.D - 2;
   const long long want = (long long)st.plen[b] + 9ll * max_faces[b];
   st.t_end[b] = want < cap ? (int)want : cap;
+}
+
+// one decode pass of fm_generate
+void step_body(fm_ctx* c) {
+  const Dims& dm = c->dm;
+  draft(c, nullptr, nullptr);
+  LAUNCH(c, teacher_edit_kernel, c->batch, 32, 0, dm, c->st, c->batch, (const GenOut*)c->gen_dev);
+  forward(c, nullptr);
+  LAUNCH(c, accept_kernel, (c->batch * 32 + 127) / 128, 128, 0, dm, c->st, c->batch, (const int*)nullptr,
+         (const int*)nullptr, (int*)nullptr, (int*)nullptr, (int*)nullptr, (const GenOut*)c->gen_dev);
+  LAUNCH(c, row_count_kernel, 1, 32, 0, dm, c->st, c->batch);
+  LAUNCH(c, step_end_kernel, 1, 32, 0, c->st, (const GenOut*)c->gen_dev);
+}
+
+void drop_graph(fm_ctx* c) {
+  if (c->graph_exec != nullptr) cudaGraphExecDestroy(c->graph_exec);
+  if (c->graph != nullptr) cudaGraphDestroy(c->graph);
+  c->graph_exec = nullptr;
+  c->graph = nullptr;
+}
+
+// Capture the pass once per batch size.  All state the kernels read lives in device memory, so the
+// same graph serves every pass.  Streams that cannot be captured (the legacy default stream) fall
+// back to plain launches of the same kernels.
+void ensure_graph(fm_ctx* c) {
+  if (c->graph_unavailable || (c->graph_exec != nullptr && c->graph_batch == c->batch)) return;
+  drop_graph(c);
+  draft(c, nullptr, nullptr);                      // makes the draft path's TMA descriptors exist
+  cudaStreamSynchronize(c->stream);
+  if (cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+    cudaGetLastError();
+    c->graph_unavailable = true;
+    return;
+  }
+  const int64_t l0 = c->launches;
+  c->capturing = true;
+  step_body(c);
+  c->capturing = false;
+  c->graph_launches = c->launches - l0;
+  c->launches = l0;
+  cudaGraph_t g = nullptr;
+  if (cudaStreamEndCapture(c->stream, &g) != cudaSuccess || g == nullptr || c->launch_error != FM_OK) {
+    cudaGetLastError();
+    if (g != nullptr) cudaGraphDestroy(g);
+    c->graph_unavailable = true;
+    c->launch_error = FM_OK;
+    return;
+  }
+  c->graph = g;
+  if (cudaGraphInstantiate(&c->graph_exec, g, 0) != cudaSuccess) {
+    cudaGetLastError();
+    drop_graph(c);
+    c->graph_unavailable = true;
+    return;
+  }
+  c->graph_batch = c->batch;
 }
 
 }  // namespace
@@ -639,6 +703,11 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
   for (int i = 0; i < dm.dh / 2; ++i)
     freq[i] = dm.theta != 0.f ? pow((double)dm.theta, -2.0 * (double)i / (double)dm.dh) : 0.0;
   TRYCUDA(cudaMemcpy(c->inv_freq, freq.data(), freq.size() * sizeof(double), cudaMemcpyHostToDevice));
+  {
+    const size_t n = (size_t)(dm.max_tokens + 1) * (dm.dh / 2);
+    rope_table_kernel<<<(unsigned)((n + 255) / 256), 256, 0, c->stream>>>(c->rope_tab, c->inv_freq, dm.max_tokens + 1, dm.dh / 2);
+    TRYCUDA(cudaGetLastError());
+  }
   TRYCUDA(cudaHostAlloc(reinterpret_cast<void**>(&c->host_done), 64, cudaHostAllocMapped));
   *c->host_done = 0;
   TRYCUDA(cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->host_done_dev), c->host_done, 0));
@@ -679,6 +748,7 @@ int fm_destroy(fm_ctx* c) {
   if (c == nullptr) return FM_ERR_INVALID_ARG;
   cudaStreamSynchronize(c->stream);
   for (auto& e : c->prof_ev) cudaEventDestroy(e);
+  drop_graph(c);
   if (c->host_done != nullptr) cudaFreeHost(c->host_done);
   delete c;
   return FM_OK;
@@ -808,6 +878,8 @@ int fm_generate(fm_ctx* c, int32_t max_faces, int32_t* out_tok, int32_t out_stri
   if (out_len != nullptr && c->gen_fresh) CUDA_OK(cudaMemsetAsync(out_len, 0, c->batch * sizeof(int), c->stream));
   c->gen_fresh = false;
   CUDA_OK(cudaStreamSynchronize(c->stream));       // `g` lives on this stack frame
+  if (!c->prof_on) ensure_graph(c);
+  const bool use_graph = !c->prof_on && c->graph_exec != nullptr;
   cudaEvent_t e0, e1;
   CUDA_OK(cudaEventCreate(&e0));
   CUDA_OK(cudaEventCreate(&e1));
@@ -820,13 +892,12 @@ int fm_generate(fm_ctx* c, int32_t max_faces, int32_t* out_tok, int32_t out_stri
   while (!finished && steps < bound) {
     const long long poll = max_steps > 0 ? bound : 8;
     for (long long i = 0; i < poll; ++i) {
-      draft(c, nullptr, nullptr);
-      if (teacher != nullptr) LAUNCH(c, teacher_edit_kernel, c->batch, 32, 0, dm, c->st, c->batch, c->gen_dev);
-      forward(c, nullptr);
-      LAUNCH(c, accept_kernel, (c->batch * 32 + 127) / 128, 128, 0, dm, c->st, c->batch, (const int*)nullptr,
-             (const int*)nullptr, (int*)nullptr, (int*)nullptr, (int*)nullptr, (const GenOut*)c->gen_dev);
-      LAUNCH(c, row_count_kernel, 1, 32, 0, dm, c->st, c->batch);
-      LAUNCH(c, step_end_kernel, 1, 32, 0, c->st, (const GenOut*)c->gen_dev);
+      if (use_graph) {
+        CUDA_OK(cudaGraphLaunch(c->graph_exec, c->stream));
+        c->launches += c->graph_launches;
+      } else {
+        step_body(c);
+      }
       ++steps;
     }
     CUDA_OK(cudaStreamSynchronize(c->stream));

@@ -10,10 +10,23 @@ struct PartView {
   int ldm;                // elements between rows
 };
 
+// loads are issued eight at a time (independent), the additions stay in split order
 __device__ inline float part_sum(const PartView& pv, int row, int m) {
   const float* p = pv.part + (size_t)row * pv.ldm + m;
   float v = 0.f;
-  for (int z = 0; z < pv.nsplit; ++z) v += __ldcg(p + (size_t)z * pv.split_stride);
+  int z = 0;
+  for (; z + 8 <= pv.nsplit; z += 8) {
+    float t[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) t[u] = __ldcg(p + (size_t)(z + u) * pv.split_stride);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v += t[u];
+  }
+  float t[8];
+#pragma unroll
+  for (int u = 0; u < 8; ++u) t[u] = (z + u < pv.nsplit) ? __ldcg(p + (size_t)(z + u) * pv.split_stride) : 0.f;
+#pragma unroll
+  for (int u = 0; u < 8; ++u) if (z + u < pv.nsplit) v += t[u];
   return v;
 }
 
@@ -21,7 +34,7 @@ __device__ inline float gelu_erf(float x) { return 0.5f * x * (1.f + erff(x * 0.
 
 enum FoldMode { FOLD_F32 = 0, FOLD_BF16 = 1, FOLD_GELU_BF16 = 2 };
 
-// out[row][m] = f(sum of partials); grid (rows, ceil(M / (4*256))), block 256
+// out[row][m] = f(sum of partials); grid (rows, ceil(M / 256)), block 256
 template <int MODE>
 __global__ void fold_kernel(PartView pv, void* __restrict__ out, int ldo, int M) {
   const int row = blockIdx.x;

@@ -74,12 +74,23 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
 }
 
 // ------------------------------------------------------------------------------------------
-// RoPE on q and k (rotate-half pairs (i, i+dh/2), angle = pos * theta^(-2i/dh), evaluated in
-// double), then append k, v to the level's cache at slot P + pos % cap.
+// RoPE on q and k (rotate-half pairs (i, i+dh/2), angle = pos * theta^(-2i/dh); cos/sin come from
+// a table evaluated in double precision when the context is created), then append k, v to the
+// level's cache at slot P + pos % cap.
 // qkv: split-K partials of [rows, (H+2Hkv)*dh]; q_out: fp32 [rows, H*dh]; caches: bf16 [B, Hkv, slots, dh].
+// grid (rows, (H + 2*Hkv) / 2): each CTA of dh threads handles two heads of one row.
 // ------------------------------------------------------------------------------------------
+__global__ void rope_table_kernel(float2* __restrict__ tab, const double* __restrict__ inv_freq, int n_pos, int half) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (size_t)n_pos * half) return;
+  const int pos = (int)(i / half), k = (int)(i - (size_t)pos * half);
+  double s, c;
+  sincos((double)pos * inv_freq[k], &s, &c);
+  tab[i] = make_float2((float)c, (float)s);
+}
+
 __global__ void rope_append_kernel(Dims dm, SeqState st, int batch, int level, PartView qkv,
-                                   const double* __restrict__ inv_freq, float* __restrict__ q_out,
+                                   const float2* __restrict__ rope_tab, float* __restrict__ q_out,
                                    bf16* __restrict__ Kc, bf16* __restrict__ Vc) {
   const int row = blockIdx.x;
   int b, p;
@@ -87,36 +98,26 @@ __global__ void rope_append_kernel(Dims dm, SeqState st, int batch, int level, P
   const int H = dm.H, Hkv = dm.Hkv, dh = dm.dh, half = dh / 2;
   const int slots = dm.P + dm.cap[level];
   const int slot = dm.P + (p % dm.cap[level]);
-  extern __shared__ float cs[];                     // cos[half], sin[half]
-  for (int i = threadIdx.x; i < half; i += blockDim.x) {
-    double s = 0.0, c = 1.0;
-    if (dm.theta != 0.f) sincos((double)p * inv_freq[i], &s, &c);
-    cs[i] = (float)c;
-    cs[half + i] = (float)s;
-  }
-  __syncthreads();
-  // q and k heads: one thread per rotation pair
-  const int pairs = (H + Hkv) * half;
-  for (int t = threadIdx.x; t < pairs; t += blockDim.x) {
-    const int head = t / half, i = t - head * half;
-    const float x1 = part_sum(qkv, row, head * dh + i), x2 = part_sum(qkv, row, head * dh + half + i);
-    const float c = cs[i], s = cs[half + i];
+  const int head = blockIdx.y * 2 + threadIdx.x / half;     // 0..H-1 q, H..H+Hkv-1 k, then v
+  const int i = threadIdx.x % half;
+  if (head >= H + 2 * Hkv) return;
+  const float x1 = part_sum(qkv, row, head * dh + i), x2 = part_sum(qkv, row, head * dh + half + i);
+  if (head < H + Hkv) {
+    float c = 1.f, s = 0.f;
+    if (dm.theta != 0.f) { const float2 cs = rope_tab[(size_t)p * half + i]; c = cs.x; s = cs.y; }
     const float y1 = x1 * c - x2 * s, y2 = x2 * c + x1 * s;
     if (head < H) {
       q_out[(size_t)row * H * dh + head * dh + i] = valid ? y1 : 0.f;
       q_out[(size_t)row * H * dh + head * dh + half + i] = valid ? y2 : 0.f;
     } else if (valid) {
-      const int hk = head - H;
-      bf16* dst = Kc + (((size_t)b * Hkv + hk) * slots + slot) * dh;
+      bf16* dst = Kc + (((size_t)b * Hkv + (head - H)) * slots + slot) * dh;
       dst[i] = __float2bfloat16(y1);
       dst[half + i] = __float2bfloat16(y2);
     }
-  }
-  if (valid) {
-    for (int t = threadIdx.x; t < Hkv * dh; t += blockDim.x) {
-      const int hk = t / dh, i = t - hk * dh;
-      Vc[(((size_t)b * Hkv + hk) * slots + slot) * dh + i] = __float2bfloat16(part_sum(qkv, row, (H + Hkv) * dh + t));
-    }
+  } else if (valid) {
+    bf16* dst = Vc + (((size_t)b * Hkv + (head - H - Hkv)) * slots + slot) * dh;
+    dst[i] = __float2bfloat16(x1);
+    dst[half + i] = __float2bfloat16(x2);
   }
 }
 
