@@ -11,11 +11,11 @@
 #include <string.h>
 
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "fm_attention.cuh"
 #include "fm_common.cuh"
-#include "fm_gemm.cuh"
 #include "fm_gemm_tc.cuh"
 #include "fm_kernels.cuh"
 
@@ -52,8 +52,8 @@ struct fm_ctx {
   // state
   SeqState st;
   // activations
-  float *xc, *xv, *xf, *qbuf, *logits, *tmp3d;
-  bf16 *a_norm, *a_cat, *a_attn, *a_ff;
+  float *xc, *xv, *xf, *logits, *tmp3d;
+  bf16 *qbuf, *a_norm, *a_cat, *a_attn, *a_ff;
   float *hc_ring, *hv_ring, *trif_ring, *triv_ring, *zc, *zv, *zf;
   // draft
   bf16 *dh_a, *up_in_v, *up_in_f, *feat_n;
@@ -67,9 +67,10 @@ struct fm_ctx {
   struct TmapKey { const void* base; uint64_t rows, cols; uint32_t box_rows; };
   std::vector<TmapKey> tmap_keys;
   size_t tmaps_cap, tmaps_uploaded;
-  // split-K partial tiles of the GEMM in flight
-  float* gpart;
-  size_t gpart_floats;
+  // per-tile sums of squares of the residual rows (RMSNorm statistics handed between GEMMs)
+  float* ssq;
+  int ssq_tiles, ssq_ld;
+  bool use_pdl;
   // prefill temporaries
   bf16* pre_a;
   float* pre_o;
@@ -86,6 +87,7 @@ struct fm_ctx {
   size_t prof_used;
   double prof_ms[3], prof_bytes[3];
   long long prof_n[3];
+  int split_target;     // CTAs a GEMM launch aims for (M tiles x K splits)
   int launch_error;     // first error met while enqueueing (capacity, descriptor creation)
   // one decode pass (draft, teacher edit, verify, accept) captured as a CUDA graph
   cudaGraph_t graph;
@@ -190,7 +192,9 @@ void carve(fm_ctx* c, Carver& cv) {
   // activations (row counts padded to 16 so that later tiles never run off the end)
   const size_t Rc = align_up(B * dm.R1, 16), Rv = align_up(B * dm.mv, 16), Rf = align_up(B * dm.mf, 16);
   c->xc = cv.take<float>(Rc * d); c->xv = cv.take<float>(Rv * d); c->xf = cv.take<float>(Rf * d);
-  c->qbuf = cv.take<float>(Rc * hd);
+  c->qbuf = cv.take<bf16>(Rc * hd);
+  c->ssq_tiles = (int)((d + 127) / 128); c->ssq_ld = (int)Rc;
+  c->ssq = cv.take<float>((size_t)c->ssq_tiles * Rc);
   c->logits = cv.take<float>(Rc * dm.Vpad); c->tmp3d = cv.take<float>(Rv * 3 * d);
   c->a_norm = cv.take<bf16>(Rc * d); c->a_cat = cv.take<bf16>(Rv * 3 * d);
   c->a_attn = cv.take<bf16>(Rc * hd); c->a_ff = cv.take<bf16>(Rc * dm.dff);
@@ -220,15 +224,6 @@ void carve(fm_ctx* c, Carver& cv) {
   for (int s = 0; s < 5; ++s) n_layers += c->cfg.layers[s];
   c->tmaps_cap = (size_t)6 * n_layers + 128;
   c->tmaps = cv.take<CUtensorMap>(c->tmaps_cap);
-  {
-    // per row at most ~2 * 148 * 128 partial floats (split * padded M), see gemm()
-    size_t rows_max = align_up(B * dm.R1, 16);
-    const size_t nf_rows = align_up((8 + 9 * (size_t)dm.Ef) * B, 16);
-    rows_max = rows_max > nf_rows ? rows_max : nf_rows;
-    rows_max = rows_max > 256 ? rows_max : 256;
-    c->gpart_floats = rows_max * 40960;
-    c->gpart = cv.take<float>(c->gpart_floats);
-  }
   // prefill temporaries
   c->pre_a = cv.take<bf16>((size_t)PREFILL_CHUNK * d);
   c->pre_o = cv.take<float>((size_t)PREFILL_CHUNK * 2 * dm.Hkv * dm.dh);
@@ -346,49 +341,75 @@ int tmap_for(fm_ctx* c, const void* base, uint64_t rows, uint64_t cols, uint32_t
   return idx;
 }
 
-// part[z][n][m] = partial of W[w_row0 + m, :] . A[a_row0 + n, :] over K range z (see fm_gemm_tc.cuh).
-// W: [w_rows_alloc, K] bf16 (rows padded to 128), A: [a_rows_alloc, K] bf16 (rows padded to 16).
-// Returns the view the consumer kernel needs.  The K split depends on (M, K) only.
-PartView gemm(fm_ctx* c, const bf16* W, size_t w_rows_alloc, int w_row0, const bf16* A, size_t a_rows_alloc, int a_row0,
-              int M, int K, int R, const int* n_active) {
-  PartView pv{c->gpart, 0, 0, 0};
-  if (R <= 0) return pv;
+// Launch with the programmatic-dependent-launch attribute: the kernel may start while its
+// predecessor is still running and must execute griddepcontrol.wait before it touches anything a
+// predecessor produces (and before it exits).  Kernels launched through LAUNCH are full barriers.
+// cluster_y > 1 makes the CTAs along the grid's y extent one thread-block cluster.
+template <typename... KArgs, typename... CArgs>
+void launch_pdl(fm_ctx* c, int cluster_y, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, CArgs&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = c->stream;
+  cudaLaunchAttribute at[2];
+  int n = 0;
+  if (c->use_pdl) {
+    at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  if (cluster_y > 1) {
+    at[n].id = cudaLaunchAttributeClusterDimension;
+    at[n].val.clusterDim.x = 1;
+    at[n].val.clusterDim.y = (unsigned)cluster_y;
+    at[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = at;
+  cfg.numAttrs = n;
+  if (cudaLaunchKernelEx(&cfg, kern, std::forward<CArgs>(args)...) != cudaSuccess && c->launch_error == FM_OK)
+    c->launch_error = FM_ERR_CUDA;
+  c->launches++;
+}
+
+tc::Epi epi_plain(void* out, int ldo) {
+  tc::Epi e{};
+  e.out = out;
+  e.ldo = ldo;
+  return e;
+}
+
+// y[n][m] = W[w_row0 + m, :] . A[a_row0 + n, :], n < R, m < M, finished by the epilogue `mode`
+// (see fm_gemm_tc.cuh).  W: [w_rows_alloc, K] bf16 (rows padded to 128), A: [a_rows_alloc, K] bf16
+// (rows padded to 16).  The K split (= cluster size) depends on (M, K) only.
+void gemm(fm_ctx* c, const bf16* W, size_t w_rows_alloc, int w_row0, const bf16* A, size_t a_rows_alloc, int a_row0,
+          int M, int K, int R, const int* n_active, int mode, tc::Epi e) {
+  if (R <= 0) return;
   const int tiles = (M + tc::BM - 1) / tc::BM, slabs = K / tc::BK;
-  int split = (148 + tiles / 2) / tiles;
-  split = split < 1 ? 1 : split;
-  split = split > slabs ? slabs : split;
-  split = split > 32 ? 32 : split;
-  const int ldm = tiles * tc::BM;
+  int split = 1;
+  while (split * 2 <= tc::MAX_SPLIT && split * 2 <= slabs && tiles * split * 2 <= c->split_target) split *= 2;
   const int Rpad = round_up(R, 16);
-  pv.nsplit = split;
-  pv.ldm = ldm;
-  pv.split_stride = (long long)Rpad * ldm;
-  if ((size_t)split * Rpad * ldm > c->gpart_floats) { c->launch_error = FM_ERR_CAPACITY; return pv; }
   const int tW = tmap_for(c, W, w_rows_alloc, K, tc::BM);
   const long pi = prof_open(c, PROF_GEMM, 2.0 * M * K);            // algorithmic bytes: the weight matrix once
   for (int n0 = 0; n0 < Rpad; n0 += 256) {                         // N tiles of at most 256 rows
     const int N = Rpad - n0 < 256 ? Rpad - n0 : 256;
     const int tA = tmap_for(c, A, a_rows_alloc, K, N);
     if (tW < 0 || tA < 0) { c->launch_error = FM_ERR_CUDA; break; }
-    tc::Args g{c->tmaps + tW, c->tmaps + tA, c->gpart + (size_t)n0 * ldm, M, K, N, (R - n0 < N ? R - n0 : N), ldm,
-               pv.split_stride, split, w_row0, a_row0 + n0, n_active, c->st.status};
+    tc::Args g{c->tmaps + tW, c->tmaps + tA, M, K, N, (R - n0 < N ? R - n0 : N), split, w_row0, a_row0 + n0, n_active,
+               c->st.status};
+    e.row0 = n0;
     const int smem = tc::smem_bytes(N);
-    LAUNCH(c, tc::gemm_tc_kernel, dim3(tiles, split), 128, smem, g);
+    const dim3 grid(tiles, split);
+    switch (mode) {
+      case tc::EPI_F32: launch_pdl(c, split, tc::gemm_tc_kernel<tc::EPI_F32>, grid, 128, smem, g, e); break;
+      case tc::EPI_BF16: launch_pdl(c, split, tc::gemm_tc_kernel<tc::EPI_BF16>, grid, 128, smem, g, e); break;
+      case tc::EPI_GELU: launch_pdl(c, split, tc::gemm_tc_kernel<tc::EPI_GELU>, grid, 128, smem, g, e); break;
+      case tc::EPI_RESID: launch_pdl(c, split, tc::gemm_tc_kernel<tc::EPI_RESID>, grid, 128, smem, g, e); break;
+      default: launch_pdl(c, split, tc::gemm_tc_kernel<tc::EPI_QKV>, grid, 128, smem, g, e); break;
+    }
   }
   prof_close(c, pi);
-  return pv;
-}
-
-template <int MODE>
-void fold(fm_ctx* c, const PartView& pv, void* out, int ldo, int M, int R) {
-  if (R <= 0) return;
-  const int gy = (M + 255) / 256;
-  LAUNCH(c, fold_kernel<MODE>, dim3(R, gy), 256, 0, pv, out, ldo, M);
-}
-
-__global__ void to_bf16_kernel(const float* __restrict__ x, bf16* __restrict__ out, size_t n) {
-  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) out[i] = __float2bfloat16(x[i]);
 }
 
 // rows fed at each level in this pass (n_active[level]); n_active[3] = unfinished sequences
@@ -407,23 +428,24 @@ __global__ void row_count_kernel(Dims dm, SeqState st, int batch) {
   st.n_active[0] = cnt[0]; st.n_active[1] = cnt[1]; st.n_active[2] = cnt[2]; st.n_active[3] = act;
 }
 
-void attention(fm_ctx* c, int level, int rows, const LayerDev& L) {
+void attention(fm_ctx* c, int level, const LayerDev& L) {
   const Dims& dm = c->dm;
   AttnArgs a{dm, c->st, c->batch, level, c->qbuf, c->tmaps + L.tmK, c->tmaps + L.tmV, c->attn_part, c->attn_ticket,
              c->a_attn, c->attn_max_chunks[level], c->attn_mrows[level]};
   dim3 grid(c->attn_max_chunks[level], dm.Hkv, c->batch);
   const long pi = prof_open(c, PROF_ATTN, 0.0);
-  if (dm.dh == 64) LAUNCH(c, (attn_split_kernel<64, 256>), grid, 128, (AttnSmem<64, 256>::BYTES), a);
-  else LAUNCH(c, (attn_split_kernel<128, 128>), grid, 128, (AttnSmem<128, 128>::BYTES), a);
+  if (dm.dh == 64) launch_pdl(c, 1, attn_split_kernel<64, 256>, grid, 128, AttnSmem<64, 256>::BYTES, a);
+  else launch_pdl(c, 1, attn_split_kernel<128, 128>, grid, 128, AttnSmem<128, 128>::BYTES, a);
   prof_close(c, pi);
-  (void)rows;
 }
 
 inline size_t pad128(size_t v) { return align_up(v, 128); }
 
-// one stack of pre-norm blocks on the rows of its level (a2/a4/a6/a8/a10).  `pend` holds GEMM
-// partials that still have to be folded into x (mode 1: add, 2: store) by the first norm kernel.
-void run_stack(fm_ctx* c, int s, float* x, size_t x_rows_alloc, float* stash_ring, PartView pend, int pend_mode) {
+// One stack of pre-norm blocks on the rows of its level (a2/a4/a6/a8/a10): five launches per
+// layer.  On entry c->a_norm holds bf16(x * g1 of the first layer) and c->ssq the rows' sums of
+// squares; on exit, if `want_a`, c->a_norm holds bf16(x * next_gain) (gain 1 when null) and c->ssq
+// the sums of squares of the stack's output rows.
+void run_stack(fm_ctx* c, int s, float* x, float* stash_ring, const float* next_gain, bool want_a) {
   const Dims& dm = c->dm;
   const int level = STACK_LEVEL[s];
   const int rows = c->batch * fm_rows_per_seq(dm, level);
@@ -431,26 +453,30 @@ void run_stack(fm_ctx* c, int s, float* x, size_t x_rows_alloc, float* stash_rin
   const size_t Rc_alloc = align_up((size_t)dm.max_batch * dm.R1, 16);
   const int* na = c->st.n_active + level;
   const int nl = (int)c->layers[s].size();
-  (void)x_rows_alloc;
   for (int l = 0; l < nl; ++l) {
     const LayerDev& L = c->layers[s][l];
-    LAUNCH(c, resid_norm_kernel, rows, (d >= 1024 ? 1024 : 256), d * sizeof(float), x, pend, pend_mode, L.g1, c->a_norm, d, dm.eps);
     if (stash_ring != nullptr && l == nl - 1)
-      LAUNCH(c, ring_store_kernel, rows, 128, 0, dm, c->st, c->batch, level, x, stash_ring, d);
-    PartView pq = gemm(c, L.Wqkv, pad128(qkvw), 0, c->a_norm, Rc_alloc, 0, qkvw, d, rows, na);
-    LAUNCH(c, rope_append_kernel, dim3(rows, (dm.H + 2 * dm.Hkv + 1) / 2), dm.dh, 0, dm, c->st, c->batch, level, pq,
-           c->rope_tab, c->qbuf, L.K, L.V);
-    attention(c, level, rows, L);
-    PartView po = gemm(c, L.Wo, pad128(d), 0, c->a_attn, Rc_alloc, 0, d, hd, rows, na);
-    LAUNCH(c, resid_norm_kernel, rows, (d >= 1024 ? 1024 : 256), d * sizeof(float), x, po, 1, L.g2, c->a_norm, d, dm.eps);
-    PartView p1 = gemm(c, L.W1, pad128(dm.dff), 0, c->a_norm, Rc_alloc, 0, dm.dff, d, rows, na);
-    fold<FOLD_GELU_BF16>(c, p1, c->a_ff, dm.dff, dm.dff, rows);
-    pend = gemm(c, L.W2, pad128(d), 0, c->a_ff, Rc_alloc, 0, d, dm.dff, rows, na);
-    pend_mode = 1;
+      launch_pdl(c, 1, ring_store_kernel, rows, 128, 0, dm, c->st, c->batch, level, (const float*)x, stash_ring, d);
+    tc::Epi eq{};
+    eq.ssq_in = c->ssq; eq.ssq_tiles = c->ssq_tiles; eq.ld_ssq = c->ssq_ld; eq.inv_d_in = 1.f / d; eq.eps = dm.eps;
+    eq.dm = dm; eq.st = c->st; eq.batch = c->batch; eq.level = level; eq.rope_tab = c->rope_tab;
+    eq.q_out = c->qbuf; eq.Kc = L.K; eq.Vc = L.V;
+    eq.qscale = (float)(1.4426950408889634 / sqrt((double)dm.dh));   // 1/sqrt(dh) * log2(e)
+    gemm(c, L.Wqkv, pad128(qkvw), 0, c->a_norm, Rc_alloc, 0, qkvw, d, rows, na, tc::EPI_QKV, eq);
+    attention(c, level, L);
+    tc::Epi eo{};
+    eo.x = x; eo.ldx = d; eo.add = 1; eo.gain = L.g2; eo.a_out = c->a_norm; eo.lda = d;
+    eo.ssq_out = c->ssq; eo.ld_ssq_out = c->ssq_ld;
+    gemm(c, L.Wo, pad128(d), 0, c->a_attn, Rc_alloc, 0, d, hd, rows, na, tc::EPI_RESID, eo);
+    tc::Epi e1 = epi_plain(c->a_ff, dm.dff);
+    e1.ssq_in = c->ssq; e1.ssq_tiles = c->ssq_tiles; e1.ld_ssq = c->ssq_ld; e1.inv_d_in = 1.f / d; e1.eps = dm.eps;
+    gemm(c, L.W1, pad128(dm.dff), 0, c->a_norm, Rc_alloc, 0, dm.dff, d, rows, na, tc::EPI_GELU, e1);
+    tc::Epi e2 = eo;
+    const bool last = l == nl - 1;
+    e2.gain = last ? next_gain : c->layers[s][l + 1].g1;
+    if (last && !want_a) { e2.a_out = nullptr; e2.ssq_out = nullptr; }
+    gemm(c, L.W2, pad128(d), 0, c->a_ff, Rc_alloc, 0, d, dm.dff, rows, na, tc::EPI_RESID, e2);
   }
-  // fold the last FFN output into the residual stream (no norm)
-  LAUNCH(c, resid_norm_kernel, rows, (d >= 1024 ? 1024 : 256), d * sizeof(float), x, pend, pend_mode, (const float*)nullptr, (bf16*)nullptr, d,
-         dm.eps);
 }
 
 // the verify forward pass over st.cand / st.nrow (a1..a11)
@@ -460,34 +486,37 @@ void forward(fm_ctx* c, float* logits_out) {
   const int Rc = B * dm.R1, Rv = B * dm.mv, Rf = B * dm.mf;
   const size_t Rc_alloc = align_up((size_t)dm.max_batch * dm.R1, 16), Rv_alloc = align_up((size_t)dm.max_batch * dm.mv, 16);
   const int* na = c->st.n_active;
-  const PartView none{nullptr, 0, 0, 0};
+  // The two launches that open a pass are full barriers: the per-pass state (rows, lengths,
+  // candidates) is final before any later kernel's prologue can run.
   LAUNCH(c, row_count_kernel, 1, 32, 0, dm, c->st, B);
-  LAUNCH(c, embed_kernel, Rc, 128, 0, dm, c->st, B, c->E, c->xc);
-  run_stack(c, 0, c->xc, Rc_alloc, nullptr, none, 0);
-  LAUNCH(c, ring_store_kernel, Rc, 128, 0, dm, c->st, B, 0, c->xc, c->hc_ring, d);
-  LAUNCH(c, shorten_gather_kernel, Rv, 128, 0, dm, c->st, B, 1, c->hc_ring, c->a_cat);
-  PartView pv = gemm(c, c->S_cv, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rv, na + 1);
-  run_stack(c, 1, c->xv, Rv_alloc, nullptr, pv, 2);
-  LAUNCH(c, ring_store_kernel, Rv, 128, 0, dm, c->st, B, 1, c->xv, c->hv_ring, d);
-  LAUNCH(c, shorten_gather_kernel, Rf, 128, 0, dm, c->st, B, 2, c->hv_ring, c->a_cat);
-  pv = gemm(c, c->S_vf, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rf, na + 2);
-  run_stack(c, 2, c->xf, 0, c->zf, pv, 2);
-  LAUNCH(c, to_bf16_kernel, (Rf * d + 255) / 256, 256, 0, c->xf, c->a_norm, (size_t)Rf * d);
-  pv = gemm(c, c->U_fv, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rf, na + 2);
-  fold<FOLD_F32>(c, pv, c->tmp3d, 3 * d, 3 * d, Rf);
-  LAUNCH(c, ring_store_kernel, Rf, 128, 0, dm, c->st, B, 2, c->tmp3d, c->trif_ring, 3 * d);
-  LAUNCH(c, upsample_add_kernel, Rv, 128, 0, dm, c->st, B, 1, c->hv_ring, c->trif_ring, c->xv);
-  run_stack(c, 3, c->xv, Rv_alloc, c->zv, none, 0);
-  LAUNCH(c, to_bf16_kernel, (Rv * d + 255) / 256, 256, 0, c->xv, c->a_norm, (size_t)Rv * d);
-  pv = gemm(c, c->U_vc, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rv, na + 1);
-  fold<FOLD_F32>(c, pv, c->tmp3d, 3 * d, 3 * d, Rv);
-  LAUNCH(c, ring_store_kernel, Rv, 128, 0, dm, c->st, B, 1, c->tmp3d, c->triv_ring, 3 * d);
-  LAUNCH(c, upsample_add_kernel, Rc, 128, 0, dm, c->st, B, 0, c->hc_ring, c->triv_ring, c->xc);
-  run_stack(c, 4, c->xc, Rc_alloc, c->zc, none, 0);
-  LAUNCH(c, rmsnorm_kernel, Rc, 256, 0, c->xc, c->g_out, c->a_norm, d, dm.eps);
-  pv = gemm(c, c->W_out, dm.Vpad, 0, c->a_norm, Rc_alloc, 0, dm.V, d, Rc, na);
-  fold<FOLD_F32>(c, pv, c->logits, dm.Vpad, dm.V, Rc);
-  LAUNCH(c, verify_top2_kernel, Rc, 256, 0, dm, c->st, B, c->logits, logits_out);
+  LAUNCH(c, embed_kernel, Rc, 128, 0, dm, c->st, B, c->E, c->xc, c->layers[0][0].g1, c->a_norm, c->ssq, c->ssq_tiles, c->ssq_ld);
+  run_stack(c, 0, c->xc, nullptr, nullptr, false);
+  launch_pdl(c, 1, ring_store_kernel, Rc, 128, 0, dm, c->st, B, 0, (const float*)c->xc, c->hc_ring, d);
+  launch_pdl(c, 1, shorten_gather_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->hc_ring, c->a_cat);
+  tc::Epi es{};
+  es.x = c->xv; es.ldx = d; es.add = 0; es.gain = c->layers[1][0].g1; es.a_out = c->a_norm; es.lda = d;
+  es.ssq_out = c->ssq; es.ld_ssq_out = c->ssq_ld;
+  gemm(c, c->S_cv, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rv, na + 1, tc::EPI_RESID, es);
+  run_stack(c, 1, c->xv, nullptr, nullptr, false);
+  launch_pdl(c, 1, ring_store_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->xv, c->hv_ring, d);
+  launch_pdl(c, 1, shorten_gather_kernel, Rf, 128, 0, dm, c->st, B, 2, (const float*)c->hv_ring, c->a_cat);
+  es.x = c->xf; es.gain = c->layers[2][0].g1;
+  gemm(c, c->S_vf, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rf, na + 2, tc::EPI_RESID, es);
+  run_stack(c, 2, c->xf, c->zf, nullptr, true);                    // leaves bf16(xf) in a_norm
+  gemm(c, c->U_fv, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rf, na + 2, tc::EPI_F32, epi_plain(c->tmp3d, 3 * d));
+  launch_pdl(c, 1, ring_store_kernel, Rf, 128, 0, dm, c->st, B, 2, (const float*)c->tmp3d, c->trif_ring, 3 * d);
+  launch_pdl(c, 1, upsample_add_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->hv_ring, (const float*)c->trif_ring, c->xv,
+             (const float*)c->layers[3][0].g1, c->a_norm, c->ssq, c->ssq_tiles, c->ssq_ld);
+  run_stack(c, 3, c->xv, c->zv, nullptr, true);                    // leaves bf16(xv) in a_norm
+  gemm(c, c->U_vc, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rv, na + 1, tc::EPI_F32, epi_plain(c->tmp3d, 3 * d));
+  launch_pdl(c, 1, ring_store_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->tmp3d, c->triv_ring, 3 * d);
+  launch_pdl(c, 1, upsample_add_kernel, Rc, 128, 0, dm, c->st, B, 0, (const float*)c->hc_ring, (const float*)c->triv_ring, c->xc,
+             (const float*)c->layers[4][0].g1, c->a_norm, c->ssq, c->ssq_tiles, c->ssq_ld);
+  run_stack(c, 4, c->xc, c->zc, c->g_out, true);                   // leaves bf16(xc * g_out) and its sums of squares
+  tc::Epi el = epi_plain(c->logits, dm.Vpad);
+  el.ssq_in = c->ssq; el.ssq_tiles = c->ssq_tiles; el.ld_ssq = c->ssq_ld; el.inv_d_in = 1.f / d; el.eps = dm.eps;
+  gemm(c, c->W_out, dm.Vpad, 0, c->a_norm, Rc_alloc, 0, dm.V, d, Rc, na, tc::EPI_F32, el);
+  launch_pdl(c, 1, verify_top2_kernel, Rc, 256, 0, dm, c->st, B, (const float*)c->logits, logits_out);
 }
 
 // a13: draft heads on the stashed split-node hiddens
@@ -500,22 +529,20 @@ void draft(fm_ctx* c, float* logits_out, float* margin_out) {
     const int* na = c->st.n_active + 3;
     const size_t MB = dm.max_batch;
     LAUNCH(c, draft_prep_kernel, dim3(B, dm.NH), 256, 0, dm, c->st, B, c->zc, c->zv, c->zf, c->head_g, c->dh_a);
-    for (int h = 0; h < dm.NH; ++h) {
-      PartView ph = gemm(c, c->headA, (size_t)dm.NH * dpad, h * dpad, c->dh_a, (size_t)dm.NH * MB + 16, h * (int)MB, d, d, B, na);
-      fold<FOLD_F32>(c, ph, c->dh_y + (size_t)h * MB * d, d, d, B);
-    }
-    LAUNCH(c, draft_residual_kernel, dim3(B, dm.NH), 128, 0, dm, c->st, B, c->zc, c->zv, c->zf, c->dh_y, c->feat,
-           c->up_in_v, c->up_in_f);
-    PartView pf = gemm(c, c->U_fv, pad128(3 * d), 0, c->up_in_f, align_up((size_t)dm.Ef * MB, 16), 0, 3 * d, d, dm.Ef * B, na);
-    fold<FOLD_BF16>(c, pf, c->up_in_v + (size_t)2 * B * d, 3 * d, 3 * d, dm.Ef * B);
-    PartView pu = gemm(c, c->U_vc, pad128(3 * d), 0, c->up_in_v, align_up((2 + 3 * (size_t)dm.Ef) * MB, 16), 0, 3 * d, d,
-                       (2 + 3 * dm.Ef) * B, na);
-    fold<FOLD_F32>(c, pu, c->feat + (size_t)2 * B * d, 3 * d, 3 * d, (2 + 3 * dm.Ef) * B);
-    LAUNCH(c, rmsnorm_kernel, NF * B, 256, 0, c->feat, c->g_out, c->feat_n, d, dm.eps);
-    PartView pl = gemm(c, c->W_out, dm.Vpad, 0, c->feat_n, align_up((size_t)NF * MB, 16), 0, dm.V, d, NF * B, na);
-    fold<FOLD_F32>(c, pl, c->dlogits, dm.Vpad, dm.V, NF * B);
+    for (int h = 0; h < dm.NH; ++h)
+      gemm(c, c->headA, (size_t)dm.NH * dpad, h * dpad, c->dh_a, (size_t)dm.NH * MB + 16, h * (int)MB, d, d, B, na, tc::EPI_F32,
+           epi_plain(c->dh_y + (size_t)h * MB * d, d));
+    launch_pdl(c, 1, draft_residual_kernel, dim3(B, dm.NH), 128, 0, dm, c->st, B, (const float*)c->zc, (const float*)c->zv,
+               (const float*)c->zf, (const float*)c->dh_y, c->feat, c->up_in_v, c->up_in_f);
+    gemm(c, c->U_fv, pad128(3 * d), 0, c->up_in_f, align_up((size_t)dm.Ef * MB, 16), 0, 3 * d, d, dm.Ef * B, na, tc::EPI_BF16,
+         epi_plain(c->up_in_v + (size_t)2 * B * d, 3 * d));
+    gemm(c, c->U_vc, pad128(3 * d), 0, c->up_in_v, align_up((2 + 3 * (size_t)dm.Ef) * MB, 16), 0, 3 * d, d, (2 + 3 * dm.Ef) * B, na,
+         tc::EPI_F32, epi_plain(c->feat + (size_t)2 * B * d, 3 * d));
+    launch_pdl(c, 1, rmsnorm_kernel, NF * B, 256, 0, (const float*)c->feat, (const float*)c->g_out, c->feat_n, d, dm.eps);
+    gemm(c, c->W_out, dm.Vpad, 0, c->feat_n, align_up((size_t)NF * MB, 16), 0, dm.V, d, NF * B, na, tc::EPI_F32,
+         epi_plain(c->dlogits, dm.Vpad));
   }
-  LAUNCH(c, draft_pick_kernel, dim3(B, dm.R1), 256, 0, dm, c->st, B, c->dlogits, logits_out, margin_out);
+  launch_pdl(c, 1, draft_pick_kernel, dim3(B, dm.R1), 256, 0, dm, c->st, B, (const float*)c->dlogits, logits_out, margin_out);
 }
 
 __global__ void verify_load_kernel(Dims dm, SeqState st, int batch, const int* __restrict__ cand) {
@@ -696,7 +723,11 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
       if (L.tmK < 0 || L.tmV < 0) { delete c; return FM_ERR_CUDA; }
     }
   TRYCUDA(cudaMemcpy(c->tmaps, c->tmaps_host.data(), c->tmaps_host.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice));
-  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(256)));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(256)));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(256)));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_GELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(256)));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(256)));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(256)));
   TRYCUDA(cudaFuncSetAttribute(attn_split_kernel<64, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<64, 256>::BYTES));
   TRYCUDA(cudaFuncSetAttribute(attn_split_kernel<128, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<128, 128>::BYTES));
   std::vector<double> freq(dm.dh / 2);
@@ -717,6 +748,12 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
   c->batch = 0;
   c->phase = 0;
   c->launches = 0;
+  {
+    const char* v = getenv("FM_NO_PDL");
+    c->use_pdl = !(v != nullptr && v[0] == '1');
+    const char* t = getenv("FM_SPLIT_TARGET");
+    c->split_target = t != nullptr && atoi(t) > 0 ? atoi(t) : 160;
+  }
   *out = c;
   return FM_OK;
 }
@@ -781,9 +818,8 @@ int fm_prefill(fm_ctx* c, int32_t batch, const float* cond, const int32_t* promp
     for (int s = 0; s < 5; ++s)
       for (auto& L : c->layers[s]) {
         LAUNCH(c, rmsnorm_kernel, rows, 256, 0, cond + (size_t)r0 * dm.d, L.g1, c->pre_a, dm.d, dm.eps);
-        PartView pk = gemm(c, L.Wqkv, pad128((size_t)(dm.H + 2 * dm.Hkv) * dm.dh), dm.H * dm.dh, c->pre_a, PREFILL_CHUNK, 0,
-                           kvw, dm.d, rows, nullptr);
-        fold<FOLD_F32>(c, pk, c->pre_o, kvw, kvw, rows);
+        gemm(c, L.Wqkv, pad128((size_t)(dm.H + 2 * dm.Hkv) * dm.dh), dm.H * dm.dh, c->pre_a, PREFILL_CHUNK, 0, kvw, dm.d, rows,
+             nullptr, tc::EPI_F32, epi_plain(c->pre_o, kvw));
         LAUNCH(c, prefix_store_kernel, rows, 128, 0, dm, STACK_LEVEL[s], r0, c->pre_o, L.K, L.V);
       }
   }

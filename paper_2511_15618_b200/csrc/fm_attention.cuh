@@ -17,7 +17,7 @@ struct AttnArgs {
   Dims dm;
   SeqState st;
   int batch, level;
-  const float* q;             // [rows, H*dh] fp32, rotated
+  const bf16* q;              // [rows, H*dh] bf16, rotated and scaled by log2(e)/sqrt(dh)
   const CUtensorMap* tmK;     // cache as 2-D [B*Hkv*slots, dh], box 64 x 64
   const CUtensorMap* tmV;
   float* part;                // [B*Hkv, max_chunks, MROWS, dh + 2]
@@ -50,6 +50,8 @@ __global__ void __launch_bounds__(128) attn_split_kernel(const AttnArgs a) {
   const Dims& dm = a.dm;
   const int chunk = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t4 = lane & 3;
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();                            // queries and the new keys/values come from the previous kernel
   if (b >= a.batch) return;
   const int n = a.st.nrow[b];
   if (n <= 0) return;
@@ -104,7 +106,6 @@ __global__ void __launch_bounds__(128) attn_split_kernel(const AttnArgs a) {
     if (threadIdx.x == 0) atomicExch(a.st.status, -5);
     return;
   }
-  const float qscale = rsqrtf((float)DH) * 1.4426950408889634f;       // 1/sqrt(dh) * log2(e)
   const uint32_t Ks_u = ptx::smem_u32(Ks), Vs_u = ptx::smem_u32(Vs);
   float* gpart = a.part + ((size_t)(b * dm.Hkv + hk) * a.max_chunks + chunk) * a.mrows * (DH + 2);
 
@@ -118,16 +119,11 @@ __global__ void __launch_bounds__(128) attn_split_kernel(const AttnArgs a) {
       const bool ok = idx < M;
       const int r = ok ? idx / group : 0, gh = ok ? idx - r * group : 0;
       prow[hrow] = ok ? p0 + r : -100;
-      const float* qp = a.q + ((size_t)(b * m_rows + r) * dm.H + hk * group + gh) * DH;
+      const bf16* qp = a.q + ((size_t)(b * m_rows + r) * dm.H + hk * group + gh) * DH;
 #pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
-        float2 lo = make_float2(0.f, 0.f), hi = make_float2(0.f, 0.f);
-        if (ok) {
-          lo = *reinterpret_cast<const float2*>(qp + ks * 16 + 2 * t4);
-          hi = *reinterpret_cast<const float2*>(qp + ks * 16 + 8 + 2 * t4);
-        }
-        qa[ks][hrow] = ptx::pack_bf16(lo.x * qscale, lo.y * qscale);
-        qa[ks][2 + hrow] = ptx::pack_bf16(hi.x * qscale, hi.y * qscale);
+        qa[ks][hrow] = ok ? *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 2 * t4) : 0u;
+        qa[ks][2 + hrow] = ok ? *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8 + 2 * t4) : 0u;
       }
     }
     // ---- S = Q K^T over this warp's C/4 keys

@@ -1,15 +1,26 @@
-// Skinny weight-streaming GEMM on the 5th-generation tensor cores.
+// Skinny weight-streaming GEMM on the 5th-generation tensor cores, with the row-wise work that
+// follows each projection fused into its tail.
 //
-//   part[z][n][m] = sum_{k in K-range z} W[m, k] * A[n, k]        (bf16 operands, fp32 in TMEM)
+//   y[n][m] = sum_k W[m, k] * A[n, k]        (bf16 operands, fp32 accumulation in tensor memory)
 //
 // The weight matrix sits on the MMA's M axis (tiles of 128 output features), the few token rows
 // on its N axis (16..256, padded), so a [128 x 64] weight slab is consumed by four
 // tcgen05.mma (K = 16 each) however few rows there are.  Both operands are K-major and are
 // brought in by TMA with the 128-byte swizzle into a ring of shared-memory stages; one thread
 // issues the MMAs, accumulators live in tensor memory and are read back with tcgen05.ld.
-// The work is bandwidth bound: the grid is (M/128 tiles) x (K split) so that all SMs stream
-// weights; every CTA stores its partial tile, and the (row-wise) consumer kernel adds the
-// partials in split order -- a fixed order, so results do not depend on the number of rows.
+// The work is bandwidth bound: the grid is (M/128 tiles) x (S splits of K) so that many SMs
+// stream weights.  The S CTAs of one M tile form a thread-block cluster: each puts its partial
+// tile in its own shared memory, and after a cluster barrier every CTA adds, in rank order (a
+// fixed order, so a row's result does not depend on how many rows the launch holds), the S
+// partials of its share of the tile's columns through distributed shared memory and applies the
+// epilogue of the projection: RMSNorm scale of the operand rows, then one of
+//   EPI_F32 / EPI_BF16   plain store,
+//   EPI_GELU             bf16(gelu(y))                      (first FFN matrix),
+//   EPI_RESID            x (+)= y; next operand bf16(x * gain); per-tile sums of squares
+//                        (output projection, second FFN matrix, shorten),
+//   EPI_QKV              rotary embedding, queries out, keys / values appended to the cache.
+// The kernel is written for programmatic dependent launch: weights do not depend on the
+// previous kernel, so their first stages are requested before griddepcontrol.wait.
 #pragma once
 #include "fm_common.cuh"
 #include "fm_ptx.cuh"
@@ -19,19 +30,37 @@ namespace tc {
 constexpr int BM = 128;          // output features per CTA
 constexpr int BK = 64;           // K elements per slab (128 bytes of bf16)
 constexpr int STAGES = 4;
+constexpr int MAX_SPLIT = 8;     // portable cluster size
+
+enum EpiMode { EPI_F32 = 0, EPI_BF16 = 1, EPI_GELU = 2, EPI_RESID = 3, EPI_QKV = 4 };
 
 struct Args {
   const CUtensorMap* tmW;        // [Mpad, K] bf16, box 128 x 64
   const CUtensorMap* tmA;        // [rows, K] bf16, box N x 64
-  float* part;                   // [split][n_rows_ld][ldm]
   int M, K, N;                   // N = padded rows in the box (multiple of 16, <= 256)
   int n_store;                   // rows actually stored (<= N)
-  int ldm;                       // leading dimension of part rows (>= M)
-  long long split_stride;        // elements between splits
-  int split;                     // K splits = gridDim.y
+  int split;                     // K splits = gridDim.y = cluster size (1, 2, 4 or 8)
   int w_row0, a_row0;            // row offsets into the tensor maps (stacked weights / row groups)
-  const int* n_active;           // skip when *n_active == 0 (may be null)
+  const int* n_active;           // skip when *n_active == 0 (may be null); must not change during a pass
   int* status;
+};
+
+struct Epi {
+  int row0;                      // first output row of this launch (N tiles beyond the first)
+  const float* ssq_in;           // [ssq_tiles][ld_ssq] sums of squares of the operand rows; null = no scale
+  int ssq_tiles, ld_ssq;
+  float inv_d_in, eps;
+  void* out; int ldo;            // EPI_F32 / EPI_BF16 / EPI_GELU
+  float* x; int ldx; int add;    // EPI_RESID: residual stream, add = 0 replaces it
+  const float* gain;             //            gain of the next norm (null = 1)
+  bf16* a_out; int lda;          //            next GEMM's operand rows (may be null)
+  float* ssq_out; int ld_ssq_out;//            [M tiles][ld] sums of squares of the new x rows (may be null)
+  Dims dm; SeqState st;          // EPI_QKV
+  int batch, level;
+  const float2* rope_tab;
+  bf16* q_out;                   //            [rows, H*dh], rotated and scaled by qscale
+  bf16* Kc; bf16* Vc;            //            caches [B, Hkv, slots, dh]
+  float qscale;
 };
 
 __device__ inline uint64_t smem_desc_sw128(uint32_t addr) {
@@ -67,12 +96,46 @@ __device__ inline void ld16(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// ---- thread-block cluster: rank, barrier, loads from a peer CTA's shared memory
+__device__ inline uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ inline void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ inline float ld_peer(uint32_t local_addr, uint32_t rank) {
+  uint32_t ra;
+  float v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(ra));
+  return v;
+}
+
+// The stage ring is reused for the partial tile [N][128] fp32 (N * 512 bytes) and, behind it, for
+// the squares of EPI_RESID ([N][64 / split] fp32 <= 64 KB): STAGES * 16 KB + N * 512 >= both.
 inline int smem_bytes(int N) { return STAGES * (BM * 128 + ((N * 128 + 1023) / 1024) * 1024) + 1024 + 256; }
 
-// grid (M/128 tiles, split); block 128.  Warp 0 lane 0 feeds TMA, warp 1 lane 0 issues MMAs,
-// all four warps read the accumulator back (warp w owns TMEM lanes 32w..32w+31).
-__global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g) {
-  if (g.n_active != nullptr && *g.n_active == 0) return;
+__device__ inline float gelu_erf_f(float x) { return 0.5f * x * (1.f + erff(x * 0.70710678118654752f)); }
+
+// Pair slot q (0..63) of a 128-column tile -> its two columns.  Rotary pairs are (i, i + dh/2)
+// inside a head, so with heads of 64 a tile holds two heads with 32 pairs each, with heads of
+// 128 one head with 64 pairs.  The other epilogues use the same map (any bijection would do).
+__device__ inline void pair_cols(int q, bool head128, int& ca, int& cb) {
+  if (head128) { ca = q; cb = q + 64; }
+  else { ca = (q >> 5) * 64 + (q & 31); cb = ca + 32; }
+}
+
+// grid (M/128 tiles, split), cluster (1, split, 1); block 128.  Warp 0 lane 0 feeds TMA, warp 1
+// lane 0 issues MMAs, all four warps read the accumulator back (warp w owns TMEM lanes 32w..32w+31).
+template <int MODE>
+__global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e) {
+  if (g.n_active != nullptr && *g.n_active == 0) {   // the whole grid leaves; keep the launch chain ordered
+    ptx::grid_dep_launch();
+    ptx::grid_dep_wait();
+    return;
+  }
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int b_bytes = ((g.N * 128 + 1023) / 1024) * 1024;
@@ -82,16 +145,20 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g) {
   uint64_t* accum = empty + STAGES;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
   __shared__ int s_fail;
+  __shared__ float s_inv[256], s_rowsq[256];
+  __shared__ int s_rb[256], s_rp[256];
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tile_m = blockIdx.x, z = blockIdx.y;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tile_m = blockIdx.x;
+  const int S = g.split;
+  const int z = (int)cluster_rank();                 // == blockIdx.y: the cluster spans the grid's y extent
   const int slabs = g.K / BK;
-  const int s0 = (int)((long long)slabs * z / g.split), s1 = (int)((long long)slabs * (z + 1) / g.split);
+  const int s0 = (int)((long long)slabs * z / S), s1 = (int)((long long)slabs * (z + 1) / S);
   const int n_slabs = s1 - s0;
   uint32_t ncols = 32;
   while ((int)ncols < g.N) ncols <<= 1;
 
-  if (threadIdx.x == 0) {
+  if (tid == 0) {
     s_fail = 0;
     for (int i = 0; i < STAGES; ++i) { ptx::mbar_init(full + i, 1); ptx::mbar_init(empty + i, 1); }
     ptx::mbar_init(accum, 1);
@@ -108,12 +175,24 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g) {
   __syncthreads();
   fence_after();
   const uint32_t tmem = *tmem_slot;
+  // This CTA now holds its tensor memory and shared memory: the next kernel may start its own
+  // prologue beside us.
+  ptx::grid_dep_launch();
 
   if (warp == 0 && lane == 0) {
-    // ---- producer: stream this CTA's K range through the stage ring
-    for (int i = 0; i < n_slabs; ++i) {
+    // ---- producer: stream this CTA's K range through the stage ring.  The weight slabs of the
+    // first stages do not depend on the previous kernel and are requested before the wait.
+    const int pre = n_slabs < STAGES ? n_slabs : STAGES;
+    for (int i = 0; i < pre; ++i) {
+      ptx::mbar_expect_tx(full + i, BM * 128 + g.N * 128);
+      ptx::tma_load_2d(sm + i * stage_bytes, g.tmW, (s0 + i) * BK, g.w_row0 + tile_m * BM, full + i);
+    }
+    ptx::grid_dep_wait();
+    for (int i = 0; i < pre; ++i)
+      ptx::tma_load_2d(sm + i * stage_bytes + BM * 128, g.tmA, (s0 + i) * BK, g.a_row0, full + i);
+    for (int i = pre; i < n_slabs; ++i) {
       const int st = i % STAGES;
-      if (i >= STAGES && !ptx::mbar_wait(empty + st, ((i / STAGES) - 1) & 1)) { s_fail = 1; break; }
+      if (!ptx::mbar_wait(empty + st, ((i / STAGES) - 1) & 1)) { s_fail = 1; break; }
       unsigned char* a_dst = sm + st * stage_bytes;
       ptx::mbar_expect_tx(full + st, BM * 128 + g.N * 128);
       ptx::tma_load_2d(a_dst, g.tmW, (s0 + i) * BK, g.w_row0 + tile_m * BM, full + st);
@@ -136,29 +215,148 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g) {
     commit(accum);                                         // accumulator complete
   }
   __syncwarp();
-  // ---- epilogue: everyone waits for the accumulator, then stores the partial tile
+  ptx::grid_dep_wait();                                    // everything below touches activations
+
+  // ---- operand-row scales and row maps, while the MMAs drain
+  for (int n = tid; n < g.n_store; n += 128) {
+    if (e.ssq_in != nullptr) {
+      float ss = 0.f;
+      for (int t = 0; t < e.ssq_tiles; ++t) ss += __ldcg(e.ssq_in + (size_t)t * e.ld_ssq + e.row0 + n);
+      s_inv[n] = rsqrtf(ss * e.inv_d_in + e.eps);
+    } else {
+      s_inv[n] = 1.f;
+    }
+    if (MODE == EPI_QKV) {
+      int b, p;
+      const bool valid = fm_row_map(e.dm, e.st, e.batch, e.level, e.row0 + n, b, p);
+      s_rb[n] = valid ? b : -1;
+      s_rp[n] = p;
+    }
+  }
+  // ---- everyone waits for the accumulator; a timeout is recorded and the barriers below are
+  // still executed by every CTA of the cluster
   bool ok = n_slabs > 0 ? ptx::mbar_wait(accum, 0) : true;
   __syncwarp();
   fence_after();
+  __syncthreads();
   if (!ok || s_fail) {
-    if (threadIdx.x == 0) atomicExch(g.status, -5);
-  } else {
-    const int m = tile_m * BM + warp * 32 + lane;
-    float* dst = g.part + (size_t)z * g.split_stride + m;
-    for (int n0 = 0; n0 < g.N; n0 += 16) {
-      uint32_t r[16];
-      if (n_slabs > 0) ld16(tmem + ((uint32_t)(warp * 32) << 16) + n0, r);
-      else {
+    ok = false;
+    if (tid == 0) atomicExch(g.status, -5);
+  }
+  // ---- partial tile -> own shared memory (the ring is idle: every stage was consumed)
+  float* part = reinterpret_cast<float*>(sm);              // [n_store][128]
+  for (int n0 = 0; n0 < g.n_store; n0 += 16) {
+    uint32_t r[16];
+    if (ok && n_slabs > 0) ld16(tmem + ((uint32_t)(warp * 32) << 16) + n0, r);
+    else {
 #pragma unroll
-        for (int j = 0; j < 16; ++j) r[j] = 0u;
+      for (int j = 0; j < 16; ++j) r[j] = 0u;
+    }
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+      if (n0 + j < g.n_store) part[(n0 + j) * BM + tid] = __uint_as_float(r[j]);
+  }
+  cluster_sync();                                          // partials of all ranks are in place
+
+  // ---- this rank's share of the tile: pair slots [z*PW, (z+1)*PW), all rows
+  const int PW = 64 / S;
+  const int items = g.n_store * PW;
+  const uint32_t part_u = ptx::smem_u32(part);
+  const bool head128 = MODE == EPI_QKV && e.dm.dh == 128;
+  float* sq = reinterpret_cast<float*>(sm + (size_t)g.N * 512);   // [n_store][PW], EPI_RESID only
+  for (int it = tid; it < items; it += 128) {
+    const int n = it / PW, cc = it - n * PW;
+    int ca, cb;
+    pair_cols(z * PW + cc, head128, ca, cb);
+    float va[MAX_SPLIT], vb[MAX_SPLIT];
+#pragma unroll
+    for (int r = 0; r < MAX_SPLIT; ++r) {                  // all loads first, then the sums in rank order
+      va[r] = r < S ? ld_peer(part_u + (uint32_t)(n * BM + ca) * 4u, (uint32_t)r) : 0.f;
+      vb[r] = r < S ? ld_peer(part_u + (uint32_t)(n * BM + cb) * 4u, (uint32_t)r) : 0.f;
+    }
+    float ya = 0.f, yb = 0.f;
+#pragma unroll
+    for (int r = 0; r < MAX_SPLIT; ++r)
+      if (r < S) { ya += va[r]; yb += vb[r]; }
+    const float inv = s_inv[n];
+    ya *= inv;
+    yb *= inv;
+    const int ma = tile_m * BM + ca, mb = tile_m * BM + cb;
+    const size_t row = (size_t)(e.row0 + n);
+    if (MODE == EPI_F32) {
+      float* o = reinterpret_cast<float*>(e.out) + row * e.ldo;
+      if (ma < g.M) o[ma] = ya;
+      if (mb < g.M) o[mb] = yb;
+    } else if (MODE == EPI_BF16) {
+      bf16* o = reinterpret_cast<bf16*>(e.out) + row * e.ldo;
+      if (ma < g.M) o[ma] = __float2bfloat16(ya);
+      if (mb < g.M) o[mb] = __float2bfloat16(yb);
+    } else if (MODE == EPI_GELU) {
+      bf16* o = reinterpret_cast<bf16*>(e.out) + row * e.ldo;
+      if (ma < g.M) o[ma] = __float2bfloat16(gelu_erf_f(ya));
+      if (mb < g.M) o[mb] = __float2bfloat16(gelu_erf_f(yb));
+    } else if (MODE == EPI_RESID) {
+      float* xr = e.x + row * e.ldx;
+      float xa = 0.f, xb = 0.f;
+      if (ma < g.M) {
+        xa = (e.add ? xr[ma] : 0.f) + ya;
+        xr[ma] = xa;
+        if (e.a_out != nullptr) e.a_out[row * e.lda + ma] = __float2bfloat16(xa * (e.gain != nullptr ? e.gain[ma] : 1.f));
       }
-      if (m < g.M) {
-#pragma unroll
-        for (int j = 0; j < 16; ++j)
-          if (n0 + j < g.n_store) dst[(size_t)(n0 + j) * g.ldm] = __uint_as_float(r[j]);
+      if (mb < g.M) {
+        xb = (e.add ? xr[mb] : 0.f) + yb;
+        xr[mb] = xb;
+        if (e.a_out != nullptr) e.a_out[row * e.lda + mb] = __float2bfloat16(xb * (e.gain != nullptr ? e.gain[mb] : 1.f));
+      }
+      sq[it] = xa * xa + xb * xb;
+    } else {  // EPI_QKV: (ya, yb) is the rotary pair (i, i + dh/2) of one head
+      const Dims& dm = e.dm;
+      const int dh = dm.dh, half = dh >> 1, H = dm.H, Hkv = dm.Hkv;
+      const int head = ma / dh, i = ma - head * dh;
+      if (ma < g.M && head < H + 2 * Hkv) {
+        const int b = s_rb[n], p = s_rp[n];
+        const bool valid = b >= 0;
+        const int slots = dm.P + dm.cap[e.level];
+        if (head < H + Hkv) {
+          float c = 1.f, s = 0.f;
+          if (dm.theta != 0.f && valid) { const float2 cs = e.rope_tab[(size_t)p * half + i]; c = cs.x; s = cs.y; }
+          const float y1 = ya * c - yb * s, y2 = yb * c + ya * s;
+          if (head < H) {
+            bf16* q = e.q_out + (row * H + head) * dh;
+            q[i] = __float2bfloat16(valid ? y1 * e.qscale : 0.f);
+            q[half + i] = __float2bfloat16(valid ? y2 * e.qscale : 0.f);
+          } else if (valid) {
+            bf16* dst = e.Kc + (((size_t)b * Hkv + (head - H)) * slots + dm.P + (p % dm.cap[e.level])) * dh;
+            dst[i] = __float2bfloat16(y1);
+            dst[half + i] = __float2bfloat16(y2);
+          }
+        } else if (valid) {
+          bf16* dst = e.Vc + (((size_t)b * Hkv + (head - H - Hkv)) * slots + dm.P + (p % dm.cap[e.level])) * dh;
+          dst[i] = __float2bfloat16(ya);
+          dst[half + i] = __float2bfloat16(yb);
+        }
       }
     }
   }
+  if (MODE == EPI_RESID && e.ssq_out != nullptr) {
+    // per-row sums of squares: this rank's columns in slot order, then the ranks in rank order
+    __syncthreads();
+    for (int n = tid; n < g.n_store; n += 128) {
+      float t = 0.f;
+      for (int cc = 0; cc < PW; ++cc) t += sq[n * PW + cc];
+      s_rowsq[n] = t;
+    }
+    cluster_sync();
+    if (z == 0) {
+      const uint32_t rs_u = ptx::smem_u32(s_rowsq);
+      for (int n = tid; n < g.n_store; n += 128) {
+        float t = 0.f;
+        for (int r = 0; r < S; ++r) t += ld_peer(rs_u + (uint32_t)n * 4u, (uint32_t)r);
+        e.ssq_out[(size_t)tile_m * e.ld_ssq_out + e.row0 + n] = t;
+      }
+    }
+  }
+  cluster_sync();                                          // nobody leaves while a peer may still read its shared memory
   fence_before();
   __syncthreads();
   fence_after();

@@ -1,7 +1,7 @@
 // Element-wise, row-wise and bookkeeping kernels of the decode step.
 #pragma once
 #include "fm_common.cuh"
-#include "fm_gemm.cuh"
+#include "fm_ptx.cuh"
 
 // ------------------------------------------------------------------------------------------
 // block reductions (blockDim.x multiple of 32, <= 1024)
@@ -18,9 +18,32 @@ __device__ inline float block_sum(float v, float* sh) {
 }
 
 // ------------------------------------------------------------------------------------------
+// Hand a freshly written residual row to the first layer of a stack: the GEMM operand row
+// bf16(x * g) (the RMSNorm scale 1/rms is applied by the GEMM's epilogue) and the row's sum of
+// squares in tile 0 of `ssq` (the other tiles are zeroed: epilogues add all tiles).
+// ------------------------------------------------------------------------------------------
+__device__ inline void stack_entry_row(const float* xr, int row, int d, const float* __restrict__ g,
+                                       bf16* __restrict__ a_out, float* __restrict__ ssq, int ssq_tiles, int ld_ssq) {
+  __shared__ float sh[32];
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    const float v = xr[i];
+    ss += v * v;
+    a_out[(size_t)row * d + i] = __float2bfloat16(v * g[i]);
+  }
+  ss = block_sum(ss, sh);
+  if (threadIdx.x == 0) {
+    ssq[row] = ss;
+    for (int t = 1; t < ssq_tiles; ++t) ssq[(size_t)t * ld_ssq + row] = 0.f;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // a1. candidate embedding: x[row] = E[cand[b][j]]  (zeros for rows that are not fed)
 // ------------------------------------------------------------------------------------------
-__global__ void embed_kernel(Dims dm, SeqState st, int batch, const bf16* __restrict__ E, float* __restrict__ x) {
+__global__ void embed_kernel(Dims dm, SeqState st, int batch, const bf16* __restrict__ E, float* __restrict__ x,
+                             const float* __restrict__ g, bf16* __restrict__ a_out, float* __restrict__ ssq, int ssq_tiles,
+                             int ld_ssq) {
   const int row = blockIdx.x;
   int b, p;
   const bool valid = fm_row_map(dm, st, batch, 0, row, b, p);
@@ -34,35 +57,15 @@ __global__ void embed_kernel(Dims dm, SeqState st, int batch, const bf16* __rest
   }
   for (int i = threadIdx.x; i < dm.d; i += blockDim.x)
     x[(size_t)row * dm.d + i] = valid ? __bfloat162float(E[(size_t)tok * dm.d + i]) : 0.f;
-}
-
-// ------------------------------------------------------------------------------------------
-// Residual fold + RMSNorm: first x[row] (+)= sum of the pending GEMM partials (mode 1 adds them
-// to the residual stream, mode 2 replaces it, mode 0 leaves x alone), then, if a gain is given,
-// out = bf16(x / sqrt(mean(x^2)+eps) * g), the next GEMM's operand row.  One CTA per row.
-// ------------------------------------------------------------------------------------------
-__global__ void resid_norm_kernel(float* __restrict__ x, PartView pv, int mode, const float* __restrict__ g,
-                                  bf16* __restrict__ out, int d, float eps) {
-  __shared__ float sh[32];
-  extern __shared__ float xrow[];                   // d floats
-  float* xr = x + (size_t)blockIdx.x * d;
-  float ss = 0.f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    float v = mode == 2 ? 0.f : xr[i];
-    if (mode != 0) { v += part_sum(pv, blockIdx.x, i); xr[i] = v; }
-    xrow[i] = v;
-    ss += v * v;
-  }
-  if (g == nullptr) return;
-  ss = block_sum(ss, sh);
-  const float inv = rsqrtf(ss / (float)d + eps);
-  for (int i = threadIdx.x; i < d; i += blockDim.x)
-    out[(size_t)blockIdx.x * d + i] = __float2bfloat16(xrow[i] * inv * g[i]);
+  __syncthreads();
+  stack_entry_row(x + (size_t)row * dm.d, row, dm.d, g, a_out, ssq, ssq_tiles, ld_ssq);
 }
 
 // RMSNorm of read-only fp32 rows (conditioning vectors, draft features) -> bf16 operand rows
 __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ g, bf16* __restrict__ out,
                                int d, float eps) {
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
   __shared__ float sh[32];
   const float* xr = x + (size_t)blockIdx.x * d;
   float ss = 0.f;
@@ -74,11 +77,8 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
 }
 
 // ------------------------------------------------------------------------------------------
-// RoPE on q and k (rotate-half pairs (i, i+dh/2), angle = pos * theta^(-2i/dh); cos/sin come from
-// a table evaluated in double precision when the context is created), then append k, v to the
-// level's cache at slot P + pos % cap.
-// qkv: split-K partials of [rows, (H+2Hkv)*dh]; q_out: fp32 [rows, H*dh]; caches: bf16 [B, Hkv, slots, dh].
-// grid (rows, (H + 2*Hkv) / 2): each CTA of dh threads handles two heads of one row.
+// RoPE table: (cos, sin) of pos * theta^(-2i/dh) for every level-local position, evaluated in
+// double precision when the context is created (the rotation itself is in the QKV epilogue).
 // ------------------------------------------------------------------------------------------
 __global__ void rope_table_kernel(float2* __restrict__ tab, const double* __restrict__ inv_freq, int n_pos, int half) {
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -87,38 +87,6 @@ __global__ void rope_table_kernel(float2* __restrict__ tab, const double* __rest
   double s, c;
   sincos((double)pos * inv_freq[k], &s, &c);
   tab[i] = make_float2((float)c, (float)s);
-}
-
-__global__ void rope_append_kernel(Dims dm, SeqState st, int batch, int level, PartView qkv,
-                                   const float2* __restrict__ rope_tab, float* __restrict__ q_out,
-                                   bf16* __restrict__ Kc, bf16* __restrict__ Vc) {
-  const int row = blockIdx.x;
-  int b, p;
-  const bool valid = fm_row_map(dm, st, batch, level, row, b, p);
-  const int H = dm.H, Hkv = dm.Hkv, dh = dm.dh, half = dh / 2;
-  const int slots = dm.P + dm.cap[level];
-  const int slot = dm.P + (p % dm.cap[level]);
-  const int head = blockIdx.y * 2 + threadIdx.x / half;     // 0..H-1 q, H..H+Hkv-1 k, then v
-  const int i = threadIdx.x % half;
-  if (head >= H + 2 * Hkv) return;
-  const float x1 = part_sum(qkv, row, head * dh + i), x2 = part_sum(qkv, row, head * dh + half + i);
-  if (head < H + Hkv) {
-    float c = 1.f, s = 0.f;
-    if (dm.theta != 0.f) { const float2 cs = rope_tab[(size_t)p * half + i]; c = cs.x; s = cs.y; }
-    const float y1 = x1 * c - x2 * s, y2 = x2 * c + x1 * s;
-    if (head < H) {
-      q_out[(size_t)row * H * dh + head * dh + i] = valid ? y1 : 0.f;
-      q_out[(size_t)row * H * dh + head * dh + half + i] = valid ? y2 : 0.f;
-    } else if (valid) {
-      bf16* dst = Kc + (((size_t)b * Hkv + (head - H)) * slots + slot) * dh;
-      dst[i] = __float2bfloat16(y1);
-      dst[half + i] = __float2bfloat16(y2);
-    }
-  } else if (valid) {
-    bf16* dst = Vc + (((size_t)b * Hkv + (head - H - Hkv)) * slots + slot) * dh;
-    dst[i] = __float2bfloat16(x1);
-    dst[half + i] = __float2bfloat16(x2);
-  }
 }
 
 // prefix keys/values of one layer: kv fp32 [rows, 2*Hkv*dh] (rows = chunk of b*P+j) -> slots [0,P)
@@ -143,6 +111,8 @@ __global__ void prefix_store_kernel(Dims dm, int level, int row0, const float* _
 // ring[b][p % ring][:] = x[row][:] for rows that are fed (width = floats per entry)
 __global__ void ring_store_kernel(Dims dm, SeqState st, int batch, int level, const float* __restrict__ x,
                                   float* __restrict__ ring, int width) {
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
   const int row = blockIdx.x;
   int b, p;
   if (!fm_row_map(dm, st, batch, level, row, b, p)) return;
@@ -156,6 +126,8 @@ __global__ void ring_store_kernel(Dims dm, SeqState st, int batch, int level, co
 // the ring of the level below (zeros for negative positions and for rows that are not fed)
 __global__ void shorten_gather_kernel(Dims dm, SeqState st, int batch, int level_out, const float* __restrict__ ring,
                                       bf16* __restrict__ out) {
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
   const int row = blockIdx.x;
   int b, v;
   const bool valid = fm_row_map(dm, st, batch, level_out, row, b, v);
@@ -169,9 +141,13 @@ __global__ void shorten_gather_kernel(Dims dm, SeqState st, int batch, int level
   }
 }
 
-// a7/a9 upsample, residual half: x[row] = h_ring[b][p] + tri_ring[b][p/3][(p%3)*d ...]
+// a7/a9 upsample, residual half: x[row] = h_ring[b][p] + tri_ring[b][p/3][(p%3)*d ...]; the row is
+// then handed to the first layer of the stack above (operand row and sum of squares)
 __global__ void upsample_add_kernel(Dims dm, SeqState st, int batch, int level, const float* __restrict__ h_ring,
-                                    const float* __restrict__ tri_ring, float* __restrict__ x) {
+                                    const float* __restrict__ tri_ring, float* __restrict__ x, const float* __restrict__ g,
+                                    bf16* __restrict__ a_out, float* __restrict__ ssq, int ssq_tiles, int ld_ssq) {
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
   const int row = blockIdx.x;
   int b, p;
   const bool valid = fm_row_map(dm, st, batch, level, row, b, p);
@@ -179,6 +155,8 @@ __global__ void upsample_add_kernel(Dims dm, SeqState st, int batch, int level, 
   const float* h = h_ring + ((size_t)b * rs + (p % rs)) * d;
   const float* t = tri_ring + ((size_t)b * rsu + ((p / 3) % rsu)) * 3 * d + (p % 3) * d;
   for (int i = threadIdx.x; i < d; i += blockDim.x) x[(size_t)row * d + i] = valid ? h[i] + t[i] : 0.f;
+  __syncthreads();
+  stack_entry_row(x + (size_t)row * d, row, d, g, a_out, ssq, ssq_tiles, ld_ssq);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -224,6 +202,8 @@ __device__ inline Top2 block_top2(const float* __restrict__ z, const Dims& dm, i
 
 __global__ void verify_top2_kernel(Dims dm, SeqState st, int batch, const float* __restrict__ logits,
                                    float* __restrict__ logits_out) {
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
   const int row = blockIdx.x;
   int b, p;
   const bool valid = fm_row_map(dm, st, batch, 0, row, b, p);
@@ -384,6 +364,8 @@ __global__ void draft_residual_kernel(Dims dm, SeqState st, int batch, const flo
                                       const float* __restrict__ zf, const float* __restrict__ y /*[NH,max_batch,d]*/,
                                       float* __restrict__ feat /*[NF*B, d]*/, bf16* __restrict__ up_in_v /*[2B + 3*Ef*B, d]*/,
                                       bf16* __restrict__ up_in_f /*[Ef*B, d]*/) {
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
   const int h = blockIdx.y, b = blockIdx.x, d = dm.d;
   if (b >= batch) return;
   const int n = max(0, st.L[b] - 1);
@@ -416,6 +398,8 @@ __device__ inline int draft_feature_row(int n, int j, int b, int B) {
 // masked argmax of the chosen feature's logits -> cand[b][j]; cand[b][0] = pending main token
 __global__ void draft_pick_kernel(Dims dm, SeqState st, int batch, const float* __restrict__ logits /*[NF*B, Vpad]*/,
                                   float* __restrict__ logits_out, float* __restrict__ margin_out) {
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
   const int b = blockIdx.x, j = blockIdx.y;        // j = 0..D
   if (b >= batch) return;
   const bool fin = st.done[b] != 0 || st.nrow[b] <= 0;
