@@ -61,7 +61,7 @@ struct fm_ctx {
   // attention scratch and TMA descriptors
   float* attn_part;
   int* attn_ticket;
-  int attn_chunk, attn_max_chunks[3], attn_mrows[3];
+  int attn_chunk, attn_G[3], attn_max_groups[3], attn_mt[3];
   CUtensorMap* tmaps;                    // device array
   std::vector<CUtensorMap> tmaps_host;
   struct TmapKey { const void* base; uint64_t rows, cols; uint32_t box_rows; };
@@ -69,7 +69,7 @@ struct fm_ctx {
   size_t tmaps_cap, tmaps_uploaded;
   // per-tile sums of squares of the residual rows (RMSNorm statistics handed between GEMMs)
   float* ssq;
-  int ssq_tiles, ssq_ld;
+  int ssq_n, ssq_ld;    // slots the last producer filled, floats between slots
   bool use_pdl;
   // prefill temporaries
   bf16* pre_a;
@@ -193,8 +193,8 @@ void carve(fm_ctx* c, Carver& cv) {
   const size_t Rc = align_up(B * dm.R1, 16), Rv = align_up(B * dm.mv, 16), Rf = align_up(B * dm.mf, 16);
   c->xc = cv.take<float>(Rc * d); c->xv = cv.take<float>(Rv * d); c->xf = cv.take<float>(Rf * d);
   c->qbuf = cv.take<bf16>(Rc * hd);
-  c->ssq_tiles = (int)((d + 127) / 128); c->ssq_ld = (int)Rc;
-  c->ssq = cv.take<float>((size_t)c->ssq_tiles * Rc);
+  c->ssq_ld = (int)Rc;
+  c->ssq = cv.take<float>((size_t)((d + 127) / 128) * tc::MAX_SPLIT * Rc);
   c->logits = cv.take<float>(Rc * dm.Vpad); c->tmp3d = cv.take<float>(Rv * 3 * d);
   c->a_norm = cv.take<bf16>(Rc * d); c->a_cat = cv.take<bf16>(Rv * 3 * d);
   c->a_attn = cv.take<bf16>(Rc * hd); c->a_ff = cv.take<bf16>(Rc * dm.dff);
@@ -209,17 +209,24 @@ void carve(fm_ctx* c, Carver& cv) {
   c->up_in_f = cv.take<bf16>(align_up((size_t)dm.Ef * B, 16) * d);
   c->feat = cv.take<float>(align_up(NF * B, 16) * d); c->feat_n = cv.take<bf16>(align_up(NF * B, 16) * d);
   c->dlogits = cv.take<float>(align_up(NF * B, 16) * dm.Vpad);
-  // attention: chunk partials (max over levels), tickets, tensor maps
-  c->attn_chunk = dm.dh == 64 ? 256 : 128;
-  size_t part_max = 0;
+  // attention: chunk size, chunks per group (fixed per level so that the reduction order of a row
+  // never depends on the cache length), group partials (max over levels), tickets
+  c->attn_chunk = dm.dh == 64 ? 128 : 64;
+  size_t part_max = 0, ticket_max = 0;
   for (int l = 0; l < 3; ++l) {
-    c->attn_max_chunks[l] = (dm.P + dm.cap[l] + c->attn_chunk - 1) / c->attn_chunk;
-    c->attn_mrows[l] = round_up(fm_rows_per_seq(dm, l) * (dm.H / dm.Hkv), 16);
-    const size_t need = B * dm.Hkv * (size_t)c->attn_max_chunks[l] * c->attn_mrows[l] * (dm.dh + 2);
+    const int max_chunks = (dm.P + dm.cap[l] + c->attn_chunk - 1) / c->attn_chunk;
+    c->attn_mt[l] = (fm_rows_per_seq(dm, l) * (dm.H / dm.Hkv) + 15) / 16;
+    int G = (int)(((size_t)max_chunks * dm.Hkv * B * c->attn_mt[l] + 147) / 148);
+    G = G < 1 ? 1 : (G > 16 ? 16 : G);
+    c->attn_G[l] = G;
+    c->attn_max_groups[l] = (max_chunks + G - 1) / G;
+    const size_t need = B * dm.Hkv * (size_t)c->attn_mt[l] * c->attn_max_groups[l] * 16 * (dm.dh + 2);
     part_max = need > part_max ? need : part_max;
+    const size_t tk = B * dm.Hkv * (size_t)c->attn_mt[l];
+    ticket_max = tk > ticket_max ? tk : ticket_max;
   }
   c->attn_part = cv.take<float>(part_max);
-  c->attn_ticket = cv.take<int>(B * dm.Hkv);
+  c->attn_ticket = cv.take<int>(ticket_max);
   int n_layers = 0;
   for (int s = 0; s < 5; ++s) n_layers += c->cfg.layers[s];
   c->tmaps_cap = (size_t)6 * n_layers + 128;
@@ -392,14 +399,15 @@ void gemm(fm_ctx* c, const bf16* W, size_t w_rows_alloc, int w_row0, const bf16*
   const int Rpad = round_up(R, 16);
   const int tW = tmap_for(c, W, w_rows_alloc, K, tc::BM);
   const long pi = prof_open(c, PROF_GEMM, 2.0 * M * K);            // algorithmic bytes: the weight matrix once
-  for (int n0 = 0; n0 < Rpad; n0 += 256) {                         // N tiles of at most 256 rows
-    const int N = Rpad - n0 < 256 ? Rpad - n0 : 256;
+  for (int n0 = 0; n0 < Rpad; n0 += tc::MAX_N) {                   // N tiles of at most MAX_N rows
+    const int N = Rpad - n0 < tc::MAX_N ? Rpad - n0 : tc::MAX_N;
     const int tA = tmap_for(c, A, a_rows_alloc, K, N);
     if (tW < 0 || tA < 0) { c->launch_error = FM_ERR_CUDA; break; }
-    tc::Args g{c->tmaps + tW, c->tmaps + tA, M, K, N, (R - n0 < N ? R - n0 : N), split, w_row0, a_row0 + n0, n_active,
+    const int stages = tc::pick_stages(N);
+    tc::Args g{c->tmaps + tW, c->tmaps + tA, M, K, N, (R - n0 < N ? R - n0 : N), split, stages, w_row0, a_row0 + n0, n_active,
                c->st.status};
     e.row0 = n0;
-    const int smem = tc::smem_bytes(N);
+    const int smem = tc::smem_bytes(N, stages);
     const dim3 grid(tiles, split);
     switch (mode) {
       case tc::EPI_F32: launch_pdl(c, split, tc::gemm_tc_kernel<tc::EPI_F32>, grid, 128, smem, g, e); break;
@@ -410,6 +418,7 @@ void gemm(fm_ctx* c, const bf16* W, size_t w_rows_alloc, int w_row0, const bf16*
     }
   }
   prof_close(c, pi);
+  if (mode == tc::EPI_RESID && e.ssq_out != nullptr) c->ssq_n = tiles * split * (split == 1 ? 2 : 1);     // slots the next consumer adds
 }
 
 // rows fed at each level in this pass (n_active[level]); n_active[3] = unfinished sequences
@@ -431,11 +440,11 @@ __global__ void row_count_kernel(Dims dm, SeqState st, int batch) {
 void attention(fm_ctx* c, int level, const LayerDev& L) {
   const Dims& dm = c->dm;
   AttnArgs a{dm, c->st, c->batch, level, c->qbuf, c->tmaps + L.tmK, c->tmaps + L.tmV, c->attn_part, c->attn_ticket,
-             c->a_attn, c->attn_max_chunks[level], c->attn_mrows[level]};
-  dim3 grid(c->attn_max_chunks[level], dm.Hkv, c->batch);
+             c->a_attn, c->attn_G[level], c->attn_max_groups[level], c->attn_mt[level]};
+  dim3 grid(c->attn_max_groups[level] * c->attn_mt[level], dm.Hkv, c->batch);
   const long pi = prof_open(c, PROF_ATTN, 0.0);
-  if (dm.dh == 64) launch_pdl(c, 1, attn_split_kernel<64, 256>, grid, 128, AttnSmem<64, 256>::BYTES, a);
-  else launch_pdl(c, 1, attn_split_kernel<128, 128>, grid, 128, AttnSmem<128, 128>::BYTES, a);
+  if (dm.dh == 64) launch_pdl(c, 1, attn_stream_kernel<64, 128, 8>, grid, AttnCfg<64, 128, 8>::THREADS, AttnCfg<64, 128, 8>::BYTES, a);
+  else launch_pdl(c, 1, attn_stream_kernel<128, 64, 4>, grid, AttnCfg<128, 64, 4>::THREADS, AttnCfg<128, 64, 4>::BYTES, a);
   prof_close(c, pi);
 }
 
@@ -458,7 +467,7 @@ void run_stack(fm_ctx* c, int s, float* x, float* stash_ring, const float* next_
     if (stash_ring != nullptr && l == nl - 1)
       launch_pdl(c, 1, ring_store_kernel, rows, 128, 0, dm, c->st, c->batch, level, (const float*)x, stash_ring, d);
     tc::Epi eq{};
-    eq.ssq_in = c->ssq; eq.ssq_tiles = c->ssq_tiles; eq.ld_ssq = c->ssq_ld; eq.inv_d_in = 1.f / d; eq.eps = dm.eps;
+    eq.ssq_in = c->ssq; eq.ssq_n = c->ssq_n; eq.ld_ssq = c->ssq_ld; eq.inv_d_in = 1.f / d; eq.eps = dm.eps;
     eq.dm = dm; eq.st = c->st; eq.batch = c->batch; eq.level = level; eq.rope_tab = c->rope_tab;
     eq.q_out = c->qbuf; eq.Kc = L.K; eq.Vc = L.V;
     eq.qscale = (float)(1.4426950408889634 / sqrt((double)dm.dh));   // 1/sqrt(dh) * log2(e)
@@ -469,7 +478,7 @@ void run_stack(fm_ctx* c, int s, float* x, float* stash_ring, const float* next_
     eo.ssq_out = c->ssq; eo.ld_ssq_out = c->ssq_ld;
     gemm(c, L.Wo, pad128(d), 0, c->a_attn, Rc_alloc, 0, d, hd, rows, na, tc::EPI_RESID, eo);
     tc::Epi e1 = epi_plain(c->a_ff, dm.dff);
-    e1.ssq_in = c->ssq; e1.ssq_tiles = c->ssq_tiles; e1.ld_ssq = c->ssq_ld; e1.inv_d_in = 1.f / d; e1.eps = dm.eps;
+    e1.ssq_in = c->ssq; e1.ssq_n = c->ssq_n; e1.ld_ssq = c->ssq_ld; e1.inv_d_in = 1.f / d; e1.eps = dm.eps;
     gemm(c, L.W1, pad128(dm.dff), 0, c->a_norm, Rc_alloc, 0, dm.dff, d, rows, na, tc::EPI_GELU, e1);
     tc::Epi e2 = eo;
     const bool last = l == nl - 1;
@@ -489,7 +498,8 @@ void forward(fm_ctx* c, float* logits_out) {
   // The two launches that open a pass are full barriers: the per-pass state (rows, lengths,
   // candidates) is final before any later kernel's prologue can run.
   LAUNCH(c, row_count_kernel, 1, 32, 0, dm, c->st, B);
-  LAUNCH(c, embed_kernel, Rc, 128, 0, dm, c->st, B, c->E, c->xc, c->layers[0][0].g1, c->a_norm, c->ssq, c->ssq_tiles, c->ssq_ld);
+  LAUNCH(c, embed_kernel, Rc, 128, 0, dm, c->st, B, c->E, c->xc, c->layers[0][0].g1, c->a_norm, c->ssq);
+  c->ssq_n = 1;
   run_stack(c, 0, c->xc, nullptr, nullptr, false);
   launch_pdl(c, 1, ring_store_kernel, Rc, 128, 0, dm, c->st, B, 0, (const float*)c->xc, c->hc_ring, d);
   launch_pdl(c, 1, shorten_gather_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->hc_ring, c->a_cat);
@@ -506,15 +516,17 @@ void forward(fm_ctx* c, float* logits_out) {
   gemm(c, c->U_fv, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rf, na + 2, tc::EPI_F32, epi_plain(c->tmp3d, 3 * d));
   launch_pdl(c, 1, ring_store_kernel, Rf, 128, 0, dm, c->st, B, 2, (const float*)c->tmp3d, c->trif_ring, 3 * d);
   launch_pdl(c, 1, upsample_add_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->hv_ring, (const float*)c->trif_ring, c->xv,
-             (const float*)c->layers[3][0].g1, c->a_norm, c->ssq, c->ssq_tiles, c->ssq_ld);
+             (const float*)c->layers[3][0].g1, c->a_norm, c->ssq);
+  c->ssq_n = 1;
   run_stack(c, 3, c->xv, c->zv, nullptr, true);                    // leaves bf16(xv) in a_norm
   gemm(c, c->U_vc, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rv, na + 1, tc::EPI_F32, epi_plain(c->tmp3d, 3 * d));
   launch_pdl(c, 1, ring_store_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->tmp3d, c->triv_ring, 3 * d);
   launch_pdl(c, 1, upsample_add_kernel, Rc, 128, 0, dm, c->st, B, 0, (const float*)c->hc_ring, (const float*)c->triv_ring, c->xc,
-             (const float*)c->layers[4][0].g1, c->a_norm, c->ssq, c->ssq_tiles, c->ssq_ld);
+             (const float*)c->layers[4][0].g1, c->a_norm, c->ssq);
+  c->ssq_n = 1;
   run_stack(c, 4, c->xc, c->zc, c->g_out, true);                   // leaves bf16(xc * g_out) and its sums of squares
   tc::Epi el = epi_plain(c->logits, dm.Vpad);
-  el.ssq_in = c->ssq; el.ssq_tiles = c->ssq_tiles; el.ld_ssq = c->ssq_ld; el.inv_d_in = 1.f / d; el.eps = dm.eps;
+  el.ssq_in = c->ssq; el.ssq_n = c->ssq_n; el.ld_ssq = c->ssq_ld; el.inv_d_in = 1.f / d; el.eps = dm.eps;
   gemm(c, c->W_out, dm.Vpad, 0, c->a_norm, Rc_alloc, 0, dm.V, d, Rc, na, tc::EPI_F32, el);
   launch_pdl(c, 1, verify_top2_kernel, Rc, 256, 0, dm, c->st, B, (const float*)c->logits, logits_out);
 }
@@ -716,20 +728,21 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
   for (int s = 0; s < 5; ++s)
     for (auto& L : c->layers[s]) {
       const uint64_t rows = (uint64_t)dm.max_batch * dm.Hkv * (dm.P + dm.cap[STACK_LEVEL[s]]);
-      L.tmK = add_tmap_bf16(c, L.K, rows, dm.dh, 64);
-      c->tmap_keys.push_back({L.K, rows, (uint64_t)dm.dh, 64u});
-      L.tmV = add_tmap_bf16(c, L.V, rows, dm.dh, 64);
-      c->tmap_keys.push_back({L.V, rows, (uint64_t)dm.dh, 64u});
+      const uint32_t box = (uint32_t)c->attn_chunk;
+      L.tmK = add_tmap_bf16(c, L.K, rows, dm.dh, box);
+      c->tmap_keys.push_back({L.K, rows, (uint64_t)dm.dh, box});
+      L.tmV = add_tmap_bf16(c, L.V, rows, dm.dh, box);
+      c->tmap_keys.push_back({L.V, rows, (uint64_t)dm.dh, box});
       if (L.tmK < 0 || L.tmV < 0) { delete c; return FM_ERR_CUDA; }
     }
   TRYCUDA(cudaMemcpy(c->tmaps, c->tmaps_host.data(), c->tmaps_host.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice));
-  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(256)));
-  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(256)));
-  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_GELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(256)));
-  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(256)));
-  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(256)));
-  TRYCUDA(cudaFuncSetAttribute(attn_split_kernel<64, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<64, 256>::BYTES));
-  TRYCUDA(cudaFuncSetAttribute(attn_split_kernel<128, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<128, 128>::BYTES));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(tc::MAX_N, tc::pick_stages(tc::MAX_N))));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(tc::MAX_N, tc::pick_stages(tc::MAX_N))));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_GELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(tc::MAX_N, tc::pick_stages(tc::MAX_N))));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(tc::MAX_N, tc::pick_stages(tc::MAX_N))));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(tc::MAX_N, tc::pick_stages(tc::MAX_N))));
+  TRYCUDA(cudaFuncSetAttribute(attn_stream_kernel<64, 128, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<64, 128, 8>::BYTES));
+  TRYCUDA(cudaFuncSetAttribute(attn_stream_kernel<128, 64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<128, 64, 4>::BYTES));
   std::vector<double> freq(dm.dh / 2);
   for (int i = 0; i < dm.dh / 2; ++i)
     freq[i] = dm.theta != 0.f ? pow((double)dm.theta, -2.0 * (double)i / (double)dm.dh) : 0.0;

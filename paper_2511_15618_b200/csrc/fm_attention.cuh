@@ -1,14 +1,22 @@
 // Few-row causal attention over one level's KV cache (Sec. 3.3: the candidates of a pass are
 // masked causally among themselves; conditioning enters as prefix keys visible to every row).
 //
-// Split-KV design: one CTA per (sequence, kv-head, chunk of C cache slots).  The chunk's K and V
-// tiles are staged in shared memory by TMA (2-D tensor maps over the cache, 128-byte swizzle);
-// all query rows of the sequence that share the kv-head (rows of the pass x heads of the group)
-// form the M axis of warp-level bf16 MMAs, so the cache is read once per pass, not once per row.
-// Each warp owns a fixed quarter of the chunk's slots; softmax statistics are reduced with quad
-// shuffles; the four warps and then the chunks are merged in a fixed order, so a row's result
-// does not depend on how many other rows or sequences the launch holds.  The CTA that finishes
-// last for a (sequence, kv-head) merges the chunk partials (ticket counter, no waiting).
+// Streaming split-KV design.  The cache of a (sequence, kv-head) is cut into chunks of C slots and
+// the chunks into groups of G consecutive chunks (G is fixed per level when the context is
+// created).  One CTA streams one group: a producer warp brings the K and V tiles of its chunks in
+// with TMA (2-D tensor maps over the cache, 128-byte swizzle) through a ring of shared-memory
+// stages; NW compute warps each own a fixed 16-slot slice of every chunk and keep their own
+// running softmax state (max, sum, output) across the group's chunks, so warps never wait for one
+// another while streaming.  All query rows of the sequence that share the kv-head (rows of the
+// pass x heads of the group, 16 per CTA) form the M axis of warp-level bf16 MMAs, so the cache is
+// read once per pass, not once per row; softmax statistics are reduced with quad shuffles.
+// At the end of the group the warps' states are merged in warp order, and the groups are merged
+// in group order by the CTA that finishes last (ticket counter, nobody waits).  Slices, chunks
+// and groups are fixed by slot index, so a row's result does not depend on how many other rows or
+// sequences the launch holds, nor on the cache length at the time it is computed.
+// Programmatic dependent launch: cache entries written by earlier passes do not depend on the
+// previous kernel, so chunks that hold none of this pass's new slots are requested before
+// griddepcontrol.wait.
 #pragma once
 #include "fm_common.cuh"
 #include "fm_ptx.cuh"
@@ -18,99 +26,117 @@ struct AttnArgs {
   SeqState st;
   int batch, level;
   const bf16* q;              // [rows, H*dh] bf16, rotated and scaled by log2(e)/sqrt(dh)
-  const CUtensorMap* tmK;     // cache as 2-D [B*Hkv*slots, dh], box 64 x 64
+  const CUtensorMap* tmK;     // cache as 2-D [B*Hkv*slots, dh], box C x 64
   const CUtensorMap* tmV;
-  float* part;                // [B*Hkv, max_chunks, MROWS, dh + 2]
-  int* ticket;                // [B*Hkv], zero between launches
+  float* part;                // [B*Hkv*MT, max_groups, 16, dh + 2]
+  int* ticket;                // [B*Hkv*MT], zero between launches
   bf16* out;                  // [rows, H*dh]
-  int max_chunks, mrows;      // mrows = rows_per_seq * group rounded up to 16
+  int G;                      // chunks per group
+  int max_groups;             // groups the cache of this level can hold
+  int MT;                     // 16-row query tiles per (sequence, kv-head)
 };
 
-template <int DH, int C>
-struct AttnSmem {
+template <int DH, int C, int NW>
+struct AttnCfg {
+  static_assert(C == 16 * NW, "every compute warp owns 16 slots of a chunk");
+  static constexpr int STAGES = 4;
   static constexpr int HALVES = DH / 64;
-  static constexpr int TILE = HALVES * C * 128;            // bytes of one K (or V) tile
-  static constexpr int PART = 4 * 16 * (DH + 2) * 4;       // per-warp partials of one m-tile
-  static constexpr int BYTES = 2 * TILE + PART + 64 + 1024; // + barrier + alignment slack
+  static constexpr int TILE = C * DH * 2;                   // bytes of one K (or V) tile
+  static constexpr int STAGE = 2 * TILE;
+  static constexpr int RING = STAGES * STAGE;
+  static constexpr int MERGE = NW * 16 * (DH + 2) * 4;      // the warps' states, aliasing the ring
+  static constexpr int BYTES = (RING > MERGE ? RING : MERGE) + 128 + 1024;   // + barriers + alignment slack
+  static constexpr int THREADS = (NW + 1) * 32;
 };
 
-// position currently held by cache slot `slot` (-1: prefix entry, -2: nothing usable)
-__device__ inline int attn_slot_pos(int slot, int P, int cap, int p_max) {
-  if (slot < P) return -1;
-  const int r = slot - P;
-  if (r >= cap || r > p_max) return -2;
-  return r + ((p_max - r) / cap) * cap;
-}
-
-template <int DH, int C>
-__global__ void __launch_bounds__(128) attn_split_kernel(const AttnArgs a) {
-  using SM = AttnSmem<DH, C>;
-  constexpr int NT = C / 4 / 8;                 // 8-key n-tiles per warp
+template <int DH, int C, int NW>
+__global__ void __launch_bounds__((NW + 1) * 32) attn_stream_kernel(const AttnArgs a) {
+  using CF = AttnCfg<DH, C, NW>;
   constexpr int KS = DH / 16;                   // k-steps of Q K^T
   const Dims& dm = a.dm;
-  const int chunk = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
+  const int u = blockIdx.x / a.MT, mt = blockIdx.x - u * a.MT;
+  const int hk = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t4 = lane & 3;
   ptx::grid_dep_launch();
-  ptx::grid_dep_wait();                            // queries and the new keys/values come from the previous kernel
-  if (b >= a.batch) return;
-  const int n = a.st.nrow[b];
-  if (n <= 0) return;
-  const int Lb = a.st.L[b], ratio = fm_ratio(a.level);
+  // ---- what this CTA has to do (per-pass state is final before the pass's first kernel starts)
+  const int n = b < a.batch ? a.st.nrow[b] : 0;
+  const int Lb = b < a.batch ? a.st.L[b] : 0, ratio = fm_ratio(a.level);
   const int p0 = (Lb + ratio - 1) / ratio;
-  const int nq = (Lb + n - 1) / ratio - p0 + 1;
-  if (nq <= 0) return;
+  const int nq = n > 0 ? (Lb + n - 1) / ratio - p0 + 1 : 0;
   const int p_max = p0 + nq - 1;
   const int P = dm.P, cap = dm.cap[a.level], W = dm.window[a.level];
   const int slots = P + cap;
   const int used = P + min(cap, p_max + 1);
   const int n_chunks = (used + C - 1) / C;
-  if (chunk >= n_chunks) return;
+  const int n_groups = (n_chunks + a.G - 1) / a.G;
   const int group = dm.H / dm.Hkv;
   const int M = nq * group;
+  if (nq <= 0 || u >= n_groups || mt * 16 >= M) {
+    ptx::grid_dep_wait();                          // keep the launch chain ordered
+    return;
+  }
+  const int c_lo = u * a.G, n_my = min(a.G, n_chunks - c_lo);
   const int m_rows = fm_rows_per_seq(dm, a.level);
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  unsigned char* Ks = sm;
-  unsigned char* Vs = sm + SM::TILE;
-  float* pw = reinterpret_cast<float*>(sm + 2 * SM::TILE);            // [4][16][DH+2]
-  uint64_t* bar = reinterpret_cast<uint64_t*>(sm + 2 * SM::TILE + SM::PART);
-  __shared__ int s_last;
+  uint64_t* full = reinterpret_cast<uint64_t*>(sm + (CF::RING > CF::MERGE ? CF::RING : CF::MERGE));
+  uint64_t* empty = full + CF::STAGES;
+  __shared__ int s_last, s_fail;
 
   if (threadIdx.x == 0) {
-    ptx::mbar_init(bar, 1);
+    s_fail = 0;
+    for (int i = 0; i < CF::STAGES; ++i) { ptx::mbar_init(full + i, 1); ptx::mbar_init(empty + i, NW); }
     ptx::fence_mbar_init();
+    ptx::prefetch_tmap(a.tmK);
+    ptx::prefetch_tmap(a.tmV);
   }
   __syncthreads();
-  if (threadIdx.x == 0) {
-    ptx::mbar_expect_tx(bar, 2 * SM::TILE);
-    const int row0 = (b * dm.Hkv + hk) * slots + chunk * C;
+
+  // running state of this warp's slices: rows g and g+8 of the query tile
+  float o[DH / 8][4];
+  float mrun[2] = {-INFINITY, -INFINITY}, lrun[2] = {0.f, 0.f};
 #pragma unroll
-    for (int h = 0; h < SM::HALVES; ++h)
+  for (int i = 0; i < DH / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+
+  if (warp == NW) {
+    // ---- producer
+    if (lane == 0) {
+      const int row_base = (b * dm.Hkv + hk) * slots;
+      // slots written by this pass: P + (p mod cap), p = p0..p_max (at most a handful)
+      auto has_new = [&](int c) {
+        for (int p = p0; p <= p_max; ++p) {
+          const int s = P + p % cap;
+          if (s >= c * C && s < (c + 1) * C) return true;
+        }
+        return false;
+      };
+      auto issue = [&](int i) {
+        const int st = i % CF::STAGES;
+        unsigned char* Ks = sm + st * CF::STAGE;
+        unsigned char* Vs = Ks + CF::TILE;
+        ptx::mbar_expect_tx(full + st, CF::STAGE);
+        const int row0 = row_base + (c_lo + i) * C;
 #pragma unroll
-      for (int kb = 0; kb < C / 64; ++kb) {
-        ptx::tma_load_2d(Ks + (h * C + kb * 64) * 128, a.tmK, h * 64, row0 + kb * 64, bar);
-        ptx::tma_load_2d(Vs + (h * C + kb * 64) * 128, a.tmV, h * 64, row0 + kb * 64, bar);
+        for (int h = 0; h < CF::HALVES; ++h) {
+          ptx::tma_load_2d(Ks + h * C * 128, a.tmK, h * 64, row0, full + st);
+          ptx::tma_load_2d(Vs + h * C * 128, a.tmV, h * 64, row0, full + st);
+        }
+      };
+      int i = 0;
+      const int pre = n_my < CF::STAGES ? n_my : CF::STAGES;
+      while (i < pre && !has_new(c_lo + i)) { issue(i); ++i; }      // old entries only: before the wait
+      ptx::grid_dep_wait();
+      for (; i < n_my; ++i) {
+        if (i >= CF::STAGES && !ptx::mbar_wait(empty + i % CF::STAGES, ((i / CF::STAGES) - 1) & 1)) { s_fail = 1; break; }
+        issue(i);
       }
-  }
-  // positions held by this thread's key columns: n-tile nt, element e -> key warp*C/4 + nt*8 + 2*t4 + e
-  int kpos[NT][2];
-#pragma unroll
-  for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-    for (int e = 0; e < 2; ++e)
-      kpos[nt][e] = attn_slot_pos(chunk * C + warp * (C / 4) + nt * 8 + 2 * t4 + e, P, cap, p_max);
-
-  const bool ready = ptx::mbar_wait(bar, 0);
-  if (!ready) {                                    // never expected; leave without touching the tiles
-    if (threadIdx.x == 0) atomicExch(a.st.status, -5);
-    return;
-  }
-  const uint32_t Ks_u = ptx::smem_u32(Ks), Vs_u = ptx::smem_u32(Vs);
-  float* gpart = a.part + ((size_t)(b * dm.Hkv + hk) * a.max_chunks + chunk) * a.mrows * (DH + 2);
-
-  for (int mt = 0; mt * 16 < M; ++mt) {
-    // ---- Q fragments of this m-tile (rows idx = mt*16 + g, +8; idx = r*group + gh)
+    }
+    __syncwarp();
+  } else {
+    // ---- compute warps
+    ptx::grid_dep_wait();                          // queries come from the previous kernel
+    // Q fragments of this CTA's query tile (rows idx = mt*16 + g, +8; idx = r*group + gh)
     uint32_t qa[KS][4];
     int prow[2];
 #pragma unroll
@@ -126,75 +152,102 @@ __global__ void __launch_bounds__(128) attn_split_kernel(const AttnArgs a) {
         qa[ks][2 + hrow] = ok ? *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8 + 2 * t4) : 0u;
       }
     }
-    // ---- S = Q K^T over this warp's C/4 keys
-    float s[NT][4];
+    // slot -> position: behind the prefix, slot P + r holds position r + k*cap with
+    // k = floor((p_max - r) / cap) = wrap_q if r <= wrap_r else wrap_q - 1
+    const int wrap_q = p_max / cap, wrap_r = p_max - wrap_q * cap;
+    for (int i = 0; i < n_my; ++i) {
+      const int st = i % CF::STAGES;
+      if (!ptx::mbar_wait(full + st, (i / CF::STAGES) & 1)) { s_fail = 1; break; }
+      const uint32_t Ks_u = ptx::smem_u32(sm + st * CF::STAGE), Vs_u = Ks_u + CF::TILE;
+      // positions of this thread's key columns: n-tile nt, element e -> slot base + nt*8 + 2*t4 + e
+      int kpos[2][2];
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+      for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-    for (int ks = 0; ks < KS; ++ks) {
+        for (int e = 0; e < 2; ++e) {
+          const int slot = (c_lo + i) * C + warp * 16 + nt * 8 + 2 * t4 + e;
+          const int r = slot - P;
+          kpos[nt][e] = slot < P ? -1 : ((r >= cap || r > p_max) ? -2 : r + (r <= wrap_r ? wrap_q : wrap_q - 1) * cap);
+        }
+      // ---- S = Q K^T over this warp's 16 slots
+      float s[2][4];
+      s[0][0] = s[0][1] = s[0][2] = s[0][3] = s[1][0] = s[1][1] = s[1][2] = s[1][3] = 0.f;
 #pragma unroll
-      for (int np = 0; np < NT / 2; ++np) {
-        const int key = warp * (C / 4) + np * 16 + (lane & 7) + (lane >> 4) * 8;
+      for (int ks = 0; ks < KS; ++ks) {
+        const int key = warp * 16 + (lane & 7) + (lane >> 4) * 8;
         const int ch = ks * 2 + ((lane >> 3) & 1);
         uint32_t r0, r1, r2, r3;
         ptx::ldmatrix_x4(r0, r1, r2, r3, Ks_u + (ch >> 3) * C * 128 + ptx::swz128(key, ch & 7));
-        ptx::mma_bf16_16816(s[2 * np], qa[ks], r0, r1);
-        ptx::mma_bf16_16816(s[2 * np + 1], qa[ks], r2, r3);
+        ptx::mma_bf16_16816(s[0], qa[ks], r0, r1);
+        ptx::mma_bf16_16816(s[1], qa[ks], r2, r3);
       }
-    }
-    // ---- mask, row max, exponentials, row sums (rows g and g+8; quad = the 4 lanes sharing g)
-    float mx[2] = {-INFINITY, -INFINITY};
+      // ---- mask, running max, exponentials, running sums (rows g and g+8; quad = the 4 lanes sharing g)
+      float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
+      for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int kp = kpos[nt][e & 1], pr = prow[e >> 1];
-        const bool vis = kp == -1 || (kp >= 0 && kp <= pr && (W == 0 || kp >= pr - W + 1));
-        s[nt][e] = (vis && pr >= 0) ? s[nt][e] : -INFINITY;
-        mx[e >> 1] = fmaxf(mx[e >> 1], s[nt][e]);
+        for (int e = 0; e < 4; ++e) {
+          const int kp = kpos[nt][e & 1], pr = prow[e >> 1];
+          const bool vis = kp == -1 || (kp >= 0 && kp <= pr && (W == 0 || kp >= pr - W + 1));
+          s[nt][e] = (vis && pr >= 0) ? s[nt][e] : -INFINITY;
+          mx[e >> 1] = fmaxf(mx[e >> 1], s[nt][e]);
+        }
+      float scale[2], base[2];
+#pragma unroll
+      for (int hrow = 0; hrow < 2; ++hrow) {
+        mx[hrow] = fmaxf(mx[hrow], __shfl_xor_sync(0xffffffffu, mx[hrow], 1));
+        mx[hrow] = fmaxf(mx[hrow], __shfl_xor_sync(0xffffffffu, mx[hrow], 2));
+        const float mnew = fmaxf(mrun[hrow], mx[hrow]);
+        base[hrow] = mnew == -INFINITY ? 0.f : mnew;
+        scale[hrow] = exp2f(mrun[hrow] - base[hrow]);          // 0 while nothing was visible yet
+        mrun[hrow] = mnew;
+      }
+      float ls[2] = {0.f, 0.f};
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          s[nt][e] = exp2f(s[nt][e] - base[e >> 1]);
+          ls[e >> 1] += s[nt][e];
+        }
+#pragma unroll
+      for (int hrow = 0; hrow < 2; ++hrow) {
+        ls[hrow] += __shfl_xor_sync(0xffffffffu, ls[hrow], 1);
+        ls[hrow] += __shfl_xor_sync(0xffffffffu, ls[hrow], 2);
+        lrun[hrow] = lrun[hrow] * scale[hrow] + ls[hrow];
       }
 #pragma unroll
-    for (int hrow = 0; hrow < 2; ++hrow) {
-      mx[hrow] = fmaxf(mx[hrow], __shfl_xor_sync(0xffffffffu, mx[hrow], 1));
-      mx[hrow] = fmaxf(mx[hrow], __shfl_xor_sync(0xffffffffu, mx[hrow], 2));
-    }
-    const float base[2] = {mx[0] == -INFINITY ? 0.f : mx[0], mx[1] == -INFINITY ? 0.f : mx[1]};
-    float ls[2] = {0.f, 0.f};
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        s[nt][e] = exp2f(s[nt][e] - base[e >> 1]);
-        ls[e >> 1] += s[nt][e];
+      for (int i2 = 0; i2 < DH / 8; ++i2) {
+        o[i2][0] *= scale[0]; o[i2][1] *= scale[0];
+        o[i2][2] *= scale[1]; o[i2][3] *= scale[1];
       }
-#pragma unroll
-    for (int hrow = 0; hrow < 2; ++hrow) {
-      ls[hrow] += __shfl_xor_sync(0xffffffffu, ls[hrow], 1);
-      ls[hrow] += __shfl_xor_sync(0xffffffffu, ls[hrow], 2);
-    }
-    // ---- O = P V
-    float o[DH / 8][4];
-#pragma unroll
-    for (int i = 0; i < DH / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
-#pragma unroll
-    for (int kk = 0; kk < NT / 2; ++kk) {
+      // ---- O += P V
       uint32_t pa[4];
-      pa[0] = ptx::pack_bf16(s[2 * kk][0], s[2 * kk][1]);
-      pa[1] = ptx::pack_bf16(s[2 * kk][2], s[2 * kk][3]);
-      pa[2] = ptx::pack_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1]);
-      pa[3] = ptx::pack_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+      pa[0] = ptx::pack_bf16(s[0][0], s[0][1]);
+      pa[1] = ptx::pack_bf16(s[0][2], s[0][3]);
+      pa[2] = ptx::pack_bf16(s[1][0], s[1][1]);
+      pa[3] = ptx::pack_bf16(s[1][2], s[1][3]);
 #pragma unroll
       for (int dp = 0; dp < DH / 16; ++dp) {
-        const int key = warp * (C / 4) + kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+        const int key = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
         const int ch = dp * 2 + (lane >> 4);
         uint32_t r0, r1, r2, r3;
         ptx::ldmatrix_x4_trans(r0, r1, r2, r3, Vs_u + (ch >> 3) * C * 128 + ptx::swz128(key, ch & 7));
         ptx::mma_bf16_16816(o[2 * dp], pa, r0, r1);
         ptx::mma_bf16_16816(o[2 * dp + 1], pa, r2, r3);
       }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(empty + st);           // this warp is done with the stage
     }
-    // ---- the four warps' partials -> shared, merged in warp order -> chunk partial in global
-    __syncthreads();                                // previous m-tile's readers are done with pw
+  }
+  // ---- the warps' states -> shared (the ring is idle once every warp is here), merged in warp order
+  __syncthreads();
+  if (s_fail) {                                              // a bounded wait gave up: report, write nothing
+    if (threadIdx.x == 0) atomicExch(a.st.status, -5);
+    return;
+  }
+  float* pw = reinterpret_cast<float*>(sm);                  // [NW][16][DH+2]
+  if (warp < NW) {
     float* mine = pw + warp * 16 * (DH + 2);
 #pragma unroll
     for (int i = 0; i < DH / 8; ++i) {
@@ -204,73 +257,84 @@ __global__ void __launch_bounds__(128) attn_split_kernel(const AttnArgs a) {
       mine[(g + 8) * (DH + 2) + i * 8 + 2 * t4 + 1] = o[i][3];
     }
     if (t4 == 0) {
-      mine[g * (DH + 2) + DH] = mx[0]; mine[g * (DH + 2) + DH + 1] = ls[0];
-      mine[(g + 8) * (DH + 2) + DH] = mx[1]; mine[(g + 8) * (DH + 2) + DH + 1] = ls[1];
-    }
-    __syncthreads();
-    for (int e = threadIdx.x; e < 16 * (DH + 2); e += 128) {
-      const int i = e / (DH + 2), c = e - i * (DH + 2);
-      if (mt * 16 + i >= M) continue;
-      float mm = -INFINITY;
-#pragma unroll
-      for (int w = 0; w < 4; ++w) mm = fmaxf(mm, pw[(w * 16 + i) * (DH + 2) + DH]);
-      float v;
-      if (c == DH) v = mm;
-      else {
-        v = 0.f;
-#pragma unroll
-        for (int w = 0; w < 4; ++w) {
-          const float mw = pw[(w * 16 + i) * (DH + 2) + DH];
-          const float sc = mw == -INFINITY ? 0.f : exp2f(mw - mm);
-          v += sc * pw[(w * 16 + i) * (DH + 2) + (c == DH + 1 ? DH + 1 : c)];
-        }
-      }
-      gpart[(size_t)(mt * 16 + i) * (DH + 2) + c] = v;
+      mine[g * (DH + 2) + DH] = mrun[0]; mine[g * (DH + 2) + DH + 1] = lrun[0];
+      mine[(g + 8) * (DH + 2) + DH] = mrun[1]; mine[(g + 8) * (DH + 2) + DH + 1] = lrun[1];
     }
   }
+  __syncthreads();
+  const size_t pt = ((size_t)(b * dm.Hkv + hk) * a.MT + mt);
+  float* gpart = a.part + (pt * a.max_groups + u) * 16 * (DH + 2);
+  const bool single = n_groups == 1;
+  for (int e = threadIdx.x; e < 16 * (DH + 2); e += CF::THREADS) {
+    const int i = e / (DH + 2), c = e - i * (DH + 2);
+    const int idx = mt * 16 + i;
+    if (idx >= M) continue;
+    float mm = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) mm = fmaxf(mm, pw[(w * 16 + i) * (DH + 2) + DH]);
+    float v = 0.f, l = 0.f;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) {
+      const float mw = pw[(w * 16 + i) * (DH + 2) + DH];
+      const float sc = mw == -INFINITY ? 0.f : exp2f(mw - mm);
+      v += sc * pw[(w * 16 + i) * (DH + 2) + (c < DH ? c : DH + 1)];
+      l += sc * pw[(w * 16 + i) * (DH + 2) + DH + 1];
+    }
+    if (single) {                                            // one group: this is the result
+      if (c < DH) {
+        const int r = idx / group, gh = idx - r * group;
+        a.out[((size_t)(b * m_rows + r) * dm.H + hk * group + gh) * DH + c] = __float2bfloat16(v / l);
+      }
+    } else {
+      gpart[(size_t)i * (DH + 2) + c] = c == DH ? mm : v;    // c == DH+1 carries the merged sum
+    }
+  }
+  if (single) return;
 
-  // ---- ticket: the CTA that arrives last for this (sequence, kv-head) merges all chunk partials
+  // ---- ticket: the CTA that arrives last for this (sequence, kv-head, query tile) merges the groups
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) {
-    const int t = atomicAdd(a.ticket + b * dm.Hkv + hk, 1);
-    s_last = (t == n_chunks - 1) ? 1 : 0;
+    const int t = atomicAdd(a.ticket + pt, 1);
+    s_last = (t == n_groups - 1) ? 1 : 0;
   }
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  const float* base = a.part + (size_t)(b * dm.Hkv + hk) * a.max_chunks * a.mrows * (DH + 2);
-  const size_t cstride = (size_t)a.mrows * (DH + 2);
-  for (int e = threadIdx.x; e < M * DH; e += 128) {
-    const int idx = e / DH, c = e - idx * DH;
-    const float* pr = base + (size_t)idx * (DH + 2);
+  const float* base = a.part + pt * a.max_groups * 16 * (DH + 2);
+  constexpr size_t gstride = (size_t)16 * (DH + 2);
+  const int rows_here = min(16, M - mt * 16);
+  for (int e = threadIdx.x; e < rows_here * DH; e += CF::THREADS) {
+    const int i = e / DH, c = e - i * DH;
+    const float* pr = base + (size_t)i * (DH + 2);
     float mm = -INFINITY;
-    for (int ck = 0; ck < n_chunks; ++ck) mm = fmaxf(mm, __ldcg(pr + ck * cstride + DH));
+    for (int ck = 0; ck < n_groups; ++ck) mm = fmaxf(mm, __ldcg(pr + ck * gstride + DH));
     float acc = 0.f, lsum = 0.f;
     int ck = 0;
-    for (; ck + 4 <= n_chunks; ck += 4) {          // loads first, then the sums in chunk order
+    for (; ck + 4 <= n_groups; ck += 4) {          // loads first, then the sums in group order
       float m4[4], l4[4], v4[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const float* q = pr + (ck + u) * cstride;
-        m4[u] = __ldcg(q + DH); l4[u] = __ldcg(q + DH + 1); v4[u] = __ldcg(q + c);
+      for (int x = 0; x < 4; ++x) {
+        const float* q = pr + (ck + x) * gstride;
+        m4[x] = __ldcg(q + DH); l4[x] = __ldcg(q + DH + 1); v4[x] = __ldcg(q + c);
       }
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const float sc = m4[u] == -INFINITY ? 0.f : exp2f(m4[u] - mm);
-        acc += sc * v4[u];
-        lsum += sc * l4[u];
+      for (int x = 0; x < 4; ++x) {
+        const float sc = m4[x] == -INFINITY ? 0.f : exp2f(m4[x] - mm);
+        acc += sc * v4[x];
+        lsum += sc * l4[x];
       }
     }
-    for (; ck < n_chunks; ++ck) {
-      const float* q = pr + ck * cstride;
+    for (; ck < n_groups; ++ck) {
+      const float* q = pr + ck * gstride;
       const float mc = __ldcg(q + DH);
       const float sc = mc == -INFINITY ? 0.f : exp2f(mc - mm);
       acc += sc * __ldcg(q + c);
       lsum += sc * __ldcg(q + DH + 1);
     }
+    const int idx = mt * 16 + i;
     const int r = idx / group, gh = idx - r * group;
     a.out[((size_t)(b * m_rows + r) * dm.H + hk * group + gh) * DH + c] = __float2bfloat16(acc / lsum);
   }
-  if (threadIdx.x == 0) a.ticket[b * dm.Hkv + hk] = 0;
+  if (threadIdx.x == 0) a.ticket[pt] = 0;
 }

@@ -9,11 +9,12 @@
 // brought in by TMA with the 128-byte swizzle into a ring of shared-memory stages; one thread
 // issues the MMAs, accumulators live in tensor memory and are read back with tcgen05.ld.
 // The work is bandwidth bound: the grid is (M/128 tiles) x (S splits of K) so that many SMs
-// stream weights.  The S CTAs of one M tile form a thread-block cluster: each puts its partial
-// tile in its own shared memory, and after a cluster barrier every CTA adds, in rank order (a
-// fixed order, so a row's result does not depend on how many rows the launch holds), the S
-// partials of its share of the tile's columns through distributed shared memory and applies the
-// epilogue of the projection: RMSNorm scale of the operand rows, then one of
+// stream weights.  The S CTAs of one M tile form a thread-block cluster: every CTA owns 1/S of the
+// tile's columns; each CTA sends the columns of its partial tile to their owners' shared memory
+// with asynchronous distributed-shared-memory stores that count their bytes on an mbarrier of the
+// owner, so an owner continues as soon as its own S partials are in, adds them in rank order (a
+// fixed order, so a row's result does not depend on how many rows the launch holds) and applies
+// the epilogue of the projection: RMSNorm scale of the operand rows, then one of
 //   EPI_F32 / EPI_BF16   plain store,
 //   EPI_GELU             bf16(gelu(y))                      (first FFN matrix),
 //   EPI_RESID            x (+)= y; next operand bf16(x * gain); per-tile sums of squares
@@ -29,17 +30,19 @@ namespace tc {
 
 constexpr int BM = 128;          // output features per CTA
 constexpr int BK = 64;           // K elements per slab (128 bytes of bf16)
-constexpr int STAGES = 4;
+constexpr int MAX_STAGES = 8;
 constexpr int MAX_SPLIT = 8;     // portable cluster size
+constexpr int MAX_N = 240;       // token rows per launch: two stages + the receive buffer must fit in 227 KB
 
 enum EpiMode { EPI_F32 = 0, EPI_BF16 = 1, EPI_GELU = 2, EPI_RESID = 3, EPI_QKV = 4 };
 
 struct Args {
   const CUtensorMap* tmW;        // [Mpad, K] bf16, box 128 x 64
   const CUtensorMap* tmA;        // [rows, K] bf16, box N x 64
-  int M, K, N;                   // N = padded rows in the box (multiple of 16, <= 256)
+  int M, K, N;                   // N = padded rows in the box (multiple of 16, <= MAX_N)
   int n_store;                   // rows actually stored (<= N)
   int split;                     // K splits = gridDim.y = cluster size (1, 2, 4 or 8)
+  int stages;                    // depth of the shared-memory ring (2..MAX_STAGES)
   int w_row0, a_row0;            // row offsets into the tensor maps (stacked weights / row groups)
   const int* n_active;           // skip when *n_active == 0 (may be null); must not change during a pass
   int* status;
@@ -47,14 +50,14 @@ struct Args {
 
 struct Epi {
   int row0;                      // first output row of this launch (N tiles beyond the first)
-  const float* ssq_in;           // [ssq_tiles][ld_ssq] sums of squares of the operand rows; null = no scale
-  int ssq_tiles, ld_ssq;
+  const float* ssq_in;           // [ssq_n][ld_ssq] partial sums of squares of the operand rows; null = no scale
+  int ssq_n, ld_ssq;
   float inv_d_in, eps;
   void* out; int ldo;            // EPI_F32 / EPI_BF16 / EPI_GELU
   float* x; int ldx; int add;    // EPI_RESID: residual stream, add = 0 replaces it
   const float* gain;             //            gain of the next norm (null = 1)
   bf16* a_out; int lda;          //            next GEMM's operand rows (may be null)
-  float* ssq_out; int ld_ssq_out;//            [M tiles][ld] sums of squares of the new x rows (may be null)
+  float* ssq_out; int ld_ssq_out;//            [M tiles * split][ld] partial sums of squares of the new x rows (may be null)
   Dims dm; SeqState st;          // EPI_QKV
   int batch, level;
   const float2* rope_tab;
@@ -96,7 +99,7 @@ __device__ inline void ld16(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-// ---- thread-block cluster: rank, barrier, loads from a peer CTA's shared memory
+// ---- thread-block cluster: rank, barrier, stores into a peer CTA's shared memory
 __device__ inline uint32_t cluster_rank() {
   uint32_t r;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -105,17 +108,46 @@ __device__ inline uint32_t cluster_rank() {
 __device__ inline void cluster_sync() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ inline float ld_peer(uint32_t local_addr, uint32_t rank) {
+// 4-byte store into a peer CTA's shared memory that reports its bytes to an mbarrier of that CTA
+__device__ inline void st_async_peer(uint32_t remote_addr, float a, uint32_t remote_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(remote_addr), "r"(__float_as_uint(a)),
+               "r"(remote_bar)
+               : "memory");
+}
+__device__ inline bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(ptx::smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ inline bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, long long limit_cycles = 200000000ll) {
+  if (mbar_try_wait_cluster(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait_cluster(bar, parity))
+    if (clock64() - t0 > limit_cycles) return false;
+  return true;
+}
+__device__ inline uint32_t map_peer(uint32_t local_addr, uint32_t rank) {
   uint32_t ra;
-  float v;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
-  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(ra));
-  return v;
+  return ra;
 }
 
-// The stage ring is reused for the partial tile [N][128] fp32 (N * 512 bytes) and, behind it, for
-// the squares of EPI_RESID ([N][64 / split] fp32 <= 64 KB): STAGES * 16 KB + N * 512 >= both.
-inline int smem_bytes(int N) { return STAGES * (BM * 128 + ((N * 128 + 1023) / 1024) * 1024) + 1024 + 256; }
+// Shared memory: ring of `stages` x ([128 x 64] weight slab + [N x 64] operand slab), then the
+// receive buffer of the cluster reduction [split][N][64/split][2] fp32 = N * 512 bytes (peers write
+// into it while this CTA may still be multiplying, so it never aliases the ring), then barriers.
+inline int stage_bytes(int N) { return BM * 128 + ((N * 128 + 1023) / 1024) * 1024; }
+inline int pick_stages(int N) {
+  int st = (200 * 1024 - N * 512) / stage_bytes(N);
+  st = st > 4 ? 4 : st;
+  return st < 2 ? 2 : st;
+}
+inline int smem_bytes(int N, int stages) { return stages * stage_bytes(N) + N * 512 + 1024 + 256; }
 
 __device__ inline float gelu_erf_f(float x) { return 0.5f * x * (1.f + erff(x * 0.70710678118654752f)); }
 
@@ -138,14 +170,17 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   }
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int STAGES = g.stages;
   const int b_bytes = ((g.N * 128 + 1023) / 1024) * 1024;
   const int stage_bytes = BM * 128 + b_bytes;
-  uint64_t* full = reinterpret_cast<uint64_t*>(sm + STAGES * stage_bytes);
-  uint64_t* empty = full + STAGES;
-  uint64_t* accum = empty + STAGES;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
+  float* recv = reinterpret_cast<float*>(sm + STAGES * stage_bytes);          // [S][N][PW][2]
+  uint64_t* full = reinterpret_cast<uint64_t*>(sm + STAGES * stage_bytes + g.N * 512);
+  uint64_t* empty = full + MAX_STAGES;
+  uint64_t* accum = empty + MAX_STAGES;
+  uint64_t* rbar = accum + 1;                                                 // partials of all ranks have arrived
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(rbar + 1);
   __shared__ int s_fail;
-  __shared__ float s_inv[256], s_rowsq[256];
+  __shared__ float s_inv[256];
   __shared__ int s_rb[256], s_rp[256];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -162,7 +197,9 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
     s_fail = 0;
     for (int i = 0; i < STAGES; ++i) { ptx::mbar_init(full + i, 1); ptx::mbar_init(empty + i, 1); }
     ptx::mbar_init(accum, 1);
+    ptx::mbar_init(rbar, 1);
     ptx::fence_mbar_init();
+    ptx::mbar_expect_tx(rbar, (uint32_t)g.n_store * 512u);   // n_store rows x 128/S columns x S ranks x 4 bytes
     ptx::prefetch_tmap(g.tmW);
     ptx::prefetch_tmap(g.tmA);
   }
@@ -178,6 +215,9 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   // This CTA now holds its tensor memory and shared memory: the next kernel may start its own
   // prologue beside us.
   ptx::grid_dep_launch();
+  // Peers will write into this CTA's receive buffer and count on its barrier: make sure every
+  // CTA of the cluster runs and has initialised them.
+  if (S > 1) cluster_sync();
 
   if (warp == 0 && lane == 0) {
     // ---- producer: stream this CTA's K range through the stage ring.  The weight slabs of the
@@ -214,37 +254,96 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
     }
     commit(accum);                                         // accumulator complete
   }
-  __syncwarp();
-  ptx::grid_dep_wait();                                    // everything below touches activations
-
-  // ---- operand-row scales and row maps, while the MMAs drain
-  for (int n = tid; n < g.n_store; n += 128) {
+  else if (warp >= 2) {
+    // ---- warps 2 and 3, while the operands arrive: operand-row scales (the partial sums of
+    // squares of a row are gathered by 8 lanes, each adding its slots in slot order, then combined by
+    // a fixed shuffle tree) and row maps
+    ptx::grid_dep_wait();
+    const int t = tid - 64;
     if (e.ssq_in != nullptr) {
-      float ss = 0.f;
-      for (int t = 0; t < e.ssq_tiles; ++t) ss += __ldcg(e.ssq_in + (size_t)t * e.ld_ssq + e.row0 + n);
-      s_inv[n] = rsqrtf(ss * e.inv_d_in + e.eps);
+      const int sub = t & 7;
+      for (int n0 = 0; n0 < g.n_store; n0 += 8) {
+        const int n = n0 + (t >> 3);
+        float v[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int slot = sub + 8 * k;
+          v[k] = (n < g.n_store && slot < e.ssq_n) ? __ldcg(e.ssq_in + (size_t)slot * e.ld_ssq + e.row0 + n) : 0.f;
+        }
+        float ss = 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) ss += v[k];
+        for (int slot = sub + 64; slot < e.ssq_n; slot += 8)             // more than 64 slots: not expected
+          ss += (n < g.n_store) ? __ldcg(e.ssq_in + (size_t)slot * e.ld_ssq + e.row0 + n) : 0.f;
+        ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+        ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+        ss += __shfl_xor_sync(0xffffffffu, ss, 4);
+        if (sub == 0 && n < g.n_store) s_inv[n] = rsqrtf(ss * e.inv_d_in + e.eps);
+      }
     } else {
-      s_inv[n] = 1.f;
+      for (int n = t; n < g.n_store; n += 64) s_inv[n] = 1.f;
     }
     if (MODE == EPI_QKV) {
-      int b, p;
-      const bool valid = fm_row_map(e.dm, e.st, e.batch, e.level, e.row0 + n, b, p);
-      s_rb[n] = valid ? b : -1;
-      s_rp[n] = p;
+      for (int n = t; n < g.n_store; n += 64) {
+        int b, p;
+        const bool valid = fm_row_map(e.dm, e.st, e.batch, e.level, e.row0 + n, b, p);
+        s_rb[n] = valid ? b : -1;
+        s_rp[n] = p;
+      }
     }
   }
-  // ---- everyone waits for the accumulator; a timeout is recorded and the barriers below are
-  // still executed by every CTA of the cluster
-  bool ok = n_slabs > 0 ? ptx::mbar_wait(accum, 0) : true;
   __syncwarp();
-  fence_after();
-  __syncthreads();
-  if (!ok || s_fail) {
-    ok = false;
-    if (tid == 0) atomicExch(g.status, -5);
+
+  // ---- where this thread's accumulator column goes, and its first item of the epilogue.  Column
+  // m of the tile is half h of pair slot q; slots [r*PW, (r+1)*PW) belong to rank r, which receives
+  // [source rank][row][slot][half].  Everything that does not depend on the previous kernel
+  // (indices, gains, rotary angles) is prepared here, before the wait.
+  const int PW = 64 / S;
+  const bool head128 = MODE == EPI_QKV && e.dm.dh == 128;
+  const int items = g.n_store * PW;
+  uint32_t dst0, dbar;
+  {
+    const int q = head128 ? (tid & 63) : ((tid >> 6) * 32 + (tid & 31));
+    const int h = head128 ? (tid >> 6) : ((tid >> 5) & 1);
+    const int owner = q / PW, cc = q - owner * PW;
+    dst0 = map_peer(ptx::smem_u32(recv + ((size_t)z * g.N * PW + cc) * 2 + h), (uint32_t)owner);
+    dbar = map_peer(ptx::smem_u32(rbar), (uint32_t)owner);
   }
-  // ---- partial tile -> own shared memory (the ring is idle: every stage was consumed)
-  float* part = reinterpret_cast<float*>(sm);              // [n_store][128]
+  float pre_ga = 1.f, pre_gb = 1.f;
+  float2 pre_cs = make_float2(1.f, 0.f);
+  if (tid < items) {
+    const int n = tid / PW, cc = tid - n * PW;
+    int ca, cb;
+    pair_cols(z * PW + cc, head128, ca, cb);
+    const int ma = tile_m * BM + ca, mb = tile_m * BM + cb;
+    if (MODE == EPI_RESID && e.gain != nullptr) {
+      if (ma < g.M) pre_ga = e.gain[ma];
+      if (mb < g.M) pre_gb = e.gain[mb];
+    }
+    if (MODE == EPI_QKV && e.dm.theta != 0.f) {
+      int b, p;
+      const bool valid = fm_row_map(e.dm, e.st, e.batch, e.level, e.row0 + n, b, p);
+      const int head = ma / e.dm.dh, i = ma - head * e.dm.dh;
+      if (valid && ma < g.M && head < e.dm.H + e.dm.Hkv) pre_cs = e.rope_tab[(size_t)p * (e.dm.dh >> 1) + i];
+    }
+  }
+  ptx::grid_dep_wait();                                    // everything below touches activations
+  float pre_xa = 0.f, pre_xb = 0.f;
+  if (MODE == EPI_RESID && e.add && tid < items) {
+    const int n = tid / PW, cc = tid - n * PW;
+    int ca, cb;
+    pair_cols(z * PW + cc, head128, ca, cb);
+    const int ma = tile_m * BM + ca, mb = tile_m * BM + cb;
+    const float* xr = e.x + (size_t)(e.row0 + n) * e.ldx;
+    if (ma < g.M) pre_xa = xr[ma];
+    if (mb < g.M) pre_xb = xr[mb];
+  }
+
+  // ---- every warp waits for the accumulator and sends its 32 columns of the partial tile to
+  // their owners.  A timeout is recorded; zeros are sent so that no owner waits in vain.
+  bool ok = n_slabs > 0 ? ptx::mbar_wait(accum, 0) : true;
+  ok = __all_sync(0xffffffffu, ok);
+  fence_after();
   for (int n0 = 0; n0 < g.n_store; n0 += 16) {
     uint32_t r[16];
     if (ok && n_slabs > 0) ld16(tmem + ((uint32_t)(warp * 32) << 16) + n0, r);
@@ -254,73 +353,81 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
     }
 #pragma unroll
     for (int j = 0; j < 16; ++j)
-      if (n0 + j < g.n_store) part[(n0 + j) * BM + tid] = __uint_as_float(r[j]);
+      if (n0 + j < g.n_store) st_async_peer(dst0 + (uint32_t)((n0 + j) * PW * 8), __uint_as_float(r[j]), dbar);
   }
-  cluster_sync();                                          // partials of all ranks are in place
-
+  __syncthreads();                                         // s_inv / row maps are written
+  const bool arrived = mbar_wait_cluster(rbar, 0);
+  if (!ok || !arrived || s_fail) {
+    if (tid == 0) atomicExch(g.status, -5);
+  }
   // ---- this rank's share of the tile: pair slots [z*PW, (z+1)*PW), all rows
-  const int PW = 64 / S;
-  const int items = g.n_store * PW;
-  const uint32_t part_u = ptx::smem_u32(part);
-  const bool head128 = MODE == EPI_QKV && e.dm.dh == 128;
-  float* sq = reinterpret_cast<float*>(sm + (size_t)g.N * 512);   // [n_store][PW], EPI_RESID only
-  for (int it = tid; it < items; it += 128) {
-    const int n = it / PW, cc = it - n * PW;
+  const int L = PW < 32 ? PW : 32;                         // lanes that share a row
+  for (int it0 = 0; it0 < items; it0 += 128) {
+    const int it = it0 + tid;
+    const bool active = it < items, first = it0 == 0;
+    const int n = active ? it / PW : 0, cc = active ? it - n * PW : 0;
     int ca, cb;
     pair_cols(z * PW + cc, head128, ca, cb);
-    float va[MAX_SPLIT], vb[MAX_SPLIT];
+    float2 v[MAX_SPLIT];
 #pragma unroll
-    for (int r = 0; r < MAX_SPLIT; ++r) {                  // all loads first, then the sums in rank order
-      va[r] = r < S ? ld_peer(part_u + (uint32_t)(n * BM + ca) * 4u, (uint32_t)r) : 0.f;
-      vb[r] = r < S ? ld_peer(part_u + (uint32_t)(n * BM + cb) * 4u, (uint32_t)r) : 0.f;
-    }
+    for (int r = 0; r < MAX_SPLIT; ++r)                    // all loads first, then the sums in rank order
+      v[r] = (r < S && active) ? *reinterpret_cast<const float2*>(recv + (((size_t)r * g.N + n) * PW + cc) * 2) : make_float2(0.f, 0.f);
     float ya = 0.f, yb = 0.f;
 #pragma unroll
     for (int r = 0; r < MAX_SPLIT; ++r)
-      if (r < S) { ya += va[r]; yb += vb[r]; }
+      if (r < S) { ya += v[r].x; yb += v[r].y; }
     const float inv = s_inv[n];
     ya *= inv;
     yb *= inv;
     const int ma = tile_m * BM + ca, mb = tile_m * BM + cb;
+    const bool a_ok = active && ma < g.M, b_ok = active && mb < g.M;
     const size_t row = (size_t)(e.row0 + n);
     if (MODE == EPI_F32) {
       float* o = reinterpret_cast<float*>(e.out) + row * e.ldo;
-      if (ma < g.M) o[ma] = ya;
-      if (mb < g.M) o[mb] = yb;
+      if (a_ok) o[ma] = ya;
+      if (b_ok) o[mb] = yb;
     } else if (MODE == EPI_BF16) {
       bf16* o = reinterpret_cast<bf16*>(e.out) + row * e.ldo;
-      if (ma < g.M) o[ma] = __float2bfloat16(ya);
-      if (mb < g.M) o[mb] = __float2bfloat16(yb);
+      if (a_ok) o[ma] = __float2bfloat16(ya);
+      if (b_ok) o[mb] = __float2bfloat16(yb);
     } else if (MODE == EPI_GELU) {
       bf16* o = reinterpret_cast<bf16*>(e.out) + row * e.ldo;
-      if (ma < g.M) o[ma] = __float2bfloat16(gelu_erf_f(ya));
-      if (mb < g.M) o[mb] = __float2bfloat16(gelu_erf_f(yb));
+      if (a_ok) o[ma] = __float2bfloat16(gelu_erf_f(ya));
+      if (b_ok) o[mb] = __float2bfloat16(gelu_erf_f(yb));
     } else if (MODE == EPI_RESID) {
       float* xr = e.x + row * e.ldx;
       float xa = 0.f, xb = 0.f;
-      if (ma < g.M) {
-        xa = (e.add ? xr[ma] : 0.f) + ya;
+      if (a_ok) {
+        xa = (first ? pre_xa : (e.add ? xr[ma] : 0.f)) + ya;
         xr[ma] = xa;
-        if (e.a_out != nullptr) e.a_out[row * e.lda + ma] = __float2bfloat16(xa * (e.gain != nullptr ? e.gain[ma] : 1.f));
+        if (e.a_out != nullptr) e.a_out[row * e.lda + ma] = __float2bfloat16(xa * (first ? pre_ga : (e.gain != nullptr ? e.gain[ma] : 1.f)));
       }
-      if (mb < g.M) {
-        xb = (e.add ? xr[mb] : 0.f) + yb;
+      if (b_ok) {
+        xb = (first ? pre_xb : (e.add ? xr[mb] : 0.f)) + yb;
         xr[mb] = xb;
-        if (e.a_out != nullptr) e.a_out[row * e.lda + mb] = __float2bfloat16(xb * (e.gain != nullptr ? e.gain[mb] : 1.f));
+        if (e.a_out != nullptr) e.a_out[row * e.lda + mb] = __float2bfloat16(xb * (first ? pre_gb : (e.gain != nullptr ? e.gain[mb] : 1.f)));
       }
-      sq[it] = xa * xa + xb * xb;
+      if (e.ssq_out != nullptr) {
+        // per-row sums of squares of this rank's columns: a fixed shuffle tree over the L lanes that
+        // share the row; the next GEMM adds the (tile, rank, lane group) partials in slot order
+        float sqv = xa * xa + xb * xb;
+        for (int o = L >> 1; o > 0; o >>= 1) sqv += __shfl_xor_sync(0xffffffffu, sqv, o);
+        if (active && (cc & (L - 1)) == 0)
+          e.ssq_out[(size_t)((tile_m * S + z) * (PW / L) + cc / L) * e.ld_ssq_out + e.row0 + n] = sqv;
+      }
     } else {  // EPI_QKV: (ya, yb) is the rotary pair (i, i + dh/2) of one head
       const Dims& dm = e.dm;
       const int dh = dm.dh, half = dh >> 1, H = dm.H, Hkv = dm.Hkv;
       const int head = ma / dh, i = ma - head * dh;
-      if (ma < g.M && head < H + 2 * Hkv) {
+      if (a_ok && head < H + 2 * Hkv) {
         const int b = s_rb[n], p = s_rp[n];
         const bool valid = b >= 0;
         const int slots = dm.P + dm.cap[e.level];
         if (head < H + Hkv) {
-          float c = 1.f, s = 0.f;
-          if (dm.theta != 0.f && valid) { const float2 cs = e.rope_tab[(size_t)p * half + i]; c = cs.x; s = cs.y; }
-          const float y1 = ya * c - yb * s, y2 = yb * c + ya * s;
+          float2 cs = make_float2(1.f, 0.f);
+          if (first) cs = pre_cs;
+          else if (dm.theta != 0.f && valid) cs = e.rope_tab[(size_t)p * half + i];
+          const float y1 = ya * cs.x - yb * cs.y, y2 = yb * cs.x + ya * cs.y;
           if (head < H) {
             bf16* q = e.q_out + (row * H + head) * dh;
             q[i] = __float2bfloat16(valid ? y1 * e.qscale : 0.f);
@@ -338,25 +445,6 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
       }
     }
   }
-  if (MODE == EPI_RESID && e.ssq_out != nullptr) {
-    // per-row sums of squares: this rank's columns in slot order, then the ranks in rank order
-    __syncthreads();
-    for (int n = tid; n < g.n_store; n += 128) {
-      float t = 0.f;
-      for (int cc = 0; cc < PW; ++cc) t += sq[n * PW + cc];
-      s_rowsq[n] = t;
-    }
-    cluster_sync();
-    if (z == 0) {
-      const uint32_t rs_u = ptx::smem_u32(s_rowsq);
-      for (int n = tid; n < g.n_store; n += 128) {
-        float t = 0.f;
-        for (int r = 0; r < S; ++r) t += ld_peer(rs_u + (uint32_t)n * 4u, (uint32_t)r);
-        e.ssq_out[(size_t)tile_m * e.ld_ssq_out + e.row0 + n] = t;
-      }
-    }
-  }
-  cluster_sync();                                          // nobody leaves while a peer may still read its shared memory
   fence_before();
   __syncthreads();
   fence_after();

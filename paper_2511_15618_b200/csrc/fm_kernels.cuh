@@ -20,10 +20,10 @@ __device__ inline float block_sum(float v, float* sh) {
 // ------------------------------------------------------------------------------------------
 // Hand a freshly written residual row to the first layer of a stack: the GEMM operand row
 // bf16(x * g) (the RMSNorm scale 1/rms is applied by the GEMM's epilogue) and the row's sum of
-// squares in tile 0 of `ssq` (the other tiles are zeroed: epilogues add all tiles).
+// squares in slot 0 of `ssq` (the consumer is told that one slot is filled).
 // ------------------------------------------------------------------------------------------
 __device__ inline void stack_entry_row(const float* xr, int row, int d, const float* __restrict__ g,
-                                       bf16* __restrict__ a_out, float* __restrict__ ssq, int ssq_tiles, int ld_ssq) {
+                                       bf16* __restrict__ a_out, float* __restrict__ ssq) {
   __shared__ float sh[32];
   float ss = 0.f;
   for (int i = threadIdx.x; i < d; i += blockDim.x) {
@@ -32,18 +32,14 @@ __device__ inline void stack_entry_row(const float* xr, int row, int d, const fl
     a_out[(size_t)row * d + i] = __float2bfloat16(v * g[i]);
   }
   ss = block_sum(ss, sh);
-  if (threadIdx.x == 0) {
-    ssq[row] = ss;
-    for (int t = 1; t < ssq_tiles; ++t) ssq[(size_t)t * ld_ssq + row] = 0.f;
-  }
+  if (threadIdx.x == 0) ssq[row] = ss;
 }
 
 // ------------------------------------------------------------------------------------------
 // a1. candidate embedding: x[row] = E[cand[b][j]]  (zeros for rows that are not fed)
 // ------------------------------------------------------------------------------------------
 __global__ void embed_kernel(Dims dm, SeqState st, int batch, const bf16* __restrict__ E, float* __restrict__ x,
-                             const float* __restrict__ g, bf16* __restrict__ a_out, float* __restrict__ ssq, int ssq_tiles,
-                             int ld_ssq) {
+                             const float* __restrict__ g, bf16* __restrict__ a_out, float* __restrict__ ssq) {
   const int row = blockIdx.x;
   int b, p;
   const bool valid = fm_row_map(dm, st, batch, 0, row, b, p);
@@ -58,7 +54,7 @@ __global__ void embed_kernel(Dims dm, SeqState st, int batch, const bf16* __rest
   for (int i = threadIdx.x; i < dm.d; i += blockDim.x)
     x[(size_t)row * dm.d + i] = valid ? __bfloat162float(E[(size_t)tok * dm.d + i]) : 0.f;
   __syncthreads();
-  stack_entry_row(x + (size_t)row * dm.d, row, dm.d, g, a_out, ssq, ssq_tiles, ld_ssq);
+  stack_entry_row(x + (size_t)row * dm.d, row, dm.d, g, a_out, ssq);
 }
 
 // RMSNorm of read-only fp32 rows (conditioning vectors, draft features) -> bf16 operand rows
@@ -145,7 +141,7 @@ __global__ void shorten_gather_kernel(Dims dm, SeqState st, int batch, int level
 // then handed to the first layer of the stack above (operand row and sum of squares)
 __global__ void upsample_add_kernel(Dims dm, SeqState st, int batch, int level, const float* __restrict__ h_ring,
                                     const float* __restrict__ tri_ring, float* __restrict__ x, const float* __restrict__ g,
-                                    bf16* __restrict__ a_out, float* __restrict__ ssq, int ssq_tiles, int ld_ssq) {
+                                    bf16* __restrict__ a_out, float* __restrict__ ssq) {
   ptx::grid_dep_launch();
   ptx::grid_dep_wait();
   const int row = blockIdx.x;
@@ -156,7 +152,7 @@ __global__ void upsample_add_kernel(Dims dm, SeqState st, int batch, int level, 
   const float* t = tri_ring + ((size_t)b * rsu + ((p / 3) % rsu)) * 3 * d + (p % 3) * d;
   for (int i = threadIdx.x; i < d; i += blockDim.x) x[(size_t)row * d + i] = valid ? h[i] + t[i] : 0.f;
   __syncthreads();
-  stack_entry_row(x + (size_t)row * d, row, d, g, a_out, ssq, ssq_tiles, ld_ssq);
+  stack_entry_row(x + (size_t)row * d, row, d, g, a_out, ssq);
 }
 
 // ------------------------------------------------------------------------------------------
