@@ -119,7 +119,8 @@ size_t fm_workspace_bytes(const fm_config* cfg /*HOST*/);
  * copies and rounds the weights, zeroes state.  `cuda_stream` is a cudaStream_t (NULL = the
  * default stream); all later work of this context runs on it.  Synchronous.
  * Errors: INVALID_ARG (null, bad config), CAPACITY (workspace too small), UNSUPPORTED
- * (d_model not a multiple of 64, head_dim not 32/64/128, D > FM_MAX_DRAFT), CUDA. */
+ * (d_model or d_ff not a multiple of 64, n_heads*head_dim not a multiple of 128, head_dim not
+ * 64/128, a stack without layers, D > FM_MAX_DRAFT), CUDA. */
 int fm_create(const fm_config* cfg /*HOST*/, const fm_weights* w /*HOST*/, void* dev_workspace /*DEV*/,
               size_t workspace_bytes, void* cuda_stream, fm_ctx** out /*HOST*/);
 int fm_destroy(fm_ctx* ctx);

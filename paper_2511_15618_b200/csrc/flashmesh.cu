@@ -116,7 +116,7 @@ int check_config(const fm_config* c) {
   for (int i = 0; i < 3; ++i) if (c->window[i] < 0) return FM_ERR_INVALID_ARG;
   for (int i = 0; i < 5; ++i) if (c->layers[i] < 1) return FM_ERR_UNSUPPORTED;
   if (c->draft_len > FM_MAX_DRAFT) return FM_ERR_UNSUPPORTED;
-  if (c->d_model % 64 != 0 || c->d_ff % 64 != 0 || (c->n_heads * c->head_dim) % 64 != 0) return FM_ERR_UNSUPPORTED;
+  if (c->d_model % 64 != 0 || c->d_ff % 64 != 0 || (c->n_heads * c->head_dim) % 128 != 0) return FM_ERR_UNSUPPORTED;
   if (c->head_dim != 64 && c->head_dim != 128) return FM_ERR_UNSUPPORTED;
   if ((c->draft_len + 8) / 9 > FM_MAX_FACE_HEADS) return FM_ERR_UNSUPPORTED;
   if (c->max_tokens < c->draft_len + 2) return FM_ERR_INVALID_ARG;
@@ -256,6 +256,29 @@ int upload_bf16(bf16* dst, const float* src, size_t n, std::vector<uint16_t>& tm
   CUDA_OK(cudaMemcpy(dst, tmp.data(), n * 2, cudaMemcpyHostToDevice));
   return FM_OK;
 }
+// fp32 host matrix [M, K] -> device weight slabs for the tensor-core GEMM: M padded to tiles of
+// 128 rows (zeros), K cut into slabs of 64; slab (t, k) is stored as the 16 KB image the MMA reads
+// from shared memory (row r at r*128 bytes, its 16-byte chunk c at position c ^ (r & 7): the
+// 128-byte swizzle), slabs of one tile one after the other.
+int upload_packed(bf16* dst, const float* src, size_t M, size_t K, std::vector<uint16_t>& tmp) {
+  if (src == nullptr) return FM_ERR_INVALID_ARG;
+  const size_t tiles = (M + 127) / 128, slabs = K / 64;
+  tmp.assign(tiles * 128 * K, 0);
+  for (size_t m = 0; m < M; ++m) {
+    const size_t t = m / 128, r = m % 128;
+    for (size_t k = 0; k < K; ++k) {
+      uint32_t u;
+      memcpy(&u, src + m * K + k, 4);
+      uint16_t h;
+      if ((u & 0x7fffffffu) > 0x7f800000u) h = 0x7fc0;                        // NaN
+      else { u += 0x7fffu + ((u >> 16) & 1u); h = (uint16_t)(u >> 16); }
+      const size_t kb = k / 64, c = (k % 64) / 8, e = k % 8;
+      tmp[((t * slabs + kb) * 128 + r) * 64 + ((c ^ (r & 7)) * 8) + e] = h;
+    }
+  }
+  CUDA_OK(cudaMemcpy(dst, tmp.data(), tmp.size() * 2, cudaMemcpyHostToDevice));
+  return FM_OK;
+}
 int upload_f32(float* dst, const float* src, size_t n) {
   if (src == nullptr) return FM_ERR_INVALID_ARG;
   CUDA_OK(cudaMemcpy(dst, src, n * 4, cudaMemcpyHostToDevice));
@@ -388,8 +411,9 @@ tc::Epi epi_plain(void* out, int ldo) {
 }
 
 // y[n][m] = W[w_row0 + m, :] . A[a_row0 + n, :], n < R, m < M, finished by the epilogue `mode`
-// (see fm_gemm_tc.cuh).  W: [w_rows_alloc, K] bf16 (rows padded to 128), A: [a_rows_alloc, K] bf16
-// (rows padded to 16).  The K split (= cluster size) depends on (M, K) only.
+// (see fm_gemm_tc.cuh).  W: packed weight slabs of a matrix with K columns (w_row0 a multiple of
+// 128), A: [a_rows_alloc, K] bf16 (rows padded to 16).  The K split (= cluster size) depends on
+// (M, K) only.
 void gemm(fm_ctx* c, const bf16* W, size_t w_rows_alloc, int w_row0, const bf16* A, size_t a_rows_alloc, int a_row0,
           int M, int K, int R, const int* n_active, int mode, tc::Epi e) {
   if (R <= 0) return;
@@ -397,14 +421,15 @@ void gemm(fm_ctx* c, const bf16* W, size_t w_rows_alloc, int w_row0, const bf16*
   int split = 1;
   while (split * 2 <= tc::MAX_SPLIT && split * 2 <= slabs && tiles * split * 2 <= c->split_target) split *= 2;
   const int Rpad = round_up(R, 16);
-  const int tW = tmap_for(c, W, w_rows_alloc, K, tc::BM);
+  (void)w_rows_alloc;
+  if (w_row0 % tc::BM != 0) { c->launch_error = FM_ERR_UNSUPPORTED; return; }
   const long pi = prof_open(c, PROF_GEMM, 2.0 * M * K);            // algorithmic bytes: the weight matrix once
   for (int n0 = 0; n0 < Rpad; n0 += tc::MAX_N) {                   // N tiles of at most MAX_N rows
     const int N = Rpad - n0 < tc::MAX_N ? Rpad - n0 : tc::MAX_N;
     const int tA = tmap_for(c, A, a_rows_alloc, K, N);
-    if (tW < 0 || tA < 0) { c->launch_error = FM_ERR_CUDA; break; }
+    if (tA < 0) { c->launch_error = FM_ERR_CUDA; break; }
     const int stages = tc::pick_stages(N);
-    tc::Args g{c->tmaps + tW, c->tmaps + tA, M, K, N, (R - n0 < N ? R - n0 : N), split, stages, w_row0, a_row0 + n0, n_active,
+    tc::Args g{W, c->tmaps + tA, M, K, N, (R - n0 < N ? R - n0 : N), split, stages, w_row0 / tc::BM, a_row0 + n0, n_active,
                c->st.status};
     e.row0 = n0;
     const int smem = tc::smem_bytes(N, stages);
@@ -703,25 +728,25 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
     for (size_t l = 0; l < c->layers[s].size(); ++l) {
       const fm_layer_weights& hw = w->stack[s][l];
       LayerDev& L = c->layers[s][l];
-      TRY(upload_bf16(L.Wqkv, hw.Wqkv, qkvw * d, tmp));
-      TRY(upload_bf16(L.Wo, hw.Wo, d * hd, tmp));
-      TRY(upload_bf16(L.W1, hw.W1, (size_t)dm.dff * d, tmp));
-      TRY(upload_bf16(L.W2, hw.W2, d * dm.dff, tmp));
+      TRY(upload_packed(L.Wqkv, hw.Wqkv, qkvw, d, tmp));
+      TRY(upload_packed(L.Wo, hw.Wo, d, hd, tmp));
+      TRY(upload_packed(L.W1, hw.W1, (size_t)dm.dff, d, tmp));
+      TRY(upload_packed(L.W2, hw.W2, d, (size_t)dm.dff, tmp));
       TRY(upload_f32(L.g1, hw.g1, d));
       TRY(upload_f32(L.g2, hw.g2, d));
     }
-  TRY(upload_bf16(c->S_cv, w->S_cv, d * 3 * d, tmp));
-  TRY(upload_bf16(c->S_vf, w->S_vf, d * 3 * d, tmp));
-  TRY(upload_bf16(c->U_fv, w->U_fv, 3 * d * d, tmp));
-  TRY(upload_bf16(c->U_vc, w->U_vc, 3 * d * d, tmp));
-  TRY(upload_bf16(c->W_out, w->W_out, (size_t)dm.V * d, tmp));
+  TRY(upload_packed(c->S_cv, w->S_cv, d, 3 * d, tmp));
+  TRY(upload_packed(c->S_vf, w->S_vf, d, 3 * d, tmp));
+  TRY(upload_packed(c->U_fv, w->U_fv, 3 * d, d, tmp));
+  TRY(upload_packed(c->U_vc, w->U_vc, 3 * d, d, tmp));
+  TRY(upload_packed(c->W_out, w->W_out, (size_t)dm.V, d, tmp));
   TRY(upload_f32(c->g_out, w->g_out, d));
   const size_t dpad = align_up(d, 128);
   for (int h = 0; h < dm.NH; ++h) {
     const float* A = h < 2 ? w->head_c_A[h] : h < 4 ? w->head_v_A[h - 2] : w->head_f_A[h - 4];
     const float* g = h < 2 ? w->head_c_g[h] : h < 4 ? w->head_v_g[h - 2] : w->head_f_g[h - 4];
     if (dm.D == 0 && (A == nullptr || g == nullptr)) continue;     // no drafts: heads are unused
-    TRY(upload_bf16(c->headA + (size_t)h * dpad * d, A, d * d, tmp));
+    TRY(upload_packed(c->headA + (size_t)h * dpad * d, A, d, d, tmp));
     TRY(upload_f32(c->head_g + (size_t)h * d, g, d));
   }
   // TMA descriptors of the KV caches: each cache is a 2-D [max_batch*Hkv*slots, dh] bf16 matrix

@@ -4,10 +4,13 @@
 //   y[n][m] = sum_k W[m, k] * A[n, k]        (bf16 operands, fp32 accumulation in tensor memory)
 //
 // The weight matrix sits on the MMA's M axis (tiles of 128 output features), the few token rows
-// on its N axis (16..256, padded), so a [128 x 64] weight slab is consumed by four
-// tcgen05.mma (K = 16 each) however few rows there are.  Both operands are K-major and are
-// brought in by TMA with the 128-byte swizzle into a ring of shared-memory stages; one thread
-// issues the MMAs, accumulators live in tensor memory and are read back with tcgen05.ld.
+// on its N axis (16..240, padded), so a [128 x 64] weight slab is consumed by four
+// tcgen05.mma (K = 16 each) however few rows there are.  Both operands are K-major with the
+// 128-byte swizzle.  Weights are stored in HBM slab by slab, each [128 x 64] slab as the 16 KB
+// image the MMA reads from shared memory, so a CTA's K range is one contiguous stream fetched by
+// 16 KB bulk copies; the token rows come through a TMA tensor map.  A ring of shared-memory stages
+// decouples the copies from the one thread that issues the MMAs; accumulators live in tensor
+// memory and are read back with tcgen05.ld.
 // The work is bandwidth bound: the grid is (M/128 tiles) x (S splits of K) so that many SMs
 // stream weights.  The S CTAs of one M tile form a thread-block cluster: every CTA owns 1/S of the
 // tile's columns; each CTA sends the columns of its partial tile to their owners' shared memory
@@ -37,13 +40,13 @@ constexpr int MAX_N = 240;       // token rows per launch: two stages + the rece
 enum EpiMode { EPI_F32 = 0, EPI_BF16 = 1, EPI_GELU = 2, EPI_RESID = 3, EPI_QKV = 4 };
 
 struct Args {
-  const CUtensorMap* tmW;        // [Mpad, K] bf16, box 128 x 64
+  const bf16* W;                 // packed weight slabs: [M tile][K slab][128 x 64 swizzled image]
   const CUtensorMap* tmA;        // [rows, K] bf16, box N x 64
   int M, K, N;                   // N = padded rows in the box (multiple of 16, <= MAX_N)
   int n_store;                   // rows actually stored (<= N)
   int split;                     // K splits = gridDim.y = cluster size (1, 2, 4 or 8)
   int stages;                    // depth of the shared-memory ring (2..MAX_STAGES)
-  int w_row0, a_row0;            // row offsets into the tensor maps (stacked weights / row groups)
+  int w_tile0, a_row0;           // first M tile inside W (stacked matrices), first operand row
   const int* n_active;           // skip when *n_active == 0 (may be null); must not change during a pass
   int* status;
 };
@@ -108,10 +111,10 @@ __device__ inline uint32_t cluster_rank() {
 __device__ inline void cluster_sync() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-// 4-byte store into a peer CTA's shared memory that reports its bytes to an mbarrier of that CTA
-__device__ inline void st_async_peer(uint32_t remote_addr, float a, uint32_t remote_bar) {
-  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(remote_addr), "r"(__float_as_uint(a)),
-               "r"(remote_bar)
+// 16-byte store into a peer CTA's shared memory that reports its bytes to an mbarrier of that CTA
+__device__ inline void st_async_peer4(uint32_t remote_addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d, uint32_t remote_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(remote_addr),
+               "r"(a), "r"(b), "r"(c), "r"(d), "r"(remote_bar)
                : "memory");
 }
 __device__ inline bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
@@ -139,15 +142,16 @@ __device__ inline uint32_t map_peer(uint32_t local_addr, uint32_t rank) {
 }
 
 // Shared memory: ring of `stages` x ([128 x 64] weight slab + [N x 64] operand slab), then the
-// receive buffer of the cluster reduction [split][N][64/split][2] fp32 = N * 512 bytes (peers write
-// into it while this CTA may still be multiplying, so it never aliases the ring), then barriers.
+// receive buffer of the cluster reduction [split][64/split][2][N + 4] fp32 = (N + 4) * 512 bytes
+// (peers write into it while this CTA may still be multiplying, so it never aliases the ring;
+// the 4 floats of padding spread the readers over the banks), then barriers.
 inline int stage_bytes(int N) { return BM * 128 + ((N * 128 + 1023) / 1024) * 1024; }
 inline int pick_stages(int N) {
-  int st = (200 * 1024 - N * 512) / stage_bytes(N);
+  int st = (200 * 1024 - (N + 4) * 512) / stage_bytes(N);
   st = st > 4 ? 4 : st;
   return st < 2 ? 2 : st;
 }
-inline int smem_bytes(int N, int stages) { return stages * stage_bytes(N) + N * 512 + 1024 + 256; }
+inline int smem_bytes(int N, int stages) { return stages * stage_bytes(N) + (N + 4) * 512 + 1024 + 256; }
 
 __device__ inline float gelu_erf_f(float x) { return 0.5f * x * (1.f + erff(x * 0.70710678118654752f)); }
 
@@ -173,8 +177,9 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   const int STAGES = g.stages;
   const int b_bytes = ((g.N * 128 + 1023) / 1024) * 1024;
   const int stage_bytes = BM * 128 + b_bytes;
-  float* recv = reinterpret_cast<float*>(sm + STAGES * stage_bytes);          // [S][N][PW][2]
-  uint64_t* full = reinterpret_cast<uint64_t*>(sm + STAGES * stage_bytes + g.N * 512);
+  const int NP = g.N + 4;
+  float* recv = reinterpret_cast<float*>(sm + STAGES * stage_bytes);          // [S][PW][2][NP]
+  uint64_t* full = reinterpret_cast<uint64_t*>(sm + STAGES * stage_bytes + NP * 512);
   uint64_t* empty = full + MAX_STAGES;
   uint64_t* accum = empty + MAX_STAGES;
   uint64_t* rbar = accum + 1;                                                 // partials of all ranks have arrived
@@ -199,8 +204,8 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
     ptx::mbar_init(accum, 1);
     ptx::mbar_init(rbar, 1);
     ptx::fence_mbar_init();
-    ptx::mbar_expect_tx(rbar, (uint32_t)g.n_store * 512u);   // n_store rows x 128/S columns x S ranks x 4 bytes
-    ptx::prefetch_tmap(g.tmW);
+    // rows are sent in groups of 16: groups x 16 rows x 128/S columns x S ranks x 4 bytes
+    ptx::mbar_expect_tx(rbar, (uint32_t)((g.n_store + 15) / 16) * 16u * 512u);
     ptx::prefetch_tmap(g.tmA);
   }
   if (warp == 0) {
@@ -222,10 +227,11 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   if (warp == 0 && lane == 0) {
     // ---- producer: stream this CTA's K range through the stage ring.  The weight slabs of the
     // first stages do not depend on the previous kernel and are requested before the wait.
+    const bf16* wsrc = g.W + ((size_t)(g.w_tile0 + tile_m) * slabs + s0) * (BM * BK);
     const int pre = n_slabs < STAGES ? n_slabs : STAGES;
     for (int i = 0; i < pre; ++i) {
       ptx::mbar_expect_tx(full + i, BM * 128 + g.N * 128);
-      ptx::tma_load_2d(sm + i * stage_bytes, g.tmW, (s0 + i) * BK, g.w_row0 + tile_m * BM, full + i);
+      ptx::bulk_load(sm + i * stage_bytes, wsrc + (size_t)i * (BM * BK), BM * 128, full + i);
     }
     ptx::grid_dep_wait();
     for (int i = 0; i < pre; ++i)
@@ -235,7 +241,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
       if (!ptx::mbar_wait(empty + st, ((i / STAGES) - 1) & 1)) { s_fail = 1; break; }
       unsigned char* a_dst = sm + st * stage_bytes;
       ptx::mbar_expect_tx(full + st, BM * 128 + g.N * 128);
-      ptx::tma_load_2d(a_dst, g.tmW, (s0 + i) * BK, g.w_row0 + tile_m * BM, full + st);
+      ptx::bulk_load(a_dst, wsrc + (size_t)i * (BM * BK), BM * 128, full + st);
       ptx::tma_load_2d(a_dst + BM * 128, g.tmA, (s0 + i) * BK, g.a_row0, full + st);
     }
   } else if (warp == 1 && lane == 0) {
@@ -296,7 +302,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
 
   // ---- where this thread's accumulator column goes, and its first item of the epilogue.  Column
   // m of the tile is half h of pair slot q; slots [r*PW, (r+1)*PW) belong to rank r, which receives
-  // [source rank][row][slot][half].  Everything that does not depend on the previous kernel
+  // [source rank][slot][half][row].  Everything that does not depend on the previous kernel
   // (indices, gains, rotary angles) is prepared here, before the wait.
   const int PW = 64 / S;
   const bool head128 = MODE == EPI_QKV && e.dm.dh == 128;
@@ -306,7 +312,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
     const int q = head128 ? (tid & 63) : ((tid >> 6) * 32 + (tid & 31));
     const int h = head128 ? (tid >> 6) : ((tid >> 5) & 1);
     const int owner = q / PW, cc = q - owner * PW;
-    dst0 = map_peer(ptx::smem_u32(recv + ((size_t)z * g.N * PW + cc) * 2 + h), (uint32_t)owner);
+    dst0 = map_peer(ptx::smem_u32(recv + (((size_t)z * PW + cc) * 2 + h) * NP), (uint32_t)owner);
     dbar = map_peer(ptx::smem_u32(rbar), (uint32_t)owner);
   }
   float pre_ga = 1.f, pre_gb = 1.f;
@@ -352,8 +358,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
       for (int j = 0; j < 16; ++j) r[j] = 0u;
     }
 #pragma unroll
-    for (int j = 0; j < 16; ++j)
-      if (n0 + j < g.n_store) st_async_peer(dst0 + (uint32_t)((n0 + j) * PW * 8), __uint_as_float(r[j]), dbar);
+    for (int j = 0; j < 16; j += 4) st_async_peer4(dst0 + (uint32_t)(n0 + j) * 4u, r[j], r[j + 1], r[j + 2], r[j + 3], dbar);
   }
   __syncthreads();                                         // s_inv / row maps are written
   const bool arrived = mbar_wait_cluster(rbar, 0);
@@ -368,14 +373,17 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
     const int n = active ? it / PW : 0, cc = active ? it - n * PW : 0;
     int ca, cb;
     pair_cols(z * PW + cc, head128, ca, cb);
-    float2 v[MAX_SPLIT];
+    float va[MAX_SPLIT], vb[MAX_SPLIT];
 #pragma unroll
-    for (int r = 0; r < MAX_SPLIT; ++r)                    // all loads first, then the sums in rank order
-      v[r] = (r < S && active) ? *reinterpret_cast<const float2*>(recv + (((size_t)r * g.N + n) * PW + cc) * 2) : make_float2(0.f, 0.f);
+    for (int r = 0; r < MAX_SPLIT; ++r) {                  // all loads first, then the sums in rank order
+      const float* src = recv + (((size_t)r * PW + cc) * 2) * NP + n;
+      va[r] = (r < S && active) ? src[0] : 0.f;
+      vb[r] = (r < S && active) ? src[NP] : 0.f;
+    }
     float ya = 0.f, yb = 0.f;
 #pragma unroll
     for (int r = 0; r < MAX_SPLIT; ++r)
-      if (r < S) { ya += v[r].x; yb += v[r].y; }
+      if (r < S) { ya += va[r]; yb += vb[r]; }
     const float inv = s_inv[n];
     ya *= inv;
     yb *= inv;
