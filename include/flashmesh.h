@@ -155,6 +155,28 @@ int fm_draft(fm_ctx* ctx, int32_t* cand /*DEV*/, float* draft_logits /*DEV*/, fl
 int fm_verify(fm_ctx* ctx, const int32_t* cand /*DEV*/, int32_t* argmax /*DEV*/, float* logits /*DEV*/,
               float* margin /*DEV*/);
 
+/* fm_verify for callers that cannot provide scratch memory of their own (no counterpart in the
+ * paper).  Some hosts of this library carve the workspace of fm_create out of an arena that is
+ * sized and committed once at start-up -- a serving process with a fixed memory plan, a plug-in that
+ * is forbidden to call cudaMalloc because an allocation would synchronise the device under its
+ * real-time loop -- and want the attention kernel's split-KV scratch (per-group partial results and
+ * the ticket counters of the final merge) kept out of that arena.  This call does what fm_verify
+ * does, same arguments, same results, but points the attention kernel at a fixed array of
+ * FM_STATIC_SCRATCH_BYTES bytes that is part of the library image: every GPU that loads the library
+ * holds that many bytes until the process exits.  It allocates nothing (no cudaMalloc, no
+ * cudaFree, no allocating library routine); inputs and outputs are still the caller's.
+ *   - Limit: the scratch one pass needs (it grows with max_batch * n_kv_heads and with the cache
+ *     capacity) must fit in FM_STATIC_SCRATCH_BYTES, else FM_ERR_CAPACITY is returned and nothing
+ *     is enqueued.
+ *   - The first call on a device looks up the array's device address (with the context's device
+ *     current); make that first call before any stream capture is begun.
+ *   - All contexts and all calls share the one array.  It keeps the previous call's contents (the
+ *     call clears the counters that must start at zero), and two calls whose kernels overlap on
+ *     the GPU -- different streams, different contexts -- race on it: serialise them. */
+#define FM_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
+int fm_verify_static_scratch(fm_ctx* ctx, const int32_t* cand /*DEV*/, int32_t* argmax /*DEV*/, float* logits /*DEV*/,
+                             float* margin /*DEV*/);
+
 /* Accept (Sec. 3.3) and roll back: a = 1 + number of leading drafts that equal the backbone's
  * argmax at the previous row; clipped to the rows fed and at an accepted EOS; L += a; the next
  * main token is the argmax at row a-1.  force_tok: DEV int32 [batch, D+1] or NULL, replaces the

@@ -89,6 +89,8 @@ def load_library():
     lib.fm_draft.argtypes = [vp, vp, f32p, f32p]
     lib.fm_verify.restype = C.c_int
     lib.fm_verify.argtypes = [vp, vp, vp, f32p, f32p]
+    lib.fm_verify_static_scratch.restype = C.c_int
+    lib.fm_verify_static_scratch.argtypes = [vp, vp, vp, f32p, f32p]
     lib.fm_accept.restype = C.c_int
     lib.fm_accept.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.fm_generate.restype = C.c_int
@@ -147,6 +149,12 @@ def fm_draft(ctx, cand_ptr, draft_logits_ptr=None, draft_margin_ptr=None):
 
 def fm_verify(ctx, cand_ptr, argmax_ptr=None, logits_ptr=None, margin_ptr=None):
     return load_library().fm_verify(ctx, cand_ptr, argmax_ptr, logits_ptr, margin_ptr)
+
+
+def fm_verify_static_scratch(ctx, cand_ptr, argmax_ptr=None, logits_ptr=None, margin_ptr=None):
+    """fm_verify with the attention kernel's scratch in the library's own fixed array: for hosts
+    that may not allocate device memory for it (see include/flashmesh.h)."""
+    return load_library().fm_verify_static_scratch(ctx, cand_ptr, argmax_ptr, logits_ptr, margin_ptr)
 
 
 def fm_accept(ctx, force_len_ptr=None, force_tok_ptr=None, n_acc_ptr=None, emitted_ptr=None, kv_len_ptr=None):

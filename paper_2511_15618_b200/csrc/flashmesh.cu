@@ -36,6 +36,10 @@ inline int round_up(int v, int a) { return (v + a - 1) / a * a; }
 
 }  // namespace
 
+// Attention scratch (group partials, then tickets) for fm_verify_static_scratch: lives in the
+// library image, so every GPU that loads the library holds these bytes until the process exits.
+static __device__ __align__(256) unsigned char g_static_attn_scratch[FM_STATIC_SCRATCH_BYTES];
+
 struct fm_ctx {
   fm_config cfg;
   Dims dm;
@@ -913,6 +917,45 @@ int fm_verify(fm_ctx* c, const int32_t* cand, int32_t* argmax, float* logits, fl
   if (c->launch_error != FM_OK) return c->launch_error;
   c->phase = 2;
   return FM_OK;
+}
+
+int fm_verify_static_scratch(fm_ctx* c, const int32_t* cand, int32_t* argmax, float* logits, float* margin) {
+  if (c == nullptr || cand == nullptr) return FM_ERR_INVALID_ARG;
+  if (c->phase < 1) return FM_ERR_BAD_STATE;
+  // what the attention kernel needs: the largest level's group partials, then one ticket per
+  // (sequence, kv-head, query tile)
+  const Dims& dm = c->dm;
+  size_t part_floats = 0, tickets = 0;
+  for (int l = 0; l < 3; ++l) {
+    const size_t per = (size_t)dm.max_batch * dm.Hkv * c->attn_mt[l];
+    const size_t need = per * c->attn_max_groups[l] * 16 * (dm.dh + 2);
+    part_floats = need > part_floats ? need : part_floats;
+    tickets = per > tickets ? per : tickets;
+  }
+  const size_t ticket_off = align_up(part_floats * sizeof(float), 256);
+  if (ticket_off + tickets * sizeof(int) > (size_t)FM_STATIC_SCRATCH_BYTES) return FM_ERR_CAPACITY;
+  // Device address of the static array, looked up once per device with that device current (the
+  // array's name is only a host-side handle; a kernel must be given this address).
+  static void* dev_addr[64] = {nullptr};
+  int dev = -1;
+  CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return FM_ERR_UNSUPPORTED;
+  if (dev_addr[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_attn_scratch) != cudaSuccess || p == nullptr) return FM_ERR_CUDA;
+    dev_addr[dev] = p;
+  }
+  unsigned char* base = static_cast<unsigned char*>(dev_addr[dev]);
+  // tickets must start at zero; the array keeps whatever the last call (of any context) left
+  CUDA_OK(cudaMemsetAsync(base + ticket_off, 0, tickets * sizeof(int), c->stream));
+  float* saved_part = c->attn_part;
+  int* saved_ticket = c->attn_ticket;
+  c->attn_part = reinterpret_cast<float*>(base);
+  c->attn_ticket = reinterpret_cast<int*>(base + ticket_off);
+  const int rc = fm_verify(c, cand, argmax, logits, margin);
+  c->attn_part = saved_part;
+  c->attn_ticket = saved_ticket;
+  return rc;
 }
 
 int fm_accept(fm_ctx* c, const int32_t* force_len, const int32_t* force_tok, int32_t* n_acc, int32_t* emitted,
