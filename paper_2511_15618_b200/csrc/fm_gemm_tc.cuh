@@ -207,6 +207,14 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
     // rows are sent in groups of 16: groups x 16 rows x 128/S columns x S ranks x 4 bytes
     ptx::mbar_expect_tx(rbar, (uint32_t)((g.n_store + 15) / 16) * 16u * 512u);
     ptx::prefetch_tmap(g.tmA);
+    // The weight slabs of the first stages do not depend on the previous kernel: request them at
+    // once, so that they travel while the rest of the prologue runs.
+    const bf16* wsrc = g.W + ((size_t)(g.w_tile0 + tile_m) * slabs + s0) * (BM * BK);
+    const int pre = n_slabs < STAGES ? n_slabs : STAGES;
+    for (int i = 0; i < pre; ++i) {
+      ptx::mbar_expect_tx(full + i, BM * 128 + g.N * 128);
+      ptx::bulk_load(sm + i * stage_bytes, wsrc + (size_t)i * (BM * BK), BM * 128, full + i);
+    }
   }
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(ptx::smem_u32(tmem_slot)), "r"(ncols)
@@ -225,14 +233,10 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   if (S > 1) cluster_sync();
 
   if (warp == 0 && lane == 0) {
-    // ---- producer: stream this CTA's K range through the stage ring.  The weight slabs of the
-    // first stages do not depend on the previous kernel and are requested before the wait.
+    // ---- producer: stream this CTA's K range through the stage ring (the weight slabs of the
+    // first stages are already on their way)
     const bf16* wsrc = g.W + ((size_t)(g.w_tile0 + tile_m) * slabs + s0) * (BM * BK);
     const int pre = n_slabs < STAGES ? n_slabs : STAGES;
-    for (int i = 0; i < pre; ++i) {
-      ptx::mbar_expect_tx(full + i, BM * 128 + g.N * 128);
-      ptx::bulk_load(sm + i * stage_bytes, wsrc + (size_t)i * (BM * BK), BM * 128, full + i);
-    }
     ptx::grid_dep_wait();
     for (int i = 0; i < pre; ++i)
       ptx::tma_load_2d(sm + i * stage_bytes + BM * 128, g.tmA, (s0 + i) * BK, g.a_row0, full + i);
@@ -304,21 +308,22 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   // m of the tile is half h of pair slot q; slots [r*PW, (r+1)*PW) belong to rank r, which receives
   // [source rank][slot][half][row].  Everything that does not depend on the previous kernel
   // (indices, gains, rotary angles) is prepared here, before the wait.
-  const int PW = 64 / S;
+  const int lgS = 31 - __clz(S);                           // S is 1, 2, 4 or 8
+  const int lgPW = 6 - lgS, PW = 1 << lgPW;
   const bool head128 = MODE == EPI_QKV && e.dm.dh == 128;
   const int items = g.n_store * PW;
   uint32_t dst0, dbar;
   {
     const int q = head128 ? (tid & 63) : ((tid >> 6) * 32 + (tid & 31));
     const int h = head128 ? (tid >> 6) : ((tid >> 5) & 1);
-    const int owner = q / PW, cc = q - owner * PW;
+    const int owner = q >> lgPW, cc = q & (PW - 1);
     dst0 = map_peer(ptx::smem_u32(recv + (((size_t)z * PW + cc) * 2 + h) * NP), (uint32_t)owner);
     dbar = map_peer(ptx::smem_u32(rbar), (uint32_t)owner);
   }
   float pre_ga = 1.f, pre_gb = 1.f;
   float2 pre_cs = make_float2(1.f, 0.f);
   if (tid < items) {
-    const int n = tid / PW, cc = tid - n * PW;
+    const int n = tid >> lgPW, cc = tid & (PW - 1);
     int ca, cb;
     pair_cols(z * PW + cc, head128, ca, cb);
     const int ma = tile_m * BM + ca, mb = tile_m * BM + cb;
@@ -333,24 +338,42 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
       if (valid && ma < g.M && head < e.dm.H + e.dm.Hkv) pre_cs = e.rope_tab[(size_t)p * (e.dm.dh >> 1) + i];
     }
   }
+  // Kernel parameters the tail needs, read into registers now: a first touch of the parameter
+  // bank after the wait would sit on the critical path.
+  int k_row0 = e.row0, k_ldo = e.ldo, k_ldx = e.ldx, k_add = e.add, k_lda = e.lda, k_ldssq = e.ld_ssq_out;
+  int k_M = g.M, k_ns = g.n_store;
+  void* k_out = e.out;
+  float* k_x = e.x;
+  const float* k_gain = e.gain;
+  bf16* k_aout = e.a_out;
+  float* k_ssqo = e.ssq_out;
+  bf16 *k_q = e.q_out, *k_K = e.Kc, *k_V = e.Vc;
+  const float2* k_rope = e.rope_tab;
+  float k_qs = e.qscale, k_theta = e.dm.theta;
+  int k_H = e.dm.H, k_Hkv = e.dm.Hkv, k_dh = e.dm.dh, k_P = e.dm.P, k_cap = MODE == EPI_QKV ? e.dm.cap[e.level] : 1;
+  int* k_status = g.status;
+  asm volatile("" : "+r"(k_row0), "+r"(k_ldo), "+r"(k_ldx), "+r"(k_add), "+r"(k_lda), "+r"(k_ldssq), "+r"(k_M), "+r"(k_ns));
+  asm volatile("" : "+l"(k_out), "+l"(k_x), "+l"(k_gain), "+l"(k_aout), "+l"(k_ssqo), "+l"(k_q), "+l"(k_K), "+l"(k_V), "+l"(k_rope), "+l"(k_status));
+  asm volatile("" : "+f"(k_qs), "+f"(k_theta), "+r"(k_H), "+r"(k_Hkv), "+r"(k_dh), "+r"(k_P), "+r"(k_cap));
   ptx::grid_dep_wait();                                    // everything below touches activations
   float pre_xa = 0.f, pre_xb = 0.f;
-  if (MODE == EPI_RESID && e.add && tid < items) {
-    const int n = tid / PW, cc = tid - n * PW;
+  if (MODE == EPI_RESID && k_add && tid < items) {
+    const int n = tid >> lgPW, cc = tid & (PW - 1);
     int ca, cb;
     pair_cols(z * PW + cc, head128, ca, cb);
     const int ma = tile_m * BM + ca, mb = tile_m * BM + cb;
-    const float* xr = e.x + (size_t)(e.row0 + n) * e.ldx;
-    if (ma < g.M) pre_xa = xr[ma];
-    if (mb < g.M) pre_xb = xr[mb];
+    const float* xr = k_x + (size_t)(k_row0 + n) * k_ldx;
+    if (ma < k_M) pre_xa = xr[ma];
+    if (mb < k_M) pre_xb = xr[mb];
   }
 
+  __syncthreads();                                         // s_inv / row maps are written (long before the MMAs end)
   // ---- every warp waits for the accumulator and sends its 32 columns of the partial tile to
   // their owners.  A timeout is recorded; zeros are sent so that no owner waits in vain.
   bool ok = n_slabs > 0 ? ptx::mbar_wait(accum, 0) : true;
   ok = __all_sync(0xffffffffu, ok);
   fence_after();
-  for (int n0 = 0; n0 < g.n_store; n0 += 16) {
+  for (int n0 = 0; n0 < k_ns; n0 += 16) {
     uint32_t r[16];
     if (ok && n_slabs > 0) ld16(tmem + ((uint32_t)(warp * 32) << 16) + n0, r);
     else {
@@ -360,23 +383,22 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
 #pragma unroll
     for (int j = 0; j < 16; j += 4) st_async_peer4(dst0 + (uint32_t)(n0 + j) * 4u, r[j], r[j + 1], r[j + 2], r[j + 3], dbar);
   }
-  __syncthreads();                                         // s_inv / row maps are written
   const bool arrived = mbar_wait_cluster(rbar, 0);
   if (!ok || !arrived || s_fail) {
-    if (tid == 0) atomicExch(g.status, -5);
+    if (tid == 0) atomicExch(k_status, -5);
   }
   // ---- this rank's share of the tile: pair slots [z*PW, (z+1)*PW), all rows
-  const int L = PW < 32 ? PW : 32;                         // lanes that share a row
+  const int lgL = lgPW < 5 ? lgPW : 5, L = 1 << lgL;        // lanes that share a row
   for (int it0 = 0; it0 < items; it0 += 128) {
     const int it = it0 + tid;
     const bool active = it < items, first = it0 == 0;
-    const int n = active ? it / PW : 0, cc = active ? it - n * PW : 0;
+    const int n = active ? it >> lgPW : 0, cc = active ? it & (PW - 1) : 0;
     int ca, cb;
     pair_cols(z * PW + cc, head128, ca, cb);
     float va[MAX_SPLIT], vb[MAX_SPLIT];
 #pragma unroll
     for (int r = 0; r < MAX_SPLIT; ++r) {                  // all loads first, then the sums in rank order
-      const float* src = recv + (((size_t)r * PW + cc) * 2) * NP + n;
+      const float* src = recv + ((r << lgPW) + cc) * 2 * NP + n;
       va[r] = (r < S && active) ? src[0] : 0.f;
       vb[r] = (r < S && active) ? src[NP] : 0.f;
     }
@@ -388,65 +410,64 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
     ya *= inv;
     yb *= inv;
     const int ma = tile_m * BM + ca, mb = tile_m * BM + cb;
-    const bool a_ok = active && ma < g.M, b_ok = active && mb < g.M;
-    const size_t row = (size_t)(e.row0 + n);
+    const bool a_ok = active && ma < k_M, b_ok = active && mb < k_M;
+    const size_t row = (size_t)(k_row0 + n);
     if (MODE == EPI_F32) {
-      float* o = reinterpret_cast<float*>(e.out) + row * e.ldo;
+      float* o = reinterpret_cast<float*>(k_out) + row * k_ldo;
       if (a_ok) o[ma] = ya;
       if (b_ok) o[mb] = yb;
     } else if (MODE == EPI_BF16) {
-      bf16* o = reinterpret_cast<bf16*>(e.out) + row * e.ldo;
+      bf16* o = reinterpret_cast<bf16*>(k_out) + row * k_ldo;
       if (a_ok) o[ma] = __float2bfloat16(ya);
       if (b_ok) o[mb] = __float2bfloat16(yb);
     } else if (MODE == EPI_GELU) {
-      bf16* o = reinterpret_cast<bf16*>(e.out) + row * e.ldo;
+      bf16* o = reinterpret_cast<bf16*>(k_out) + row * k_ldo;
       if (a_ok) o[ma] = __float2bfloat16(gelu_erf_f(ya));
       if (b_ok) o[mb] = __float2bfloat16(gelu_erf_f(yb));
     } else if (MODE == EPI_RESID) {
-      float* xr = e.x + row * e.ldx;
+      float* xr = k_x + row * k_ldx;
       float xa = 0.f, xb = 0.f;
       if (a_ok) {
-        xa = (first ? pre_xa : (e.add ? xr[ma] : 0.f)) + ya;
+        xa = (first ? pre_xa : (k_add ? xr[ma] : 0.f)) + ya;
         xr[ma] = xa;
-        if (e.a_out != nullptr) e.a_out[row * e.lda + ma] = __float2bfloat16(xa * (first ? pre_ga : (e.gain != nullptr ? e.gain[ma] : 1.f)));
+        if (k_aout != nullptr) k_aout[row * k_lda + ma] = __float2bfloat16(xa * (first ? pre_ga : (k_gain != nullptr ? k_gain[ma] : 1.f)));
       }
       if (b_ok) {
-        xb = (first ? pre_xb : (e.add ? xr[mb] : 0.f)) + yb;
+        xb = (first ? pre_xb : (k_add ? xr[mb] : 0.f)) + yb;
         xr[mb] = xb;
-        if (e.a_out != nullptr) e.a_out[row * e.lda + mb] = __float2bfloat16(xb * (first ? pre_gb : (e.gain != nullptr ? e.gain[mb] : 1.f)));
+        if (k_aout != nullptr) k_aout[row * k_lda + mb] = __float2bfloat16(xb * (first ? pre_gb : (k_gain != nullptr ? k_gain[mb] : 1.f)));
       }
-      if (e.ssq_out != nullptr) {
+      if (k_ssqo != nullptr) {
         // per-row sums of squares of this rank's columns: a fixed shuffle tree over the L lanes that
         // share the row; the next GEMM adds the (tile, rank, lane group) partials in slot order
         float sqv = xa * xa + xb * xb;
         for (int o = L >> 1; o > 0; o >>= 1) sqv += __shfl_xor_sync(0xffffffffu, sqv, o);
         if (active && (cc & (L - 1)) == 0)
-          e.ssq_out[(size_t)((tile_m * S + z) * (PW / L) + cc / L) * e.ld_ssq_out + e.row0 + n] = sqv;
+          k_ssqo[(size_t)((((tile_m << lgS) + z) << (lgPW - lgL)) + (cc >> lgL)) * k_ldssq + k_row0 + n] = sqv;
       }
     } else {  // EPI_QKV: (ya, yb) is the rotary pair (i, i + dh/2) of one head
-      const Dims& dm = e.dm;
-      const int dh = dm.dh, half = dh >> 1, H = dm.H, Hkv = dm.Hkv;
+      const int dh = k_dh, half = dh >> 1, H = k_H, Hkv = k_Hkv;
       const int head = ma / dh, i = ma - head * dh;
       if (a_ok && head < H + 2 * Hkv) {
         const int b = s_rb[n], p = s_rp[n];
         const bool valid = b >= 0;
-        const int slots = dm.P + dm.cap[e.level];
+        const int slots = k_P + k_cap;
         if (head < H + Hkv) {
           float2 cs = make_float2(1.f, 0.f);
           if (first) cs = pre_cs;
-          else if (dm.theta != 0.f && valid) cs = e.rope_tab[(size_t)p * half + i];
+          else if (k_theta != 0.f && valid) cs = k_rope[(size_t)p * half + i];
           const float y1 = ya * cs.x - yb * cs.y, y2 = yb * cs.x + ya * cs.y;
           if (head < H) {
-            bf16* q = e.q_out + (row * H + head) * dh;
-            q[i] = __float2bfloat16(valid ? y1 * e.qscale : 0.f);
-            q[half + i] = __float2bfloat16(valid ? y2 * e.qscale : 0.f);
+            bf16* q = k_q + (row * H + head) * dh;
+            q[i] = __float2bfloat16(valid ? y1 * k_qs : 0.f);
+            q[half + i] = __float2bfloat16(valid ? y2 * k_qs : 0.f);
           } else if (valid) {
-            bf16* dst = e.Kc + (((size_t)b * Hkv + (head - H)) * slots + dm.P + (p % dm.cap[e.level])) * dh;
+            bf16* dst = k_K + (((size_t)b * Hkv + (head - H)) * slots + k_P + (p % k_cap)) * dh;
             dst[i] = __float2bfloat16(y1);
             dst[half + i] = __float2bfloat16(y2);
           }
         } else if (valid) {
-          bf16* dst = e.Vc + (((size_t)b * Hkv + (head - H - Hkv)) * slots + dm.P + (p % dm.cap[e.level])) * dh;
+          bf16* dst = k_V + (((size_t)b * Hkv + (head - H - Hkv)) * slots + k_P + (p % k_cap)) * dh;
           dst[i] = __float2bfloat16(ya);
           dst[half + i] = __float2bfloat16(yb);
         }
