@@ -220,8 +220,11 @@ void carve(fm_ctx* c, Carver& cv) {
   for (int l = 0; l < 3; ++l) {
     const int max_chunks = (dm.P + dm.cap[l] + c->attn_chunk - 1) / c->attn_chunk;
     c->attn_mt[l] = (fm_rows_per_seq(dm, l) * (dm.H / dm.Hkv) + 15) / 16;
+    // about one CTA per SM when the cache is full; at most 16 chunks per group
     int G = (int)(((size_t)max_chunks * dm.Hkv * B * c->attn_mt[l] + 147) / 148);
     G = G < 1 ? 1 : (G > 16 ? 16 : G);
+    const int G_min = (max_chunks + 23) / 24;          // at most 24 groups: their states (and weights) are merged from shared memory
+    G = G < G_min ? G_min : G;
     c->attn_G[l] = G;
     c->attn_max_groups[l] = (max_chunks + G - 1) / G;
     const size_t need = B * dm.Hkv * (size_t)c->attn_mt[l] * c->attn_max_groups[l] * 16 * (dm.dh + 2);
@@ -378,9 +381,9 @@ int tmap_for(fm_ctx* c, const void* base, uint64_t rows, uint64_t cols, uint32_t
 // Launch with the programmatic-dependent-launch attribute: the kernel may start while its
 // predecessor is still running and must execute griddepcontrol.wait before it touches anything a
 // predecessor produces (and before it exits).  Kernels launched through LAUNCH are full barriers.
-// cluster_y > 1 makes the CTAs along the grid's y extent one thread-block cluster.
+// `cluster` with more than one CTA makes thread-block clusters of that shape.
 template <typename... KArgs, typename... CArgs>
-void launch_pdl(fm_ctx* c, int cluster_y, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, CArgs&&... args) {
+void launch_pdl(fm_ctx* c, dim3 cluster, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, CArgs&&... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
@@ -393,11 +396,11 @@ void launch_pdl(fm_ctx* c, int cluster_y, void (*kern)(KArgs...), dim3 grid, dim
     at[n].val.programmaticStreamSerializationAllowed = 1;
     ++n;
   }
-  if (cluster_y > 1) {
+  if (cluster.x * cluster.y * cluster.z > 1) {
     at[n].id = cudaLaunchAttributeClusterDimension;
-    at[n].val.clusterDim.x = 1;
-    at[n].val.clusterDim.y = (unsigned)cluster_y;
-    at[n].val.clusterDim.z = 1;
+    at[n].val.clusterDim.x = cluster.x;
+    at[n].val.clusterDim.y = cluster.y;
+    at[n].val.clusterDim.z = cluster.z;
     ++n;
   }
   cfg.attrs = at;
@@ -439,11 +442,11 @@ void gemm(fm_ctx* c, const bf16* W, size_t w_rows_alloc, int w_row0, const bf16*
     const int smem = tc::smem_bytes(N, stages);
     const dim3 grid(tiles, split);
     switch (mode) {
-      case tc::EPI_F32: launch_pdl(c, split, tc::gemm_tc_kernel<tc::EPI_F32>, grid, 128, smem, g, e); break;
-      case tc::EPI_BF16: launch_pdl(c, split, tc::gemm_tc_kernel<tc::EPI_BF16>, grid, 128, smem, g, e); break;
-      case tc::EPI_GELU: launch_pdl(c, split, tc::gemm_tc_kernel<tc::EPI_GELU>, grid, 128, smem, g, e); break;
-      case tc::EPI_RESID: launch_pdl(c, split, tc::gemm_tc_kernel<tc::EPI_RESID>, grid, 128, smem, g, e); break;
-      default: launch_pdl(c, split, tc::gemm_tc_kernel<tc::EPI_QKV>, grid, 128, smem, g, e); break;
+      case tc::EPI_F32: launch_pdl(c, dim3(1, split, 1), tc::gemm_tc_kernel<tc::EPI_F32>, grid, 128, smem, g, e); break;
+      case tc::EPI_BF16: launch_pdl(c, dim3(1, split, 1), tc::gemm_tc_kernel<tc::EPI_BF16>, grid, 128, smem, g, e); break;
+      case tc::EPI_GELU: launch_pdl(c, dim3(1, split, 1), tc::gemm_tc_kernel<tc::EPI_GELU>, grid, 128, smem, g, e); break;
+      case tc::EPI_RESID: launch_pdl(c, dim3(1, split, 1), tc::gemm_tc_kernel<tc::EPI_RESID>, grid, 128, smem, g, e); break;
+      default: launch_pdl(c, dim3(1, split, 1), tc::gemm_tc_kernel<tc::EPI_QKV>, grid, 128, smem, g, e); break;
     }
   }
   prof_close(c, pi);
@@ -468,12 +471,13 @@ __global__ void row_count_kernel(Dims dm, SeqState st, int batch) {
 
 void attention(fm_ctx* c, int level, const LayerDev& L) {
   const Dims& dm = c->dm;
+  const int groups = c->attn_max_groups[level];
   AttnArgs a{dm, c->st, c->batch, level, c->qbuf, c->tmaps + L.tmK, c->tmaps + L.tmV, c->attn_part, c->attn_ticket,
-             c->a_attn, c->attn_G[level], c->attn_max_groups[level], c->attn_mt[level]};
-  dim3 grid(c->attn_max_groups[level] * c->attn_mt[level], dm.Hkv, c->batch);
+             c->a_attn, c->attn_G[level], groups, c->attn_mt[level]};
+  const dim3 grid(groups, dm.Hkv * c->attn_mt[level], c->batch);
   const long pi = prof_open(c, PROF_ATTN, 0.0);
-  if (dm.dh == 64) launch_pdl(c, 1, attn_stream_kernel<64, 128, 8>, grid, AttnCfg<64, 128, 8>::THREADS, AttnCfg<64, 128, 8>::BYTES, a);
-  else launch_pdl(c, 1, attn_stream_kernel<128, 64, 4>, grid, AttnCfg<128, 64, 4>::THREADS, AttnCfg<128, 64, 4>::BYTES, a);
+  if (dm.dh == 64) launch_pdl(c, dim3(1, 1, 1), attn_stream_kernel<64, 128, 8>, grid, AttnCfg<64, 128, 8>::THREADS, AttnCfg<64, 128, 8>::BYTES, a);
+  else launch_pdl(c, dim3(1, 1, 1), attn_stream_kernel<128, 64, 4>, grid, AttnCfg<128, 64, 4>::THREADS, AttnCfg<128, 64, 4>::BYTES, a);
   prof_close(c, pi);
 }
 
@@ -494,7 +498,7 @@ void run_stack(fm_ctx* c, int s, float* x, float* stash_ring, const float* next_
   for (int l = 0; l < nl; ++l) {
     const LayerDev& L = c->layers[s][l];
     if (stash_ring != nullptr && l == nl - 1)
-      launch_pdl(c, 1, ring_store_kernel, rows, 128, 0, dm, c->st, c->batch, level, (const float*)x, stash_ring, d);
+      launch_pdl(c, dim3(1, 1, 1), ring_store_kernel, rows, 128, 0, dm, c->st, c->batch, level, (const float*)x, stash_ring, d);
     tc::Epi eq{};
     eq.ssq_in = c->ssq; eq.ssq_n = c->ssq_n; eq.ld_ssq = c->ssq_ld; eq.inv_d_in = 1.f / d; eq.eps = dm.eps;
     eq.dm = dm; eq.st = c->st; eq.batch = c->batch; eq.level = level; eq.rope_tab = c->rope_tab;
@@ -530,34 +534,34 @@ void forward(fm_ctx* c, float* logits_out) {
   LAUNCH(c, embed_kernel, Rc, 128, 0, dm, c->st, B, c->E, c->xc, c->layers[0][0].g1, c->a_norm, c->ssq);
   c->ssq_n = 1;
   run_stack(c, 0, c->xc, nullptr, nullptr, false);
-  launch_pdl(c, 1, ring_store_kernel, Rc, 128, 0, dm, c->st, B, 0, (const float*)c->xc, c->hc_ring, d);
-  launch_pdl(c, 1, shorten_gather_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->hc_ring, c->a_cat);
+  launch_pdl(c, dim3(1, 1, 1), ring_store_kernel, Rc, 128, 0, dm, c->st, B, 0, (const float*)c->xc, c->hc_ring, d);
+  launch_pdl(c, dim3(1, 1, 1), shorten_gather_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->hc_ring, c->a_cat);
   tc::Epi es{};
   es.x = c->xv; es.ldx = d; es.add = 0; es.gain = c->layers[1][0].g1; es.a_out = c->a_norm; es.lda = d;
   es.ssq_out = c->ssq; es.ld_ssq_out = c->ssq_ld;
   gemm(c, c->S_cv, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rv, na + 1, tc::EPI_RESID, es);
   run_stack(c, 1, c->xv, nullptr, nullptr, false);
-  launch_pdl(c, 1, ring_store_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->xv, c->hv_ring, d);
-  launch_pdl(c, 1, shorten_gather_kernel, Rf, 128, 0, dm, c->st, B, 2, (const float*)c->hv_ring, c->a_cat);
+  launch_pdl(c, dim3(1, 1, 1), ring_store_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->xv, c->hv_ring, d);
+  launch_pdl(c, dim3(1, 1, 1), shorten_gather_kernel, Rf, 128, 0, dm, c->st, B, 2, (const float*)c->hv_ring, c->a_cat);
   es.x = c->xf; es.gain = c->layers[2][0].g1;
   gemm(c, c->S_vf, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rf, na + 2, tc::EPI_RESID, es);
   run_stack(c, 2, c->xf, c->zf, nullptr, true);                    // leaves bf16(xf) in a_norm
   gemm(c, c->U_fv, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rf, na + 2, tc::EPI_F32, epi_plain(c->tmp3d, 3 * d));
-  launch_pdl(c, 1, ring_store_kernel, Rf, 128, 0, dm, c->st, B, 2, (const float*)c->tmp3d, c->trif_ring, 3 * d);
-  launch_pdl(c, 1, upsample_add_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->hv_ring, (const float*)c->trif_ring, c->xv,
+  launch_pdl(c, dim3(1, 1, 1), ring_store_kernel, Rf, 128, 0, dm, c->st, B, 2, (const float*)c->tmp3d, c->trif_ring, 3 * d);
+  launch_pdl(c, dim3(1, 1, 1), upsample_add_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->hv_ring, (const float*)c->trif_ring, c->xv,
              (const float*)c->layers[3][0].g1, c->a_norm, c->ssq);
   c->ssq_n = 1;
   run_stack(c, 3, c->xv, c->zv, nullptr, true);                    // leaves bf16(xv) in a_norm
   gemm(c, c->U_vc, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rv, na + 1, tc::EPI_F32, epi_plain(c->tmp3d, 3 * d));
-  launch_pdl(c, 1, ring_store_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->tmp3d, c->triv_ring, 3 * d);
-  launch_pdl(c, 1, upsample_add_kernel, Rc, 128, 0, dm, c->st, B, 0, (const float*)c->hc_ring, (const float*)c->triv_ring, c->xc,
+  launch_pdl(c, dim3(1, 1, 1), ring_store_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->tmp3d, c->triv_ring, 3 * d);
+  launch_pdl(c, dim3(1, 1, 1), upsample_add_kernel, Rc, 128, 0, dm, c->st, B, 0, (const float*)c->hc_ring, (const float*)c->triv_ring, c->xc,
              (const float*)c->layers[4][0].g1, c->a_norm, c->ssq);
   c->ssq_n = 1;
   run_stack(c, 4, c->xc, c->zc, c->g_out, true);                   // leaves bf16(xc * g_out) and its sums of squares
   tc::Epi el = epi_plain(c->logits, dm.Vpad);
   el.ssq_in = c->ssq; el.ssq_n = c->ssq_n; el.ld_ssq = c->ssq_ld; el.inv_d_in = 1.f / d; el.eps = dm.eps;
   gemm(c, c->W_out, dm.Vpad, 0, c->a_norm, Rc_alloc, 0, dm.V, d, Rc, na, tc::EPI_F32, el);
-  launch_pdl(c, 1, verify_top2_kernel, Rc, 256, 0, dm, c->st, B, (const float*)c->logits, logits_out);
+  launch_pdl(c, dim3(1, 1, 1), verify_top2_kernel, Rc, 256, 0, dm, c->st, B, (const float*)c->logits, logits_out);
 }
 
 // a13: draft heads on the stashed split-node hiddens
@@ -573,17 +577,17 @@ void draft(fm_ctx* c, float* logits_out, float* margin_out) {
     for (int h = 0; h < dm.NH; ++h)
       gemm(c, c->headA, (size_t)dm.NH * dpad, h * dpad, c->dh_a, (size_t)dm.NH * MB + 16, h * (int)MB, d, d, B, na, tc::EPI_F32,
            epi_plain(c->dh_y + (size_t)h * MB * d, d));
-    launch_pdl(c, 1, draft_residual_kernel, dim3(B, dm.NH), 128, 0, dm, c->st, B, (const float*)c->zc, (const float*)c->zv,
+    launch_pdl(c, dim3(1, 1, 1), draft_residual_kernel, dim3(B, dm.NH), 128, 0, dm, c->st, B, (const float*)c->zc, (const float*)c->zv,
                (const float*)c->zf, (const float*)c->dh_y, c->feat, c->up_in_v, c->up_in_f);
     gemm(c, c->U_fv, pad128(3 * d), 0, c->up_in_f, align_up((size_t)dm.Ef * MB, 16), 0, 3 * d, d, dm.Ef * B, na, tc::EPI_BF16,
          epi_plain(c->up_in_v + (size_t)2 * B * d, 3 * d));
     gemm(c, c->U_vc, pad128(3 * d), 0, c->up_in_v, align_up((2 + 3 * (size_t)dm.Ef) * MB, 16), 0, 3 * d, d, (2 + 3 * dm.Ef) * B, na,
          tc::EPI_F32, epi_plain(c->feat + (size_t)2 * B * d, 3 * d));
-    launch_pdl(c, 1, rmsnorm_kernel, NF * B, 256, 0, (const float*)c->feat, (const float*)c->g_out, c->feat_n, d, dm.eps);
+    launch_pdl(c, dim3(1, 1, 1), rmsnorm_kernel, NF * B, 256, 0, (const float*)c->feat, (const float*)c->g_out, c->feat_n, d, dm.eps);
     gemm(c, c->W_out, dm.Vpad, 0, c->feat_n, align_up((size_t)NF * MB, 16), 0, dm.V, d, NF * B, na, tc::EPI_F32,
          epi_plain(c->dlogits, dm.Vpad));
   }
-  launch_pdl(c, 1, draft_pick_kernel, dim3(B, dm.R1), 256, 0, dm, c->st, B, (const float*)c->dlogits, logits_out, margin_out);
+  launch_pdl(c, dim3(1, 1, 1), draft_pick_kernel, dim3(B, dm.R1), 256, 0, dm, c->st, B, (const float*)c->dlogits, logits_out, margin_out);
 }
 
 __global__ void verify_load_kernel(Dims dm, SeqState st, int batch, const int* __restrict__ cand) {
