@@ -68,7 +68,7 @@ struct fm_ctx {
   int attn_chunk, attn_G[3], attn_max_groups[3], attn_mt[3];
   CUtensorMap* tmaps;                    // device array
   std::vector<CUtensorMap> tmaps_host;
-  struct TmapKey { const void* base; uint64_t rows, cols; uint32_t box_rows; };
+  struct TmapKey { const void* base; uint64_t rows, cols; uint32_t box_rows; uint32_t parts; };   // parts = 0: 2-D map
   std::vector<TmapKey> tmap_keys;
   size_t tmaps_cap, tmaps_uploaded;
   // per-tile sums of squares of the residual rows (RMSNorm statistics handed between GEMMs)
@@ -92,6 +92,7 @@ struct fm_ctx {
   double prof_ms[3], prof_bytes[3];
   long long prof_n[3];
   int split_target;     // CTAs a GEMM launch aims for (M tiles x K splits)
+  int stage_cap;        // tuning knob: upper bound on the GEMM ring depth (0 = none)
   int launch_error;     // first error met while enqueueing (capacity, descriptor creation)
   // one decode pass (draft, teacher edit, verify, accept) captured as a CUDA graph
   cudaGraph_t graph;
@@ -200,8 +201,9 @@ void carve(fm_ctx* c, Carver& cv) {
   c->ssq_ld = (int)Rc;
   c->ssq = cv.take<float>((size_t)((d + 127) / 128) * tc::MAX_SPLIT * Rc);
   c->logits = cv.take<float>(Rc * dm.Vpad); c->tmp3d = cv.take<float>(Rv * 3 * d);
-  c->a_norm = cv.take<bf16>(Rc * d); c->a_cat = cv.take<bf16>(Rv * 3 * d);
-  c->a_attn = cv.take<bf16>(Rc * hd); c->a_ff = cv.take<bf16>(Rc * dm.dff);
+  // GEMM operand rows of the backbone hold two bfloat16 terms per value: [hi | lo]
+  c->a_norm = cv.take<bf16>(Rc * 2 * d); c->a_cat = cv.take<bf16>(Rv * 6 * d);
+  c->a_attn = cv.take<bf16>(Rc * 2 * hd); c->a_ff = cv.take<bf16>(Rc * 2 * dm.dff);
   c->hc_ring = cv.take<float>(B * FM_RING_C * d); c->hv_ring = cv.take<float>(B * FM_RING_V * d);
   c->trif_ring = cv.take<float>(B * FM_RING_F * 3 * d); c->triv_ring = cv.take<float>(B * FM_RING_V * 3 * d);
   c->zc = cv.take<float>(B * FM_RING_C * d); c->zv = cv.take<float>(B * FM_RING_V * d);
@@ -362,17 +364,36 @@ int add_tmap_bf16(fm_ctx* c, const void* base, uint64_t rows, uint64_t cols, uin
   return (int)c->tmaps_host.size() - 1;
 }
 
+// GEMM operand rows [rows, parts * K] bf16 seen as a 3-D tensor (K, rows, parts): box 64 columns x
+// box_rows rows x parts, 128-byte swizzle, so that one copy brings the hi and the lo tile of a K slab,
+// one tile after the other.
+int add_tmap_operand(fm_ctx* c, const void* base, uint64_t rows, uint64_t K, uint32_t parts, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (fn == nullptr) return -1;
+  CUtensorMap m;
+  const cuuint64_t gdim[3] = {K, rows, parts};
+  const cuuint64_t gstride[2] = {parts * K * 2, K * 2};
+  const cuuint32_t box[3] = {64, box_rows, parts};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  if (fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), gdim, gstride, box, estr,
+         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return -1;
+  c->tmaps_host.push_back(m);
+  return (int)c->tmaps_host.size() - 1;
+}
+
 // index of the tensor map for a bf16 matrix / box, created on first use (all call sites are
 // visited by the first pass, before any timing or capture)
-int tmap_for(fm_ctx* c, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+int tmap_for(fm_ctx* c, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t parts) {
   for (size_t i = 0; i < c->tmap_keys.size(); ++i) {
     const auto& k = c->tmap_keys[i];
-    if (k.base == base && k.rows == rows && k.cols == cols && k.box_rows == box_rows) return (int)i;
+    if (k.base == base && k.rows == rows && k.cols == cols && k.box_rows == box_rows && k.parts == parts) return (int)i;
   }
   if (c->tmaps_host.size() >= c->tmaps_cap || c->capturing) return -1;   // descriptors are made before capture
-  const int idx = add_tmap_bf16(c, base, rows, cols, box_rows);
+  const int idx = add_tmap_operand(c, base, rows, cols, parts, box_rows);
   if (idx < 0) return -1;
-  c->tmap_keys.push_back({base, rows, cols, box_rows});
+  c->tmap_keys.push_back({base, rows, cols, box_rows, parts});
   cudaMemcpyAsync(c->tmaps + idx, &c->tmaps_host[idx], sizeof(CUtensorMap), cudaMemcpyHostToDevice, c->stream);
   cudaStreamSynchronize(c->stream);
   return idx;
@@ -405,8 +426,13 @@ void launch_pdl(fm_ctx* c, dim3 cluster, void (*kern)(KArgs...), dim3 grid, dim3
   }
   cfg.attrs = at;
   cfg.numAttrs = n;
-  if (cudaLaunchKernelEx(&cfg, kern, std::forward<CArgs>(args)...) != cudaSuccess && c->launch_error == FM_OK)
-    c->launch_error = FM_ERR_CUDA;
+  const cudaError_t err = cudaLaunchKernelEx(&cfg, kern, std::forward<CArgs>(args)...);
+  if (err != cudaSuccess) {
+    if (getenv("FM_DEBUG") != nullptr)
+      fprintf(stderr, "flashmesh: launch failed: %s (grid %u %u %u, block %u, smem %zu, cluster %u %u %u)\n", cudaGetErrorString(err),
+              grid.x, grid.y, grid.z, block.x, smem, cluster.x, cluster.y, cluster.z);
+    if (c->launch_error == FM_OK) c->launch_error = FM_ERR_CUDA;
+  }
   c->launches++;
 }
 
@@ -419,35 +445,37 @@ tc::Epi epi_plain(void* out, int ldo) {
 
 // y[n][m] = W[w_row0 + m, :] . A[a_row0 + n, :], n < R, m < M, finished by the epilogue `mode`
 // (see fm_gemm_tc.cuh).  W: packed weight slabs of a matrix with K columns (w_row0 a multiple of
-// 128), A: [a_rows_alloc, K] bf16 (rows padded to 16).  The K split (= cluster size) depends on
-// (M, K) only.
+// 128), A: [a_rows_alloc, a_parts * K] bf16 (rows padded to 16; a_parts = 2: [hi | lo] terms).  The
+// K split (= cluster size) depends on the shapes only.
 void gemm(fm_ctx* c, const bf16* W, size_t w_rows_alloc, int w_row0, const bf16* A, size_t a_rows_alloc, int a_row0,
-          int M, int K, int R, const int* n_active, int mode, tc::Epi e) {
+          int M, int K, int R, const int* n_active, int mode, tc::Epi e, int a_parts = 1) {
   if (R <= 0) return;
-  const int tiles = (M + tc::BM - 1) / tc::BM, slabs = K / tc::BK;
-  int split = 1;
-  while (split * 2 <= tc::MAX_SPLIT && split * 2 <= slabs && tiles * split * 2 <= c->split_target) split *= 2;
-  const int Rpad = round_up(R, 16);
   (void)w_rows_alloc;
   if (w_row0 % tc::BM != 0) { c->launch_error = FM_ERR_UNSUPPORTED; return; }
+  const int tiles = (M + tc::BM - 1) / tc::BM, slabs = K / tc::BK;
+  // Few rows: one N tile, K split over a cluster so that enough SMs stream weights.  Many rows:
+  // N tiles of 32 rows as well (each weight slab then comes from HBM once and from L2 for the other
+  // N tiles), which keeps the K split, and with it the cluster reduction, small.
+  const int Rpad = round_up(R, 16);
+  const int N = Rpad <= 32 ? Rpad : 32;
+  const int n_tiles = (Rpad + N - 1) / N;
+  int split = 1;
+  while (split * 2 <= tc::MAX_SPLIT && split * 2 <= slabs && tiles * n_tiles * split * 2 <= c->split_target) split *= 2;
+  const int tA = tmap_for(c, A, a_rows_alloc, (uint64_t)K, N, (uint32_t)a_parts);
+  if (tA < 0) { c->launch_error = FM_ERR_CUDA; return; }
+  int stages = tc::pick_stages(N, (slabs + split - 1) / split, a_parts);
+  if (c->stage_cap > 0 && stages > c->stage_cap) stages = c->stage_cap;
   const long pi = prof_open(c, PROF_GEMM, 2.0 * M * K);            // algorithmic bytes: the weight matrix once
-  for (int n0 = 0; n0 < Rpad; n0 += tc::MAX_N) {                   // N tiles of at most MAX_N rows
-    const int N = Rpad - n0 < tc::MAX_N ? Rpad - n0 : tc::MAX_N;
-    const int tA = tmap_for(c, A, a_rows_alloc, K, N);
-    if (tA < 0) { c->launch_error = FM_ERR_CUDA; break; }
-    const int stages = tc::pick_stages(N);
-    tc::Args g{W, c->tmaps + tA, M, K, N, (R - n0 < N ? R - n0 : N), split, stages, w_row0 / tc::BM, a_row0 + n0, n_active,
-               c->st.status};
-    e.row0 = n0;
-    const int smem = tc::smem_bytes(N, stages);
-    const dim3 grid(tiles, split);
-    switch (mode) {
-      case tc::EPI_F32: launch_pdl(c, dim3(1, split, 1), tc::gemm_tc_kernel<tc::EPI_F32>, grid, 128, smem, g, e); break;
-      case tc::EPI_BF16: launch_pdl(c, dim3(1, split, 1), tc::gemm_tc_kernel<tc::EPI_BF16>, grid, 128, smem, g, e); break;
-      case tc::EPI_GELU: launch_pdl(c, dim3(1, split, 1), tc::gemm_tc_kernel<tc::EPI_GELU>, grid, 128, smem, g, e); break;
-      case tc::EPI_RESID: launch_pdl(c, dim3(1, split, 1), tc::gemm_tc_kernel<tc::EPI_RESID>, grid, 128, smem, g, e); break;
-      default: launch_pdl(c, dim3(1, split, 1), tc::gemm_tc_kernel<tc::EPI_QKV>, grid, 128, smem, g, e); break;
-    }
+  tc::Args g{W, c->tmaps + tA, M, K, N, R, split, stages, a_parts, w_row0 / tc::BM, a_row0, n_active, c->st.status};
+  e.row0 = 0;
+  const int smem = tc::smem_bytes(N, stages, a_parts);
+  const dim3 grid(tiles, split, n_tiles), cl(1, split, 1);
+  switch (mode) {
+    case tc::EPI_F32: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_F32>, grid, 128, smem, g, e); break;
+    case tc::EPI_BF16: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_BF16>, grid, 128, smem, g, e); break;
+    case tc::EPI_GELU: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_GELU>, grid, 128, smem, g, e); break;
+    case tc::EPI_RESID: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_RESID>, grid, 128, smem, g, e); break;
+    default: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_QKV>, grid, 128, smem, g, e); break;
   }
   prof_close(c, pi);
   if (mode == tc::EPI_RESID && e.ssq_out != nullptr) c->ssq_n = tiles * split * (split == 1 ? 2 : 1);     // slots the next consumer adds
@@ -504,20 +532,21 @@ void run_stack(fm_ctx* c, int s, float* x, float* stash_ring, const float* next_
     eq.dm = dm; eq.st = c->st; eq.batch = c->batch; eq.level = level; eq.rope_tab = c->rope_tab;
     eq.q_out = c->qbuf; eq.Kc = L.K; eq.Vc = L.V;
     eq.qscale = (float)(1.4426950408889634 / sqrt((double)dm.dh));   // 1/sqrt(dh) * log2(e)
-    gemm(c, L.Wqkv, pad128(qkvw), 0, c->a_norm, Rc_alloc, 0, qkvw, d, rows, na, tc::EPI_QKV, eq);
+    gemm(c, L.Wqkv, pad128(qkvw), 0, c->a_norm, Rc_alloc, 0, qkvw, d, rows, na, tc::EPI_QKV, eq, 2);
     attention(c, level, L);
     tc::Epi eo{};
-    eo.x = x; eo.ldx = d; eo.add = 1; eo.gain = L.g2; eo.a_out = c->a_norm; eo.lda = d;
+    eo.x = x; eo.ldx = d; eo.add = 1; eo.gain = L.g2; eo.a_out = c->a_norm; eo.lda = 2 * d; eo.lo_off = d;
     eo.ssq_out = c->ssq; eo.ld_ssq_out = c->ssq_ld;
-    gemm(c, L.Wo, pad128(d), 0, c->a_attn, Rc_alloc, 0, d, hd, rows, na, tc::EPI_RESID, eo);
-    tc::Epi e1 = epi_plain(c->a_ff, dm.dff);
+    gemm(c, L.Wo, pad128(d), 0, c->a_attn, Rc_alloc, 0, d, hd, rows, na, tc::EPI_RESID, eo, 2);
+    tc::Epi e1 = epi_plain(c->a_ff, 2 * dm.dff);
+    e1.lo_off = dm.dff;
     e1.ssq_in = c->ssq; e1.ssq_n = c->ssq_n; e1.ld_ssq = c->ssq_ld; e1.inv_d_in = 1.f / d; e1.eps = dm.eps;
-    gemm(c, L.W1, pad128(dm.dff), 0, c->a_norm, Rc_alloc, 0, dm.dff, d, rows, na, tc::EPI_GELU, e1);
+    gemm(c, L.W1, pad128(dm.dff), 0, c->a_norm, Rc_alloc, 0, dm.dff, d, rows, na, tc::EPI_GELU, e1, 2);
     tc::Epi e2 = eo;
     const bool last = l == nl - 1;
     e2.gain = last ? next_gain : c->layers[s][l + 1].g1;
     if (last && !want_a) { e2.a_out = nullptr; e2.ssq_out = nullptr; }
-    gemm(c, L.W2, pad128(d), 0, c->a_ff, Rc_alloc, 0, d, dm.dff, rows, na, tc::EPI_RESID, e2);
+    gemm(c, L.W2, pad128(d), 0, c->a_ff, Rc_alloc, 0, d, dm.dff, rows, na, tc::EPI_RESID, e2, 2);
   }
 }
 
@@ -537,22 +566,22 @@ void forward(fm_ctx* c, float* logits_out) {
   launch_pdl(c, dim3(1, 1, 1), ring_store_kernel, Rc, 128, 0, dm, c->st, B, 0, (const float*)c->xc, c->hc_ring, d);
   launch_pdl(c, dim3(1, 1, 1), shorten_gather_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->hc_ring, c->a_cat);
   tc::Epi es{};
-  es.x = c->xv; es.ldx = d; es.add = 0; es.gain = c->layers[1][0].g1; es.a_out = c->a_norm; es.lda = d;
+  es.x = c->xv; es.ldx = d; es.add = 0; es.gain = c->layers[1][0].g1; es.a_out = c->a_norm; es.lda = 2 * d; es.lo_off = d;
   es.ssq_out = c->ssq; es.ld_ssq_out = c->ssq_ld;
-  gemm(c, c->S_cv, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rv, na + 1, tc::EPI_RESID, es);
+  gemm(c, c->S_cv, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rv, na + 1, tc::EPI_RESID, es, 2);
   run_stack(c, 1, c->xv, nullptr, nullptr, false);
   launch_pdl(c, dim3(1, 1, 1), ring_store_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->xv, c->hv_ring, d);
   launch_pdl(c, dim3(1, 1, 1), shorten_gather_kernel, Rf, 128, 0, dm, c->st, B, 2, (const float*)c->hv_ring, c->a_cat);
   es.x = c->xf; es.gain = c->layers[2][0].g1;
-  gemm(c, c->S_vf, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rf, na + 2, tc::EPI_RESID, es);
+  gemm(c, c->S_vf, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rf, na + 2, tc::EPI_RESID, es, 2);
   run_stack(c, 2, c->xf, c->zf, nullptr, true);                    // leaves bf16(xf) in a_norm
-  gemm(c, c->U_fv, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rf, na + 2, tc::EPI_F32, epi_plain(c->tmp3d, 3 * d));
+  gemm(c, c->U_fv, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rf, na + 2, tc::EPI_F32, epi_plain(c->tmp3d, 3 * d), 2);
   launch_pdl(c, dim3(1, 1, 1), ring_store_kernel, Rf, 128, 0, dm, c->st, B, 2, (const float*)c->tmp3d, c->trif_ring, 3 * d);
   launch_pdl(c, dim3(1, 1, 1), upsample_add_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->hv_ring, (const float*)c->trif_ring, c->xv,
              (const float*)c->layers[3][0].g1, c->a_norm, c->ssq);
   c->ssq_n = 1;
   run_stack(c, 3, c->xv, c->zv, nullptr, true);                    // leaves bf16(xv) in a_norm
-  gemm(c, c->U_vc, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rv, na + 1, tc::EPI_F32, epi_plain(c->tmp3d, 3 * d));
+  gemm(c, c->U_vc, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rv, na + 1, tc::EPI_F32, epi_plain(c->tmp3d, 3 * d), 2);
   launch_pdl(c, dim3(1, 1, 1), ring_store_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->tmp3d, c->triv_ring, 3 * d);
   launch_pdl(c, dim3(1, 1, 1), upsample_add_kernel, Rc, 128, 0, dm, c->st, B, 0, (const float*)c->hc_ring, (const float*)c->triv_ring, c->xc,
              (const float*)c->layers[4][0].g1, c->a_norm, c->ssq);
@@ -560,7 +589,7 @@ void forward(fm_ctx* c, float* logits_out) {
   run_stack(c, 4, c->xc, c->zc, c->g_out, true);                   // leaves bf16(xc * g_out) and its sums of squares
   tc::Epi el = epi_plain(c->logits, dm.Vpad);
   el.ssq_in = c->ssq; el.ssq_n = c->ssq_n; el.ld_ssq = c->ssq_ld; el.inv_d_in = 1.f / d; el.eps = dm.eps;
-  gemm(c, c->W_out, dm.Vpad, 0, c->a_norm, Rc_alloc, 0, dm.V, d, Rc, na, tc::EPI_F32, el);
+  gemm(c, c->W_out, dm.Vpad, 0, c->a_norm, Rc_alloc, 0, dm.V, d, Rc, na, tc::EPI_F32, el, 2);
   launch_pdl(c, dim3(1, 1, 1), verify_top2_kernel, Rc, 256, 0, dm, c->st, B, (const float*)c->logits, logits_out);
 }
 
@@ -763,17 +792,17 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
       const uint64_t rows = (uint64_t)dm.max_batch * dm.Hkv * (dm.P + dm.cap[STACK_LEVEL[s]]);
       const uint32_t box = (uint32_t)c->attn_chunk;
       L.tmK = add_tmap_bf16(c, L.K, rows, dm.dh, box);
-      c->tmap_keys.push_back({L.K, rows, (uint64_t)dm.dh, box});
+      c->tmap_keys.push_back({L.K, rows, (uint64_t)dm.dh, box, 0u});
       L.tmV = add_tmap_bf16(c, L.V, rows, dm.dh, box);
-      c->tmap_keys.push_back({L.V, rows, (uint64_t)dm.dh, box});
+      c->tmap_keys.push_back({L.V, rows, (uint64_t)dm.dh, box, 0u});
       if (L.tmK < 0 || L.tmV < 0) { delete c; return FM_ERR_CUDA; }
     }
   TRYCUDA(cudaMemcpy(c->tmaps, c->tmaps_host.data(), c->tmaps_host.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice));
-  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(tc::MAX_N, tc::pick_stages(tc::MAX_N))));
-  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(tc::MAX_N, tc::pick_stages(tc::MAX_N))));
-  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_GELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(tc::MAX_N, tc::pick_stages(tc::MAX_N))));
-  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(tc::MAX_N, tc::pick_stages(tc::MAX_N))));
-  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::smem_bytes(tc::MAX_N, tc::pick_stages(tc::MAX_N))));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_GELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
   TRYCUDA(cudaFuncSetAttribute(attn_stream_kernel<64, 128, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<64, 128, 8>::BYTES));
   TRYCUDA(cudaFuncSetAttribute(attn_stream_kernel<128, 64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<128, 64, 4>::BYTES));
   std::vector<double> freq(dm.dh / 2);
@@ -799,6 +828,8 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
     c->use_pdl = !(v != nullptr && v[0] == '1');
     const char* t = getenv("FM_SPLIT_TARGET");
     c->split_target = t != nullptr && atoi(t) > 0 ? atoi(t) : 160;
+    const char* sc = getenv("FM_STAGE_CAP");
+    c->stage_cap = sc != nullptr ? atoi(sc) : 4;        // measured: deeper rings cost more than they prefetch
   }
   *out = c;
   return FM_OK;

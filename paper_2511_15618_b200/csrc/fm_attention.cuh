@@ -32,7 +32,7 @@ struct AttnArgs {
   const CUtensorMap* tmV;
   float* part;                // [B*Hkv*MT, max_groups, 16, dh + 2]
   int* ticket;                // [B*Hkv*MT], zero between launches
-  bf16* out;                  // [rows, H*dh]
+  bf16* out;                  // [rows, 2*H*dh]: the next GEMM's operand rows as [hi | lo] bfloat16 terms
   int G;                      // chunks per group
   int max_groups;             // groups the cache of this level can hold (= gridDim.x)
   int MT;                     // 16-row query tiles per (sequence, kv-head)
@@ -54,6 +54,11 @@ struct AttnCfg {
 };
 
 namespace attn {
+__device__ inline void store_out(bf16* out, size_t at, float v, int lo_off) {
+  const bf16 hi = __float2bfloat16(v);
+  out[at] = hi;
+  out[at + lo_off] = __float2bfloat16(v - __bfloat162float(hi));
+}
 __device__ inline int div_ratio(int x, int level) { return level == 0 ? x : (level == 1 ? x / 3 : x / 9); }
 }  // namespace attn
 
@@ -339,7 +344,7 @@ __global__ void __launch_bounds__((NW + 1) * 32) attn_stream_kernel(const AttnAr
       const int idx = mt * 16 + i;
       if (idx >= M) continue;
       const int r = group == 1 ? idx : idx / group, gh = idx - r * group;
-      a.out[((size_t)(b * m_rows + r) * dm.H + hk * group + gh) * DH + c] = __float2bfloat16(res[e] / res[16 * DH + i]);
+      attn::store_out(a.out, ((size_t)(b * m_rows + r) * 2 * dm.H + hk * group + gh) * DH + c, res[e] / res[16 * DH + i], dm.H * DH);
     }
     return;
   }
@@ -404,7 +409,7 @@ __global__ void __launch_bounds__((NW + 1) * 32) attn_stream_kernel(const AttnAr
     for (int ck = 0; ck < n_groups; ++ck) acc += wr[ck] * pr[ck * gstride];   // group order
     const int idx = mt * 16 + i;
     const int r = group == 1 ? idx : idx / group, gh = idx - r * group;
-    a.out[((size_t)(b * m_rows + r) * dm.H + hk * group + gh) * DH + c] = __float2bfloat16(acc / wr[n_groups]);
+    attn::store_out(a.out, ((size_t)(b * m_rows + r) * 2 * dm.H + hk * group + gh) * DH + c, acc / wr[n_groups], dm.H * DH);
   }
   if (threadIdx.x == 0) a.ticket[pt] = 0;
 }

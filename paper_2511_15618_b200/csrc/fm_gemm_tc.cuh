@@ -11,6 +11,11 @@
 // 16 KB bulk copies; the token rows come through a TMA tensor map.  A ring of shared-memory stages
 // decouples the copies from the one thread that issues the MMAs; accumulators live in tensor
 // memory and are read back with tcgen05.ld.
+// Operand rows may come as two bfloat16 terms per value, [hi | lo] side by side (hi = bf16(v),
+// lo = bf16(v - hi)): the hi tile and the lo tile of a slab then sit one after the other in shared
+// memory and form one operand of 2N rows, so each weight slab is still read once; the two
+// products land in separate accumulator columns and are added when the accumulator is read.  This
+// removes the rounding of the activations from the error budget at no cost in weight traffic.
 // The work is bandwidth bound: the grid is (M/128 tiles) x (S splits of K) so that many SMs
 // stream weights.  The S CTAs of one M tile form a thread-block cluster: every CTA owns 1/S of the
 // tile's columns; each CTA sends the columns of its partial tile to their owners' shared memory
@@ -41,11 +46,12 @@ enum EpiMode { EPI_F32 = 0, EPI_BF16 = 1, EPI_GELU = 2, EPI_RESID = 3, EPI_QKV =
 
 struct Args {
   const bf16* W;                 // packed weight slabs: [M tile][K slab][128 x 64 swizzled image]
-  const CUtensorMap* tmA;        // [rows, K] bf16, box N x 64
-  int M, K, N;                   // N = padded rows in the box (multiple of 16, <= MAX_N)
-  int n_store;                   // rows actually stored (<= N)
+  const CUtensorMap* tmA;        // operand rows [rows, a_parts * K] bf16 as (K, rows, parts), box 64 x N x a_parts
+  int M, K, N;                   // N = token rows per CTA = rows of the operand box (multiple of 16, <= MAX_N)
+  int n_store;                   // rows of the launch; N tile z (= blockIdx.z) covers rows [z*N, z*N + N)
   int split;                     // K splits = gridDim.y = cluster size (1, 2, 4 or 8)
   int stages;                    // depth of the shared-memory ring (2..MAX_STAGES)
+  int a_parts;                   // 1: plain bf16 operand rows, 2: hi + lo terms
   int w_tile0, a_row0;           // first M tile inside W (stacked matrices), first operand row
   const int* n_active;           // skip when *n_active == 0 (may be null); must not change during a pass
   int* status;
@@ -57,6 +63,8 @@ struct Epi {
   int ssq_n, ld_ssq;
   float inv_d_in, eps;
   void* out; int ldo;            // EPI_F32 / EPI_BF16 / EPI_GELU
+  int lo_off;                    // bf16 outputs (out of EPI_BF16 / EPI_GELU, a_out of EPI_RESID): when > 0 the
+                                 // lo term of every value is stored lo_off elements behind its hi term
   float* x; int ldx; int add;    // EPI_RESID: residual stream, add = 0 replaces it
   const float* gain;             //            gain of the next norm (null = 1)
   bf16* a_out; int lda;          //            next GEMM's operand rows (may be null)
@@ -145,13 +153,27 @@ __device__ inline uint32_t map_peer(uint32_t local_addr, uint32_t rank) {
 // receive buffer of the cluster reduction [split][64/split][2][N + 4] fp32 = (N + 4) * 512 bytes
 // (peers write into it while this CTA may still be multiplying, so it never aliases the ring;
 // the 4 floats of padding spread the readers over the banks), then barriers.
-inline int stage_bytes(int N) { return BM * 128 + ((N * 128 + 1023) / 1024) * 1024; }
-inline int pick_stages(int N) {
-  int st = (200 * 1024 - (N + 4) * 512) / stage_bytes(N);
-  st = st > 4 ? 4 : st;
+inline int stage_bytes(int N, int parts) { return BM * 128 + parts * (((N * 128 + 1023) / 1024) * 1024); }
+// as many stages as the CTA has slabs (its whole K range is then requested at once), at most 8
+// and what fits beside the receive buffer
+inline int pick_stages(int N, int n_slabs, int parts) {
+  int st = (200 * 1024 - (N + 4) * 512) / stage_bytes(N, parts);
+  st = st > MAX_STAGES ? MAX_STAGES : st;
+  st = st > n_slabs ? n_slabs : st;
   return st < 2 ? 2 : st;
 }
-inline int smem_bytes(int N, int stages) { return stages * stage_bytes(N) + (N + 4) * 512 + 1024 + 256; }
+inline int smem_bytes(int N, int stages, int parts) { return stages * stage_bytes(N, parts) + (N + 4) * 512 + 1024 + 256; }
+
+inline int max_smem_bytes() {
+  const int a = smem_bytes(32, pick_stages(32, MAX_STAGES, 1), 1), b = smem_bytes(32, pick_stages(32, MAX_STAGES, 2), 2);
+  return a > b ? a : b;
+}
+
+__device__ inline void store_hi_lo(bf16* p, float v, int lo_off) {
+  const bf16 hi = __float2bfloat16(v);
+  p[0] = hi;
+  if (lo_off > 0) p[lo_off] = __float2bfloat16(v - __bfloat162float(hi));
+}
 
 __device__ inline float gelu_erf_f(float x) { return 0.5f * x * (1.f + erff(x * 0.70710678118654752f)); }
 
@@ -163,7 +185,7 @@ __device__ inline void pair_cols(int q, bool head128, int& ca, int& cb) {
   else { ca = (q >> 5) * 64 + (q & 31); cb = ca + 32; }
 }
 
-// grid (M/128 tiles, split), cluster (1, split, 1); block 128.  Warp 0 lane 0 feeds TMA, warp 1
+// grid (M/128 tiles, split, N tiles of the token rows), cluster (1, split, 1); block 128.  Warp 0 lane 0 feeds TMA, warp 1
 // lane 0 issues MMAs, all four warps read the accumulator back (warp w owns TMEM lanes 32w..32w+31).
 template <int MODE>
 __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e) {
@@ -176,7 +198,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int STAGES = g.stages;
   const int b_bytes = ((g.N * 128 + 1023) / 1024) * 1024;
-  const int stage_bytes = BM * 128 + b_bytes;
+  const int stage_bytes = BM * 128 + g.a_parts * b_bytes;
   const int NP = g.N + 4;
   float* recv = reinterpret_cast<float*>(sm + STAGES * stage_bytes);          // [S][PW][2][NP]
   uint64_t* full = reinterpret_cast<uint64_t*>(sm + STAGES * stage_bytes + NP * 512);
@@ -190,13 +212,18 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tile_m = blockIdx.x;
+  // token rows of this CTA: N tile blockIdx.z of the launch's rows
+  const int row_lo = (int)blockIdx.z * g.N;
+  const int ns = min(g.N, g.n_store - row_lo);               // rows of this tile that exist
+  const int row0 = e.row0 + row_lo;                        // first output row
+  const int a_row = g.a_row0 + row_lo;                     // first operand row
   const int S = g.split;
   const int z = (int)cluster_rank();                 // == blockIdx.y: the cluster spans the grid's y extent
   const int slabs = g.K / BK;
   const int s0 = (int)((long long)slabs * z / S), s1 = (int)((long long)slabs * (z + 1) / S);
   const int n_slabs = s1 - s0;
   uint32_t ncols = 32;
-  while ((int)ncols < g.N) ncols <<= 1;
+  while ((int)ncols < g.a_parts * g.N) ncols <<= 1;
 
   if (tid == 0) {
     s_fail = 0;
@@ -205,14 +232,14 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
     ptx::mbar_init(rbar, 1);
     ptx::fence_mbar_init();
     // rows are sent in groups of 16: groups x 16 rows x 128/S columns x S ranks x 4 bytes
-    ptx::mbar_expect_tx(rbar, (uint32_t)((g.n_store + 15) / 16) * 16u * 512u);
+    ptx::mbar_expect_tx(rbar, (uint32_t)((ns + 15) / 16) * 16u * 512u);
     ptx::prefetch_tmap(g.tmA);
     // The weight slabs of the first stages do not depend on the previous kernel: request them at
     // once, so that they travel while the rest of the prologue runs.
     const bf16* wsrc = g.W + ((size_t)(g.w_tile0 + tile_m) * slabs + s0) * (BM * BK);
     const int pre = n_slabs < STAGES ? n_slabs : STAGES;
     for (int i = 0; i < pre; ++i) {
-      ptx::mbar_expect_tx(full + i, BM * 128 + g.N * 128);
+      ptx::mbar_expect_tx(full + i, BM * 128 + g.a_parts * g.N * 128);
       ptx::bulk_load(sm + i * stage_bytes, wsrc + (size_t)i * (BM * BK), BM * 128, full + i);
     }
   }
@@ -232,25 +259,28 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   // CTA of the cluster runs and has initialised them.
   if (S > 1) cluster_sync();
 
-  if (warp == 0 && lane == 0) {
-    // ---- producer: stream this CTA's K range through the stage ring (the weight slabs of the
-    // first stages are already on their way)
-    const bf16* wsrc = g.W + ((size_t)(g.w_tile0 + tile_m) * slabs + s0) * (BM * BK);
+  if (warp == 0) {
+    // ---- operand rows of the first stages (their weight slabs are already on their way): one
+    // copy per slab brings the hi and the lo tile; lanes issue them side by side
     const int pre = n_slabs < STAGES ? n_slabs : STAGES;
     ptx::grid_dep_wait();
-    for (int i = 0; i < pre; ++i)
-      ptx::tma_load_2d(sm + i * stage_bytes + BM * 128, g.tmA, (s0 + i) * BK, g.a_row0, full + i);
+    if (lane < pre) ptx::tma_load_3d(sm + lane * stage_bytes + BM * 128, g.tmA, (s0 + lane) * BK, a_row, 0, full + lane);
+  }
+  if (warp == 0 && lane == 0) {
+    // ---- producer: stream the rest of this CTA's K range through the stage ring
+    const bf16* wsrc = g.W + ((size_t)(g.w_tile0 + tile_m) * slabs + s0) * (BM * BK);
+    const int pre = n_slabs < STAGES ? n_slabs : STAGES;
     for (int i = pre; i < n_slabs; ++i) {
       const int st = i % STAGES;
       if (!ptx::mbar_wait(empty + st, ((i / STAGES) - 1) & 1)) { s_fail = 1; break; }
       unsigned char* a_dst = sm + st * stage_bytes;
-      ptx::mbar_expect_tx(full + st, BM * 128 + g.N * 128);
+      ptx::mbar_expect_tx(full + st, BM * 128 + g.a_parts * g.N * 128);
       ptx::bulk_load(a_dst, wsrc + (size_t)i * (BM * BK), BM * 128, full + st);
-      ptx::tma_load_2d(a_dst + BM * 128, g.tmA, (s0 + i) * BK, g.a_row0, full + st);
+      ptx::tma_load_3d(a_dst + BM * 128, g.tmA, (s0 + i) * BK, a_row, 0, full + st);
     }
   } else if (warp == 1 && lane == 0) {
     // ---- MMA issuer
-    const uint32_t idesc = instr_desc_bf16(g.N);
+    const uint32_t idesc = instr_desc_bf16(g.a_parts * g.N);   // hi and lo tiles: one operand of 2N rows
     for (int i = 0; i < n_slabs; ++i) {
       const int st = i % STAGES;
       if (!ptx::mbar_wait(full + st, (i / STAGES) & 1)) { s_fail = 1; break; }
@@ -272,31 +302,31 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
     const int t = tid - 64;
     if (e.ssq_in != nullptr) {
       const int sub = t & 7;
-      for (int n0 = 0; n0 < g.n_store; n0 += 8) {
+      for (int n0 = 0; n0 < ns; n0 += 8) {
         const int n = n0 + (t >> 3);
         float v[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const int slot = sub + 8 * k;
-          v[k] = (n < g.n_store && slot < e.ssq_n) ? __ldcg(e.ssq_in + (size_t)slot * e.ld_ssq + e.row0 + n) : 0.f;
+          v[k] = (n < ns && slot < e.ssq_n) ? __ldcg(e.ssq_in + (size_t)slot * e.ld_ssq + row0 + n) : 0.f;
         }
         float ss = 0.f;
 #pragma unroll
         for (int k = 0; k < 8; ++k) ss += v[k];
         for (int slot = sub + 64; slot < e.ssq_n; slot += 8)             // more than 64 slots: not expected
-          ss += (n < g.n_store) ? __ldcg(e.ssq_in + (size_t)slot * e.ld_ssq + e.row0 + n) : 0.f;
+          ss += (n < ns) ? __ldcg(e.ssq_in + (size_t)slot * e.ld_ssq + row0 + n) : 0.f;
         ss += __shfl_xor_sync(0xffffffffu, ss, 1);
         ss += __shfl_xor_sync(0xffffffffu, ss, 2);
         ss += __shfl_xor_sync(0xffffffffu, ss, 4);
-        if (sub == 0 && n < g.n_store) s_inv[n] = rsqrtf(ss * e.inv_d_in + e.eps);
+        if (sub == 0 && n < ns) s_inv[n] = rsqrtf(ss * e.inv_d_in + e.eps);
       }
     } else {
-      for (int n = t; n < g.n_store; n += 64) s_inv[n] = 1.f;
+      for (int n = t; n < ns; n += 64) s_inv[n] = 1.f;
     }
     if (MODE == EPI_QKV) {
-      for (int n = t; n < g.n_store; n += 64) {
+      for (int n = t; n < ns; n += 64) {
         int b, p;
-        const bool valid = fm_row_map(e.dm, e.st, e.batch, e.level, e.row0 + n, b, p);
+        const bool valid = fm_row_map(e.dm, e.st, e.batch, e.level, row0 + n, b, p);
         s_rb[n] = valid ? b : -1;
         s_rp[n] = p;
       }
@@ -311,14 +341,18 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   const int lgS = 31 - __clz(S);                           // S is 1, 2, 4 or 8
   const int lgPW = 6 - lgS, PW = 1 << lgPW;
   const bool head128 = MODE == EPI_QKV && e.dm.dh == 128;
-  const int items = g.n_store * PW;
-  uint32_t dst0, dbar;
+  const int items = ns * PW;
+  uint32_t dst0 = 0, dbar = 0;
+  float* recv_own;                                         // S == 1: this thread's row run in the local buffer
   {
     const int q = head128 ? (tid & 63) : ((tid >> 6) * 32 + (tid & 31));
     const int h = head128 ? (tid >> 6) : ((tid >> 5) & 1);
     const int owner = q >> lgPW, cc = q & (PW - 1);
-    dst0 = map_peer(ptx::smem_u32(recv + (((size_t)z * PW + cc) * 2 + h) * NP), (uint32_t)owner);
-    dbar = map_peer(ptx::smem_u32(rbar), (uint32_t)owner);
+    recv_own = recv + (((size_t)z * PW + cc) * 2 + h) * NP;
+    if (S > 1) {
+      dst0 = map_peer(ptx::smem_u32(recv_own), (uint32_t)owner);
+      dbar = map_peer(ptx::smem_u32(rbar), (uint32_t)owner);
+    }
   }
   float pre_ga = 1.f, pre_gb = 1.f;
   float2 pre_cs = make_float2(1.f, 0.f);
@@ -333,15 +367,15 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
     }
     if (MODE == EPI_QKV && e.dm.theta != 0.f) {
       int b, p;
-      const bool valid = fm_row_map(e.dm, e.st, e.batch, e.level, e.row0 + n, b, p);
+      const bool valid = fm_row_map(e.dm, e.st, e.batch, e.level, row0 + n, b, p);
       const int head = ma / e.dm.dh, i = ma - head * e.dm.dh;
       if (valid && ma < g.M && head < e.dm.H + e.dm.Hkv) pre_cs = e.rope_tab[(size_t)p * (e.dm.dh >> 1) + i];
     }
   }
   // Kernel parameters the tail needs, read into registers now: a first touch of the parameter
   // bank after the wait would sit on the critical path.
-  int k_row0 = e.row0, k_ldo = e.ldo, k_ldx = e.ldx, k_add = e.add, k_lda = e.lda, k_ldssq = e.ld_ssq_out;
-  int k_M = g.M, k_ns = g.n_store;
+  int k_row0 = row0, k_ldo = e.ldo, k_ldx = e.ldx, k_add = e.add, k_lda = e.lda, k_ldssq = e.ld_ssq_out;
+  int k_M = g.M, k_ns = ns, k_lo = e.lo_off;
   void* k_out = e.out;
   float* k_x = e.x;
   const float* k_gain = e.gain;
@@ -352,7 +386,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   float k_qs = e.qscale, k_theta = e.dm.theta;
   int k_H = e.dm.H, k_Hkv = e.dm.Hkv, k_dh = e.dm.dh, k_P = e.dm.P, k_cap = MODE == EPI_QKV ? e.dm.cap[e.level] : 1;
   int* k_status = g.status;
-  asm volatile("" : "+r"(k_row0), "+r"(k_ldo), "+r"(k_ldx), "+r"(k_add), "+r"(k_lda), "+r"(k_ldssq), "+r"(k_M), "+r"(k_ns));
+  asm volatile("" : "+r"(k_row0), "+r"(k_ldo), "+r"(k_ldx), "+r"(k_add), "+r"(k_lda), "+r"(k_ldssq), "+r"(k_M), "+r"(k_ns), "+r"(k_lo));
   asm volatile("" : "+l"(k_out), "+l"(k_x), "+l"(k_gain), "+l"(k_aout), "+l"(k_ssqo), "+l"(k_q), "+l"(k_K), "+l"(k_V), "+l"(k_rope), "+l"(k_status));
   asm volatile("" : "+f"(k_qs), "+f"(k_theta), "+r"(k_H), "+r"(k_Hkv), "+r"(k_dh), "+r"(k_P), "+r"(k_cap));
   ptx::grid_dep_wait();                                    // everything below touches activations
@@ -375,15 +409,30 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   fence_after();
   for (int n0 = 0; n0 < k_ns; n0 += 16) {
     uint32_t r[16];
-    if (ok && n_slabs > 0) ld16(tmem + ((uint32_t)(warp * 32) << 16) + n0, r);
-    else {
+    if (ok && n_slabs > 0) {
+      ld16(tmem + ((uint32_t)(warp * 32) << 16) + n0, r);
+      if (g.a_parts == 2) {                                // the lo products: columns N..2N-1
+        uint32_t r2[16];
+        ld16(tmem + ((uint32_t)(warp * 32) << 16) + g.N + n0, r2);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+      }
+    } else {
 #pragma unroll
       for (int j = 0; j < 16; ++j) r[j] = 0u;
     }
+    if (S > 1) {
 #pragma unroll
-    for (int j = 0; j < 16; j += 4) st_async_peer4(dst0 + (uint32_t)(n0 + j) * 4u, r[j], r[j + 1], r[j + 2], r[j + 3], dbar);
+      for (int j = 0; j < 16; j += 4) st_async_peer4(dst0 + (uint32_t)(n0 + j) * 4u, r[j], r[j + 1], r[j + 2], r[j + 3], dbar);
+    } else {                                               // no split: the tile stays in this CTA
+#pragma unroll
+      for (int j = 0; j < 16; j += 4)
+        *reinterpret_cast<uint4*>(recv_own + n0 + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
+    }
   }
-  const bool arrived = mbar_wait_cluster(rbar, 0);
+  bool arrived = true;
+  if (S > 1) arrived = mbar_wait_cluster(rbar, 0);
+  else __syncthreads();
   if (!ok || !arrived || s_fail) {
     if (tid == 0) atomicExch(k_status, -5);
   }
@@ -418,24 +467,24 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
       if (b_ok) o[mb] = yb;
     } else if (MODE == EPI_BF16) {
       bf16* o = reinterpret_cast<bf16*>(k_out) + row * k_ldo;
-      if (a_ok) o[ma] = __float2bfloat16(ya);
-      if (b_ok) o[mb] = __float2bfloat16(yb);
+      if (a_ok) store_hi_lo(o + ma, ya, k_lo);
+      if (b_ok) store_hi_lo(o + mb, yb, k_lo);
     } else if (MODE == EPI_GELU) {
       bf16* o = reinterpret_cast<bf16*>(k_out) + row * k_ldo;
-      if (a_ok) o[ma] = __float2bfloat16(gelu_erf_f(ya));
-      if (b_ok) o[mb] = __float2bfloat16(gelu_erf_f(yb));
+      if (a_ok) store_hi_lo(o + ma, gelu_erf_f(ya), k_lo);
+      if (b_ok) store_hi_lo(o + mb, gelu_erf_f(yb), k_lo);
     } else if (MODE == EPI_RESID) {
       float* xr = k_x + row * k_ldx;
       float xa = 0.f, xb = 0.f;
       if (a_ok) {
         xa = (first ? pre_xa : (k_add ? xr[ma] : 0.f)) + ya;
         xr[ma] = xa;
-        if (k_aout != nullptr) k_aout[row * k_lda + ma] = __float2bfloat16(xa * (first ? pre_ga : (k_gain != nullptr ? k_gain[ma] : 1.f)));
+        if (k_aout != nullptr) store_hi_lo(k_aout + row * k_lda + ma, xa * (first ? pre_ga : (k_gain != nullptr ? k_gain[ma] : 1.f)), k_lo);
       }
       if (b_ok) {
         xb = (first ? pre_xb : (k_add ? xr[mb] : 0.f)) + yb;
         xr[mb] = xb;
-        if (k_aout != nullptr) k_aout[row * k_lda + mb] = __float2bfloat16(xb * (first ? pre_gb : (k_gain != nullptr ? k_gain[mb] : 1.f)));
+        if (k_aout != nullptr) store_hi_lo(k_aout + row * k_lda + mb, xb * (first ? pre_gb : (k_gain != nullptr ? k_gain[mb] : 1.f)), k_lo);
       }
       if (k_ssqo != nullptr) {
         // per-row sums of squares of this rank's columns: a fixed shuffle tree over the L lanes that

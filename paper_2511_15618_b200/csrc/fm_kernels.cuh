@@ -18,9 +18,17 @@ __device__ inline float block_sum(float v, float* sh) {
 }
 
 // ------------------------------------------------------------------------------------------
+// A GEMM operand value as two bfloat16 terms: hi = bf16(v) at p[0], lo = bf16(v - hi) at p[lo_off].
+__device__ inline void store_hi_lo(bf16* p, float v, int lo_off) {
+  const bf16 hi = __float2bfloat16(v);
+  p[0] = hi;
+  p[lo_off] = __float2bfloat16(v - __bfloat162float(hi));
+}
+
 // Hand a freshly written residual row to the first layer of a stack: the GEMM operand row
-// bf16(x * g) (the RMSNorm scale 1/rms is applied by the GEMM's epilogue) and the row's sum of
-// squares in slot 0 of `ssq` (the consumer is told that one slot is filled).
+// x * g as [hi | lo] terms, row length 2d (the RMSNorm scale 1/rms is applied by the GEMM's
+// epilogue) and the row's sum of squares in slot 0 of `ssq` (the consumer is told that one slot is
+// filled).
 // ------------------------------------------------------------------------------------------
 __device__ inline void stack_entry_row(const float* xr, int row, int d, const float* __restrict__ g,
                                        bf16* __restrict__ a_out, float* __restrict__ ssq) {
@@ -29,7 +37,7 @@ __device__ inline void stack_entry_row(const float* xr, int row, int d, const fl
   for (int i = threadIdx.x; i < d; i += blockDim.x) {
     const float v = xr[i];
     ss += v * v;
-    a_out[(size_t)row * d + i] = __float2bfloat16(v * g[i]);
+    store_hi_lo(a_out + (size_t)row * 2 * d + i, v * g[i], d);
   }
   ss = block_sum(ss, sh);
   if (threadIdx.x == 0) ssq[row] = ss;
@@ -118,8 +126,9 @@ __global__ void ring_store_kernel(Dims dm, SeqState st, int batch, int level, co
   for (int i = threadIdx.x; i < width; i += blockDim.x) dst[i] = src[i];
 }
 
-// a3/a5 shorten, gather half: row v of level `level_out` <- bf16 [h_{3v-2}; h_{3v-1}; h_{3v}] from
-// the ring of the level below (zeros for negative positions and for rows that are not fed)
+// a3/a5 shorten, gather half: row v of level `level_out` <- [h_{3v-2}; h_{3v-1}; h_{3v}] from the ring
+// of the level below (zeros for negative positions and for rows that are not fed), as [hi | lo]
+// terms: row length 6d
 __global__ void shorten_gather_kernel(Dims dm, SeqState st, int batch, int level_out, const float* __restrict__ ring,
                                       bf16* __restrict__ out) {
   ptx::grid_dep_launch();
@@ -133,7 +142,7 @@ __global__ void shorten_gather_kernel(Dims dm, SeqState st, int batch, int level
     const bool ok = valid && pos >= 0;
     const float* src = ring + ((size_t)b * rs + ((pos + rs) % rs)) * d;
     for (int i = threadIdx.x; i < d; i += blockDim.x)
-      out[(size_t)row * 3 * d + part * d + i] = __float2bfloat16(ok ? src[i] : 0.f);
+      store_hi_lo(out + (size_t)row * 6 * d + part * d + i, ok ? src[i] : 0.f, 3 * d);
   }
 }
 
