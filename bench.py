@@ -45,6 +45,33 @@ def _fill_prompt(cfg, seq, n_faces):
     return [int(t) for t in np.tile(base, reps)[:9 * n_faces]]
 
 
+def reduce_over_ranks(maxed, summed, device):
+    """Whole-job figures from per-rank ones: element-wise MAX of `maxed` (times) and SUM of
+    `summed` (tokens, launches) over the ranks of the default process group.  Sequences are
+    independent, so this reduction of the report is the only communication of a multi-GPU run."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return list(maxed), list(summed)
+    tm = torch.tensor(list(maxed), dtype=torch.float64, device=device)
+    ts = torch.tensor(list(summed), dtype=torch.float64, device=device)
+    dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+    dist.all_reduce(ts, op=dist.ReduceOp.SUM)
+    return tm.tolist(), ts.tolist()
+
+
+def rank_sequences(rank, batch_per_rank):
+    """Global sequence ids (seeds of conditioning and prompts) owned by a rank: weak scaling, every
+    rank decodes its own `batch_per_rank` sequences."""
+    return [rank * batch_per_rank + b for b in range(batch_per_rank)]
+
+
+# DRAM traffic of the dominant kernel per launch from ncu (dram__bytes_read.sum +
+# dram__bytes_write.sum; profiles/gemm_traffic_medium.md), keyed by workload; None where the kernel
+# changed since the capture or none was taken.
+NCU_TRAFFIC = {"medium": 6.47e6}      # bytes per GEMM launch, mean over the four projections of a layer
+
+
 class ClockSampler:
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -118,12 +145,13 @@ def run_ours(args):
     need_faces = -(-(K + W + 8) * (D + 1) // 9) + 1
     max_tokens = 1 + 9 * (start_faces + cfg.prompt_faces[1] + need_faces) + D + 2
     w = S.make_weights(cfg)
-    conds = np.stack([S.make_condition(cfg, rank * B + b) for b in range(B)])
+    seqs = rank_sequences(rank, B)
+    conds = np.stack([S.make_condition(cfg, q) for q in seqs])
     rng = np.random.default_rng([cfg.seed, 77, rank])
     prompts = []
     for b in range(B):                    # ragged fills around the target (exact for batch 1)
         f = start_faces if B == 1 else max(1, int(start_faces * rng.uniform(0.5, 1.0)))
-        prompts.append(_fill_prompt(cfg, rank * B + b, f))
+        prompts.append(_fill_prompt(cfg, seqs[b], f))
     dev = FlashMesh(cfg, w, device=f"cuda:{local}", max_tokens=max_tokens)
     del w
 
@@ -168,9 +196,17 @@ def run_ours(args):
     assert (got[:, :n_chk] == pt[:, :n_chk]).all(), "speculative output differs from plain decoding"
 
     if args.timed_only:
+        cand, _, _ = dev.draft()
+        dev.verify(cand)
+        _, _, kv = dev.accept()
+        sb = dev.verify_bytes(kv.cpu().numpy().tolist())
+        peak, _ = _peaks()
         if rank == 0:
-            print(json.dumps({"metric": METRIC, "value": emitted / (ms * 1e-3), "ms_per_step": ms / max(1, steps),
-                              "steps": steps, "gpu_launches": launches, "note": "timed passes only"}), flush=True)
+            print(json.dumps({"metric": METRIC, "value": emitted / (ms * 1e-3), "unit": "tokens/s", "workload": args.workload,
+                              "batch": B, "ms_per_step": ms / max(1, steps), "steps": steps, "gpu_launches": launches,
+                              "mean_accept_len": emitted / max(1, steps * B),
+                              "verify_step_frac_of_hbm_peak": sb / (ms / max(1, steps) * 1e-3) / 1e9 / peak,
+                              "note": "timed passes only"}), flush=True)
         return
 
     # ---- the same passes once more with per-kernel-class events (roofline of the dominant kernel)
@@ -197,18 +233,10 @@ def run_ours(args):
     e2e = run_e2e(dev, cfg, truth, keep, prompts, max(8, min(K, 64)))
 
     peak, peak_kind = _peaks()
-    if world > 1:
-        t = torch.tensor([ms, float(emitted), float(launches)], dtype=torch.float64, device="cuda")
-        tmax = t.clone()
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        tsum = t.clone()
-        dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
-        ms, emitted, launches = float(tmax[0]), int(tsum[1]), int(tsum[2])
-        e = torch.tensor([e2e["tokens"], e2e["seconds"]], dtype=torch.float64, device="cuda")
-        emax, esum = e.clone(), e.clone()
-        dist.all_reduce(emax, op=dist.ReduceOp.MAX)
-        dist.all_reduce(esum, op=dist.ReduceOp.SUM)
-        e2e["tokens"], e2e["seconds"] = float(esum[0]), float(emax[1])
+    (ms, e2e_s), (emitted, launches, e2e_tok) = reduce_over_ranks(
+        [ms, e2e["seconds"]], [float(emitted), float(launches), e2e["tokens"]], "cuda")
+    emitted, launches = int(emitted), int(launches)
+    e2e["tokens"], e2e["seconds"] = e2e_tok, e2e_s
     value = emitted / (ms * 1e-3)
     gemm_gbs = prof.gemm_bytes / (prof.gemm_ms * 1e-3) / 1e9 if prof.gemm_ms > 0 else 0.0
     step_ms = ms / max(1, steps)
@@ -234,7 +262,8 @@ def run_ours(args):
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "kernel": "weight-streaming GEMM (all launches of the timed passes)",
                      "achieved": gemm_gbs, "peak": peak, "unit": "GB/s", "frac": gemm_gbs / peak,
-                     "peak_kind": peak_kind, "traffic": None,
+                     "peak_kind": peak_kind, "traffic": NCU_TRAFFIC.get(args.workload),
+                     "algorithmic_bytes_per_launch": prof.gemm_bytes / max(1, prof.gemm_launches),
                      "launches": int(prof.gemm_launches), "ms_per_pass": prof.gemm_ms / max(1, stp.steps),
                      "attention_ms_per_pass": prof.attn_ms / max(1, stp.steps)},
         "verify_step": {"algorithmic_bytes": step_bytes, "ms": step_ms, "GB/s": step_bytes / (step_ms * 1e-3) / 1e9,
@@ -242,6 +271,17 @@ def run_ours(args):
                         "note": "whole pass (draft heads + verify + accept) against the verify bytes"},
     }
     if rank == 0:
+        if world == 1 and args.workload == "medium" and not args.no_batched:
+            # the metric also asks for batch 16: the batched-ragged workload, timed passes only
+            dev.close()
+            del dev
+            torch.cuda.empty_cache()
+            r = subprocess.run([sys.executable, os.path.abspath(__file__), "--workload", "batched", "--steps", "30", "--warmup", "3",
+                                "--timed-only", "--no-cpu"], capture_output=True, text=True)
+            try:
+                line["batch16"] = json.loads(r.stdout.strip().splitlines()[-1])
+            except Exception:
+                line["batch16"] = {"error": (r.stderr or r.stdout)[-300:]}
         if world == 1 and not args.no_cpu:
             line["cpu_baseline"] = cpu_baseline(args.workload, budget_s=args.cpu_seconds)
         print(json.dumps(line), flush=True)
@@ -360,6 +400,7 @@ def main():
     ap.add_argument("--start-frac", type=float, default=0.5, help="fraction of the run already in the caches")
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-batched", action="store_true", help="skip the batch-16 add-on of the default run")
     ap.add_argument("--timed-only", action="store_true", help="stop after the timed passes (for profiler captures)")
     args = ap.parse_args()
     args.warmup = max(3, args.warmup) if args.impl == "ours" else args.warmup

@@ -62,16 +62,8 @@ def test_large_model_lockstep_head_dim_128():
     conds = [S.make_condition(cfg, b) for b in range(B)]
     prompts = [[int(t) for t in S.make_prompt(cfg, b)] for b in range(B)]
     dev = _dev(cfg, w)
-    # float32 oracle: the float64 copy of 2 G parameters would need 16 GB; the two modes agree to 1e-4.
-    # Verify logits are held to the 2e-2 bound.  Draft logits are computed from the split-node
-    # hiddens, which already carry the backbone's accumulated bfloat16 error (measured 1.98e-2 on the
-    # verify logits of this 40-layer, d = 2048 model), and add the heads' own roundings on top:
-    # measured 2.28e-2.  They are checked here against 2.5e-2 and listed as over the bound in the
-    # design notes; draft ids are still compared wherever the oracle's margin is decisive.
-    rep = run_lockstep(cfg, w, conds, prompts, dev, 1, 6, dtype=np.float32, check_drafts=False)
-    assert rep["steps"] == 6 and rep["max_logit_err"] <= 2e-2
-    dev2 = _dev(cfg, w)
-    rep2 = run_lockstep(cfg, w, conds, prompts, dev2, 1, 3, dtype=np.float32, tol=2.5e-2)
-    assert rep2["max_draft_err"] <= 2.5e-2 and rep2["max_logit_err"] <= 2e-2
+    # float32 oracle: the float64 copy of 2 G parameters would need 16 GB; the two modes agree to 1e-4
+    rep = run_lockstep(cfg, w, conds, prompts, dev, 1, 6, dtype=np.float32)
+    assert rep["steps"] == 6 and rep["max_logit_err"] <= 2e-2 and rep["max_draft_err"] <= 2e-2
     assert dev.device_status() == 0
     print(rep)
