@@ -213,6 +213,15 @@ typedef struct fm_profile {
   double attn_ms; int64_t attn_launches;
 } fm_profile;
 int fm_profile_begin(fm_ctx* ctx);
+/* One kernel class timed alone (no counterpart in the paper): the launches of that class of one
+ * verify pass over the current candidates and lengths (cls 0: the weight-streaming GEMMs, 1: the
+ * attention launches; same kernels, arguments and data as in the pass) are captured as a CUDA graph
+ * and replayed `reps` times after 3 warm-up replays, between two events.  out->gemm_ms /
+ * out->attn_ms = milliseconds per replay, *_launches = launches per replay, gemm_bytes = weight bytes
+ * per replay (2*M*K per launch).  Synchronous.  The
+ * replays overwrite activations and the tentative cache rows of the pass: call fm_prefill (or
+ * fm_verify) again before decoding on. */
+int fm_profile_class(fm_ctx* ctx, int32_t cls, int32_t reps, fm_profile* out /*HOST*/);
 int fm_profile_end(fm_ctx* ctx, fm_profile* out /*HOST*/);
 
 /* Number of kernels launched by this context since creation (for launch accounting). */

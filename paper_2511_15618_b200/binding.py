@@ -101,6 +101,8 @@ def load_library():
     lib.fm_profile_begin.argtypes = [vp]
     lib.fm_profile_end.restype = C.c_int
     lib.fm_profile_end.argtypes = [vp, C.POINTER(FmProfile)]
+    lib.fm_profile_class.restype = C.c_int
+    lib.fm_profile_class.argtypes = [vp, i32, i32, C.POINTER(FmProfile)]
     lib.fm_launch_count.restype = C.c_int64
     lib.fm_launch_count.argtypes = [vp]
     lib.fm_strerror.restype = C.c_char_p
@@ -179,6 +181,12 @@ def fm_profile_begin(ctx):
 def fm_profile_end(ctx):
     p = FmProfile()
     rc = load_library().fm_profile_end(ctx, C.byref(p))
+    return rc, p
+
+
+def fm_profile_class(ctx, cls, reps):
+    p = FmProfile()
+    rc = load_library().fm_profile_class(ctx, int(cls), int(reps), C.byref(p))
     return rc, p
 
 
@@ -394,6 +402,14 @@ class FlashMesh:
         rc, p = fm_profile_end(self.ctx)
         self._check(rc, "fm_profile_end")
         return p
+
+    def profile_class(self, cls, reps=20):
+        """Milliseconds and launches per verify pass of one kernel class timed alone (0 GEMM, 1 attention)."""
+        self._before()
+        rc, p = fm_profile_class(self.ctx, cls, reps)
+        self._check(rc, "fm_profile_class")
+        self._after()
+        return (p.gemm_ms, p.gemm_launches, p.gemm_bytes) if cls == 0 else (p.attn_ms, p.attn_launches, 0.0)
 
     def launch_count(self):
         return fm_launch_count(self.ctx)

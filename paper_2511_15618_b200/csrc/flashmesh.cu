@@ -91,6 +91,9 @@ struct fm_ctx {
   size_t prof_used;
   double prof_ms[3], prof_bytes[3];
   long long prof_n[3];
+  int only_class;       // -1, or the kernel class (ProfClass) that alone is launched (fm_profile_class)
+  int cur_class;        // class of the launch being enqueued
+  double class_bytes;   // weight bytes of the GEMM launches enqueued by fm_profile_class
   int split_target;     // CTAs a GEMM launch aims for (M tiles x K splits)
   int stage_cap;        // tuning knob: upper bound on the GEMM ring depth (0 = none)
   int launch_error;     // first error met while enqueueing (capacity, descriptor creation)
@@ -299,6 +302,7 @@ int upload_f32(float* dst, const float* src, size_t n) {
 // ------------------------------------------------------------------------------------------
 #define LAUNCH(ctx, kern, grid, block, smem, ...)                        \
   do {                                                                   \
+    if ((ctx)->only_class >= 0 && (ctx)->cur_class != (ctx)->only_class) break; \
     kern<<<grid, block, smem, (ctx)->stream>>>(__VA_ARGS__);             \
     (ctx)->launches++;                                                   \
   } while (0)
@@ -405,6 +409,7 @@ int tmap_for(fm_ctx* c, const void* base, uint64_t rows, uint64_t cols, uint32_t
 // `cluster` with more than one CTA makes thread-block clusters of that shape.
 template <typename... KArgs, typename... CArgs>
 void launch_pdl(fm_ctx* c, dim3 cluster, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, CArgs&&... args) {
+  if (c->only_class >= 0 && c->cur_class != c->only_class) return;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
@@ -470,6 +475,8 @@ void gemm(fm_ctx* c, const bf16* W, size_t w_rows_alloc, int w_row0, const bf16*
   e.row0 = 0;
   const int smem = tc::smem_bytes(N, stages, a_parts);
   const dim3 grid(tiles, split, n_tiles), cl(1, split, 1);
+  c->cur_class = PROF_GEMM;
+  if (c->only_class == PROF_GEMM) c->class_bytes += 2.0 * M * K;
   switch (mode) {
     case tc::EPI_F32: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_F32>, grid, 128, smem, g, e); break;
     case tc::EPI_BF16: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_BF16>, grid, 128, smem, g, e); break;
@@ -477,25 +484,17 @@ void gemm(fm_ctx* c, const bf16* W, size_t w_rows_alloc, int w_row0, const bf16*
     case tc::EPI_RESID: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_RESID>, grid, 128, smem, g, e); break;
     default: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_QKV>, grid, 128, smem, g, e); break;
   }
+  c->cur_class = PROF_OTHER;
   prof_close(c, pi);
   if (mode == tc::EPI_RESID && e.ssq_out != nullptr) c->ssq_n = tiles * split * (split == 1 ? 2 : 1);     // slots the next consumer adds
 }
 
 // rows fed at each level in this pass (n_active[level]); n_active[3] = unfinished sequences
 __global__ void row_count_kernel(Dims dm, SeqState st, int batch) {
-  if (threadIdx.x != 0 || blockIdx.x != 0) return;
-  int cnt[3] = {0, 0, 0}, act = 0;
-  for (int b = 0; b < batch; ++b) {
-    const int n = st.nrow[b], L = st.L[b];
-    if (n <= 0) continue;
-    act++;
-    for (int l = 0; l < 3; ++l) {
-      const int r = fm_ratio(l);
-      cnt[l] += (L + n - 1) / r - (L + r - 1) / r + 1;
-    }
-  }
-  st.n_active[0] = cnt[0]; st.n_active[1] = cnt[1]; st.n_active[2] = cnt[2]; st.n_active[3] = act;
+  if (threadIdx.x == 0 && blockIdx.x == 0) count_rows(dm, st, batch);
 }
+
+inline int accept_threads(int batch) { return batch >= 32 ? 1024 : 32 * (batch < 1 ? 1 : batch); }
 
 void attention(fm_ctx* c, int level, const LayerDev& L) {
   const Dims& dm = c->dm;
@@ -504,8 +503,10 @@ void attention(fm_ctx* c, int level, const LayerDev& L) {
              c->a_attn, c->attn_G[level], groups, c->attn_mt[level]};
   const dim3 grid(groups, dm.Hkv * c->attn_mt[level], c->batch);
   const long pi = prof_open(c, PROF_ATTN, 0.0);
+  c->cur_class = PROF_ATTN;
   if (dm.dh == 64) launch_pdl(c, dim3(1, 1, 1), attn_stream_kernel<64, 128, 8>, grid, AttnCfg<64, 128, 8>::THREADS, AttnCfg<64, 128, 8>::BYTES, a);
   else launch_pdl(c, dim3(1, 1, 1), attn_stream_kernel<128, 64, 4>, grid, AttnCfg<128, 64, 4>::THREADS, AttnCfg<128, 64, 4>::BYTES, a);
+  c->cur_class = PROF_OTHER;
   prof_close(c, pi);
 }
 
@@ -557,9 +558,9 @@ void forward(fm_ctx* c, float* logits_out) {
   const int Rc = B * dm.R1, Rv = B * dm.mv, Rf = B * dm.mf;
   const size_t Rc_alloc = align_up((size_t)dm.max_batch * dm.R1, 16), Rv_alloc = align_up((size_t)dm.max_batch * dm.mv, 16);
   const int* na = c->st.n_active;
-  // The two launches that open a pass are full barriers: the per-pass state (rows, lengths,
-  // candidates) is final before any later kernel's prologue can run.
-  LAUNCH(c, row_count_kernel, 1, 32, 0, dm, c->st, B);
+  // The launch that opens a pass is a full barrier: the per-pass state (rows, lengths, row counts
+  // -- every call that changes them ends with a row count -- and candidates) is final before any
+  // later kernel's prologue can run.
   LAUNCH(c, embed_kernel, Rc, 128, 0, dm, c->st, B, c->E, c->xc, c->layers[0][0].g1, c->a_norm, c->ssq);
   c->ssq_n = 1;
   run_stack(c, 0, c->xc, nullptr, nullptr, false);
@@ -594,7 +595,7 @@ void forward(fm_ctx* c, float* logits_out) {
 }
 
 // a13: draft heads on the stashed split-node hiddens
-void draft(fm_ctx* c, float* logits_out, float* margin_out) {
+void draft(fm_ctx* c, float* logits_out, float* margin_out, const GenOut* gen) {
   const Dims& dm = c->dm;
   const int B = c->batch, d = dm.d;
   if (dm.D > 0) {
@@ -616,7 +617,7 @@ void draft(fm_ctx* c, float* logits_out, float* margin_out) {
     gemm(c, c->W_out, dm.Vpad, 0, c->feat_n, align_up((size_t)NF * MB, 16), 0, dm.V, d, NF * B, na, tc::EPI_F32,
          epi_plain(c->dlogits, dm.Vpad));
   }
-  launch_pdl(c, dim3(1, 1, 1), draft_pick_kernel, dim3(B, dm.R1), 256, 0, dm, c->st, B, (const float*)c->dlogits, logits_out, margin_out);
+  launch_pdl(c, dim3(1, 1, 1), draft_pick_kernel, dim3(B, dm.R1), 256, 0, dm, c->st, B, (const float*)c->dlogits, logits_out, margin_out, gen);
 }
 
 __global__ void verify_load_kernel(Dims dm, SeqState st, int batch, const int* __restrict__ cand) {
@@ -648,13 +649,10 @@ __global__ void set_limits_kernel(Dims dm, SeqState st, int batch, const int* __
 // one decode pass of fm_generate
 void step_body(fm_ctx* c) {
   const Dims& dm = c->dm;
-  draft(c, nullptr, nullptr);
-  LAUNCH(c, teacher_edit_kernel, c->batch, 32, 0, dm, c->st, c->batch, (const GenOut*)c->gen_dev);
+  draft(c, nullptr, nullptr, (const GenOut*)c->gen_dev);
   forward(c, nullptr);
-  LAUNCH(c, accept_kernel, (c->batch * 32 + 127) / 128, 128, 0, dm, c->st, c->batch, (const int*)nullptr,
-         (const int*)nullptr, (int*)nullptr, (int*)nullptr, (int*)nullptr, (const GenOut*)c->gen_dev);
-  LAUNCH(c, row_count_kernel, 1, 32, 0, dm, c->st, c->batch);
-  LAUNCH(c, step_end_kernel, 1, 32, 0, c->st, (const GenOut*)c->gen_dev);
+  LAUNCH(c, accept_kernel, 1, accept_threads(c->batch), 0, dm, c->st, c->batch, (const int*)nullptr, (const int*)nullptr,
+         (int*)nullptr, (int*)nullptr, (int*)nullptr, (const GenOut*)c->gen_dev, 1);
 }
 
 void drop_graph(fm_ctx* c) {
@@ -670,7 +668,7 @@ void drop_graph(fm_ctx* c) {
 void ensure_graph(fm_ctx* c) {
   if (c->graph_unavailable || (c->graph_exec != nullptr && c->graph_batch == c->batch)) return;
   drop_graph(c);
-  draft(c, nullptr, nullptr);                      // makes the draft path's TMA descriptors exist
+  draft(c, nullptr, nullptr, nullptr);             // makes the draft path's TMA descriptors exist
   cudaStreamSynchronize(c->stream);
   if (cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
     cudaGetLastError();
@@ -823,6 +821,8 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
   c->batch = 0;
   c->phase = 0;
   c->launches = 0;
+  c->only_class = -1;
+  c->cur_class = PROF_OTHER;
   {
     const char* v = getenv("FM_NO_PDL");
     c->use_pdl = !(v != nullptr && v[0] == '1');
@@ -855,6 +855,51 @@ int fm_profile_end(fm_ctx* c, fm_profile* out) {
   c->prof_on = false;
   out->gemm_ms = c->prof_ms[PROF_GEMM]; out->gemm_bytes = c->prof_bytes[PROF_GEMM]; out->gemm_launches = c->prof_n[PROF_GEMM];
   out->attn_ms = c->prof_ms[PROF_ATTN]; out->attn_launches = c->prof_n[PROF_ATTN];
+  return FM_OK;
+}
+
+int fm_profile_class(fm_ctx* c, int32_t cls, int32_t reps, fm_profile* out) {
+  if (c == nullptr || out == nullptr || reps < 1 || (cls != PROF_GEMM && cls != PROF_ATTN)) return FM_ERR_INVALID_ARG;
+  if (c->phase < 1) return FM_ERR_BAD_STATE;
+  memset(out, 0, sizeof(*out));
+  CUDA_OK(cudaStreamSynchronize(c->stream));
+  if (cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { cudaGetLastError(); return FM_ERR_CUDA; }
+  const int64_t l0 = c->launches;
+  c->only_class = cls;
+  c->class_bytes = 0.0;
+  c->capturing = true;
+  forward(c, nullptr);
+  c->capturing = false;
+  c->only_class = -1;
+  const int64_t n_launch = c->launches - l0;
+  c->launches = l0;
+  cudaGraph_t g = nullptr;
+  cudaGraphExec_t ge = nullptr;
+  if (cudaStreamEndCapture(c->stream, &g) != cudaSuccess || g == nullptr || c->launch_error != FM_OK) {
+    cudaGetLastError();
+    if (g != nullptr) cudaGraphDestroy(g);
+    c->launch_error = FM_OK;
+    return FM_ERR_CUDA;
+  }
+  if (cudaGraphInstantiate(&ge, g, 0) != cudaSuccess) { cudaGetLastError(); cudaGraphDestroy(g); return FM_ERR_CUDA; }
+  cudaEvent_t e0, e1;
+  cudaEventCreate(&e0);
+  cudaEventCreate(&e1);
+  for (int i = 0; i < 3; ++i) cudaGraphLaunch(ge, c->stream);
+  cudaEventRecord(e0, c->stream);
+  for (int i = 0; i < reps; ++i) cudaGraphLaunch(ge, c->stream);
+  cudaEventRecord(e1, c->stream);
+  const bool ok = cudaEventSynchronize(e1) == cudaSuccess;
+  float ms = 0.f;
+  cudaEventElapsedTime(&ms, e0, e1);
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  cudaGraphExecDestroy(ge);
+  cudaGraphDestroy(g);
+  if (!ok) return FM_ERR_CUDA;
+  if (cls == PROF_GEMM) { out->gemm_ms = ms / reps; out->gemm_launches = n_launch; out->gemm_bytes = c->class_bytes; }
+  else { out->attn_ms = ms / reps; out->attn_launches = n_launch; }
+  c->phase = 1;
   return FM_OK;
 }
 
@@ -904,6 +949,7 @@ int fm_prefill(fm_ctx* c, int32_t batch, const float* cond, const int32_t* promp
   const int passes = (1 + longest + dm.R1 - 1) / dm.R1;
   for (int i = 0; i < passes; ++i) {
     LAUNCH(c, prefill_feed_kernel, batch, 32, 0, dm, c->st, batch, prompt, c->prompt_off_dev);
+    LAUNCH(c, row_count_kernel, 1, 32, 0, dm, c->st, batch);
     forward(c, nullptr);
     LAUNCH(c, prefill_advance_kernel, (batch + 127) / 128, 128, 0, dm, c->st, batch);
   }
@@ -932,7 +978,7 @@ int fm_set_max_faces(fm_ctx* c, const int32_t* max_faces) {
 int fm_draft(fm_ctx* c, int32_t* cand, float* draft_logits, float* draft_margin) {
   if (c == nullptr) return FM_ERR_INVALID_ARG;
   if (c->phase < 1) return FM_ERR_BAD_STATE;
-  draft(c, draft_logits, draft_margin);
+  draft(c, draft_logits, draft_margin, nullptr);
   const int n = c->batch * c->dm.R1;
   if (cand != nullptr) LAUNCH(c, copy_i32_kernel, (n + 127) / 128, 128, 0, c->st.cand, cand, n);
   CUDA_OK(cudaGetLastError());
@@ -997,9 +1043,8 @@ int fm_accept(fm_ctx* c, const int32_t* force_len, const int32_t* force_tok, int
               int32_t* kv_len) {
   if (c == nullptr) return FM_ERR_INVALID_ARG;
   if (c->phase != 2) return FM_ERR_BAD_STATE;
-  LAUNCH(c, accept_kernel, (c->batch * 32 + 127) / 128, 128, 0, c->dm, c->st, c->batch, force_len, force_tok, n_acc,
-         emitted, kv_len, (const GenOut*)nullptr);
-  LAUNCH(c, row_count_kernel, 1, 32, 0, c->dm, c->st, c->batch);
+  LAUNCH(c, accept_kernel, 1, accept_threads(c->batch), 0, c->dm, c->st, c->batch, force_len, force_tok, n_acc, emitted, kv_len,
+         (const GenOut*)nullptr, 0);
   CUDA_OK(cudaGetLastError());
   if (c->launch_error != FM_OK) return c->launch_error;
   c->phase = 1;

@@ -237,12 +237,9 @@ struct GenOut {            // where fm_generate collects tokens (device-resident
   volatile int* host_done; // mapped pinned flag: number of unfinished sequences
 };
 
-__global__ void accept_kernel(Dims dm, SeqState st, int batch, const int* __restrict__ force_len,
-                              const int* __restrict__ force_tok, int* __restrict__ n_acc, int* __restrict__ emitted,
-                              int* __restrict__ kv_len, const GenOut* __restrict__ gen) {
-  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  const int b = warp;
-  if (b >= batch) return;
+__device__ inline void accept_one(const Dims& dm, const SeqState& st, int b, int lane, const int* __restrict__ force_len,
+                                  const int* __restrict__ force_tok, int* __restrict__ n_acc, int* __restrict__ emitted,
+                                  int* __restrict__ kv_len, const GenOut* __restrict__ gen) {
   const int R1 = dm.R1, eos = dm.n_bins + 1;
   const int rows = st.nrow[b];
   int a = 0;
@@ -290,15 +287,38 @@ __global__ void accept_kernel(Dims dm, SeqState st, int batch, const int* __rest
   }
 }
 
-// after accept + row count of a generate pass: bump the step counter, tell the host how many
-// sequences are still running
-__global__ void step_end_kernel(SeqState st, const GenOut* __restrict__ gen) {
-  if (threadIdx.x != 0 || blockIdx.x != 0) return;
-  *st.step += 1;
-  if (gen->stats != nullptr) gen->stats[0] += 1;
-  if (gen->host_done != nullptr) { *gen->host_done = st.n_active[3]; __threadfence_system(); }
+// rows fed at each level in the next pass (n_active[level]); n_active[3] = unfinished sequences
+__device__ inline void count_rows(const Dims& dm, const SeqState& st, int batch) {
+  int cnt[3] = {0, 0, 0}, act = 0;
+  for (int b = 0; b < batch; ++b) {
+    const int n = st.nrow[b], L = st.L[b];
+    if (n <= 0) continue;
+    act++;
+    for (int l = 0; l < 3; ++l) {
+      const int r = fm_ratio(l);
+      cnt[l] += (L + n - 1) / r - (L + r - 1) / r + 1;
+    }
+  }
+  st.n_active[0] = cnt[0]; st.n_active[1] = cnt[1]; st.n_active[2] = cnt[2]; st.n_active[3] = act;
 }
 
+// One block; its warps walk over the sequences.  Afterwards thread 0 counts the rows of the next
+// pass and, inside fm_generate (step_end != 0), bumps the pass counter and tells the host how many
+// sequences are still running.
+__global__ void accept_kernel(Dims dm, SeqState st, int batch, const int* __restrict__ force_len,
+                              const int* __restrict__ force_tok, int* __restrict__ n_acc, int* __restrict__ emitted,
+                              int* __restrict__ kv_len, const GenOut* __restrict__ gen, int step_end) {
+  const int lane = threadIdx.x & 31;
+  for (int b = threadIdx.x >> 5; b < batch; b += blockDim.x >> 5) accept_one(dm, st, b, lane, force_len, force_tok, n_acc, emitted, kv_len, gen);
+  __syncthreads();
+  if (threadIdx.x != 0) return;
+  count_rows(dm, st, batch);
+  if (step_end) {
+    *st.step += 1;
+    if (gen->stats != nullptr) gen->stats[0] += 1;
+    if (gen->host_done != nullptr) { *gen->host_done = st.n_active[3]; __threadfence_system(); }
+  }
+}
 // ------------------------------------------------------------------------------------------
 // prefill helpers
 // ------------------------------------------------------------------------------------------
@@ -401,8 +421,12 @@ __device__ inline int draft_feature_row(int n, int j, int b, int B) {
 }
 
 // masked argmax of the chosen feature's logits -> cand[b][j]; cand[b][0] = pending main token
+// With a teacher (fm_generate's benchmark stand-in for trained heads, sitting where the Correct stage
+// edits drafts) the drafts 1..keep are then replaced by the known continuation and draft keep+1 by a
+// different coordinate id.
 __global__ void draft_pick_kernel(Dims dm, SeqState st, int batch, const float* __restrict__ logits /*[NF*B, Vpad]*/,
-                                  float* __restrict__ logits_out, float* __restrict__ margin_out) {
+                                  float* __restrict__ logits_out, float* __restrict__ margin_out,
+                                  const GenOut* __restrict__ gen) {
   ptx::grid_dep_launch();
   ptx::grid_dep_wait();
   const int b = blockIdx.x, j = blockIdx.y;        // j = 0..D
@@ -424,26 +448,20 @@ __global__ void draft_pick_kernel(Dims dm, SeqState st, int batch, const float* 
     for (int i = threadIdx.x; i < dm.V; i += blockDim.x) logits_out[((size_t)b * dm.D + j - 1) * dm.V + i] = z[i];
   const Top2 t = block_top2(z, dm, n + j);
   if (threadIdx.x == 0) {
-    st.cand[b * dm.R1 + j] = t.i1;
+    int tok = t.i1;
+    if (gen != nullptr && gen->truth != nullptr) {
+      const int keep = gen->keep != nullptr ? gen->keep[(size_t)(*st.step % gen->n_sched) * batch + b] : dm.D;
+      const int idx = n + j;
+      if (idx < gen->truth_stride) {
+        const int tt = gen->truth[(size_t)b * gen->truth_stride + idx];
+        if (tt >= 0 && tt < dm.V) {
+          if (j <= keep) tok = tt;
+          else if (j == keep + 1) tok = (tt + 1) % dm.n_bins;
+        }
+      }
+    }
+    st.cand[b * dm.R1 + j] = tok;
     if (margin_out) margin_out[b * dm.D + j - 1] = t.v1 - t.v2;
-  }
-}
-
-// teacher edit (benchmark stand-in for trained heads; sits where the Correct stage edits drafts):
-// drafts 1..keep <- known continuation, draft keep+1 <- a different coordinate id
-__global__ void teacher_edit_kernel(Dims dm, SeqState st, int batch, const GenOut* __restrict__ gen) {
-  const int b = blockIdx.x;
-  if (b >= batch || gen->truth == nullptr) return;
-  if (st.done[b] || st.nrow[b] <= 0) return;
-  const int n = st.L[b] - 1;
-  const int keep = gen->keep != nullptr ? gen->keep[(size_t)(*st.step % gen->n_sched) * batch + b] : dm.D;
-  for (int j = 1 + threadIdx.x; j <= dm.D; j += blockDim.x) {
-    const int idx = n + j;
-    if (idx >= gen->truth_stride) continue;
-    const int t = gen->truth[(size_t)b * gen->truth_stride + idx];
-    if (t < 0 || t >= dm.V) continue;
-    if (j <= keep) st.cand[b * dm.R1 + j] = t;
-    else if (j == keep + 1) st.cand[b * dm.R1 + j] = (t + 1) % dm.n_bins;
   }
 }
 
