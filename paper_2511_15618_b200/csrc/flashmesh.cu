@@ -526,9 +526,10 @@ void run_stack(fm_ctx* c, int s, float* x, float* stash_ring, const float* next_
   const int nl = (int)c->layers[s].size();
   for (int l = 0; l < nl; ++l) {
     const LayerDev& L = c->layers[s][l];
-    if (stash_ring != nullptr && l == nl - 1)
-      launch_pdl(c, dim3(1, 1, 1), ring_store_kernel, rows, 128, 0, dm, c->st, c->batch, level, (const float*)x, stash_ring, d);
     tc::Epi eq{};
+    if (stash_ring != nullptr && l == nl - 1) {          // split-node hiddens: the input of the stack's last layer
+      eq.stash_x = x; eq.stash_ring = stash_ring; eq.stash_d = d; eq.stash_rs = fm_ring(level);
+    }
     eq.ssq_in = c->ssq; eq.ssq_n = c->ssq_n; eq.ld_ssq = c->ssq_ld; eq.inv_d_in = 1.f / d; eq.eps = dm.eps;
     eq.dm = dm; eq.st = c->st; eq.batch = c->batch; eq.level = level; eq.rope_tab = c->rope_tab;
     eq.q_out = c->qbuf; eq.Kc = L.K; eq.Vc = L.V;
@@ -564,28 +565,24 @@ void forward(fm_ctx* c, float* logits_out) {
   LAUNCH(c, embed_kernel, Rc, 128, 0, dm, c->st, B, c->E, c->xc, c->layers[0][0].g1, c->a_norm, c->ssq);
   c->ssq_n = 1;
   run_stack(c, 0, c->xc, nullptr, nullptr, false);
-  launch_pdl(c, dim3(1, 1, 1), ring_store_kernel, Rc, 128, 0, dm, c->st, B, 0, (const float*)c->xc, c->hc_ring, d);
-  launch_pdl(c, dim3(1, 1, 1), shorten_gather_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->hc_ring, c->a_cat);
+  launch_pdl(c, dim3(1, 1, 1), shorten_gather_kernel, Rv + Rc, 128, 0, dm, c->st, B, 1, (const float*)c->xc, c->hc_ring, c->a_cat, Rv);
   tc::Epi es{};
   es.x = c->xv; es.ldx = d; es.add = 0; es.gain = c->layers[1][0].g1; es.a_out = c->a_norm; es.lda = 2 * d; es.lo_off = d;
   es.ssq_out = c->ssq; es.ld_ssq_out = c->ssq_ld;
   gemm(c, c->S_cv, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rv, na + 1, tc::EPI_RESID, es, 2);
   run_stack(c, 1, c->xv, nullptr, nullptr, false);
-  launch_pdl(c, dim3(1, 1, 1), ring_store_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->xv, c->hv_ring, d);
-  launch_pdl(c, dim3(1, 1, 1), shorten_gather_kernel, Rf, 128, 0, dm, c->st, B, 2, (const float*)c->hv_ring, c->a_cat);
+  launch_pdl(c, dim3(1, 1, 1), shorten_gather_kernel, Rf + Rv, 128, 0, dm, c->st, B, 2, (const float*)c->xv, c->hv_ring, c->a_cat, Rf);
   es.x = c->xf; es.gain = c->layers[2][0].g1;
   gemm(c, c->S_vf, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rf, na + 2, tc::EPI_RESID, es, 2);
   run_stack(c, 2, c->xf, c->zf, nullptr, true);                    // leaves bf16(xf) in a_norm
   gemm(c, c->U_fv, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rf, na + 2, tc::EPI_F32, epi_plain(c->tmp3d, 3 * d), 2);
-  launch_pdl(c, dim3(1, 1, 1), ring_store_kernel, Rf, 128, 0, dm, c->st, B, 2, (const float*)c->tmp3d, c->trif_ring, 3 * d);
-  launch_pdl(c, dim3(1, 1, 1), upsample_add_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->hv_ring, (const float*)c->trif_ring, c->xv,
-             (const float*)c->layers[3][0].g1, c->a_norm, c->ssq);
+  launch_pdl(c, dim3(1, 1, 1), upsample_add_kernel, Rv + Rf, 128, 0, dm, c->st, B, 1, (const float*)c->hv_ring, (const float*)c->tmp3d,
+             c->trif_ring, c->xv, (const float*)c->layers[3][0].g1, c->a_norm, c->ssq, Rv);
   c->ssq_n = 1;
   run_stack(c, 3, c->xv, c->zv, nullptr, true);                    // leaves bf16(xv) in a_norm
   gemm(c, c->U_vc, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rv, na + 1, tc::EPI_F32, epi_plain(c->tmp3d, 3 * d), 2);
-  launch_pdl(c, dim3(1, 1, 1), ring_store_kernel, Rv, 128, 0, dm, c->st, B, 1, (const float*)c->tmp3d, c->triv_ring, 3 * d);
-  launch_pdl(c, dim3(1, 1, 1), upsample_add_kernel, Rc, 128, 0, dm, c->st, B, 0, (const float*)c->hc_ring, (const float*)c->triv_ring, c->xc,
-             (const float*)c->layers[4][0].g1, c->a_norm, c->ssq);
+  launch_pdl(c, dim3(1, 1, 1), upsample_add_kernel, Rc + Rv, 128, 0, dm, c->st, B, 0, (const float*)c->hc_ring, (const float*)c->tmp3d,
+             c->triv_ring, c->xc, (const float*)c->layers[4][0].g1, c->a_norm, c->ssq, Rc);
   c->ssq_n = 1;
   run_stack(c, 4, c->xc, c->zc, c->g_out, true);                   // leaves bf16(xc * g_out) and its sums of squares
   tc::Epi el = epi_plain(c->logits, dm.Vpad);

@@ -75,6 +75,9 @@ struct Epi {
   bf16* q_out;                   //            [rows, H*dh], rotated and scaled by qscale
   bf16* Kc; bf16* Vc;            //            caches [B, Hkv, slots, dh]
   float qscale;
+  const float* stash_x;          //            when stash_ring is set: residual rows [rows, stash_d] that the CTAs
+  float* stash_ring;             //            of K split 0 copy, column block by column block, into the carry ring
+  int stash_d, stash_rs;         //            [B, stash_rs, stash_d] at entry pos mod stash_rs (split-node hiddens)
 };
 
 __device__ inline uint64_t smem_desc_sw128(uint32_t addr) {
@@ -402,6 +405,15 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   }
 
   __syncthreads();                                         // s_inv / row maps are written (long before the MMAs end)
+  if (MODE == EPI_QKV && e.stash_ring != nullptr && z == 0) {
+    // the rows' residual values, as they enter this layer, go into the carry ring (the draft heads
+    // read them after the pass); this CTA copies column tile_m*128 + tid
+    const int col = tile_m * BM + tid;
+    if (col < e.stash_d)
+      for (int n = 0; n < ns; ++n)
+        if (s_rb[n] >= 0)
+          e.stash_ring[((size_t)s_rb[n] * e.stash_rs + s_rp[n] % e.stash_rs) * e.stash_d + col] = e.stash_x[(size_t)(row0 + n) * e.stash_d + col];
+  }
   // ---- every warp waits for the accumulator and sends its 32 columns of the partial tile to
   // their owners.  A timeout is recorded; zeros are sent so that no owner waits in vain.
   bool ok = n_slabs > 0 ? ptx::mbar_wait(accum, 0) : true;

@@ -112,53 +112,73 @@ __global__ void prefix_store_kernel(Dims dm, int level, int row0, const float* _
 // ------------------------------------------------------------------------------------------
 // hourglass carry rings
 // ------------------------------------------------------------------------------------------
-// ring[b][p % ring][:] = x[row][:] for rows that are fed (width = floats per entry)
-__global__ void ring_store_kernel(Dims dm, SeqState st, int batch, int level, const float* __restrict__ x,
-                                  float* __restrict__ ring, int width) {
-  ptx::grid_dep_launch();
-  ptx::grid_dep_wait();
-  const int row = blockIdx.x;
-  int b, p;
-  if (!fm_row_map(dm, st, batch, level, row, b, p)) return;
-  const int rs = fm_ring(level);
-  float* dst = ring + ((size_t)b * rs + (p % rs)) * width;
-  const float* src = x + (size_t)row * width;
-  for (int i = threadIdx.x; i < width; i += blockDim.x) dst[i] = src[i];
+// first level-local position of sequence b in this pass
+__device__ inline int fm_first_pos(const SeqState& st, int b, int level) {
+  const int r = fm_ratio(level);
+  return (st.L[b] + r - 1) / r;
 }
 
-// a3/a5 shorten, gather half: row v of level `level_out` <- [h_{3v-2}; h_{3v-1}; h_{3v}] from the ring
-// of the level below (zeros for negative positions and for rows that are not fed), as [hi | lo]
-// terms: row length 6d
-__global__ void shorten_gather_kernel(Dims dm, SeqState st, int batch, int level_out, const float* __restrict__ ring,
-                                      bf16* __restrict__ out) {
+// a3/a5 shorten, gather half, fused with the ring store of the level below.  Blocks [0, rows_out):
+// row v of level `level_out` <- [h_{3v-2}; h_{3v-1}; h_{3v}] (zeros for negative positions and for
+// rows that are not fed) as [hi | lo] terms, row length 6d; a hidden of this pass is read from
+// x_below, an older one from the carry ring.  Blocks [rows_out, rows_out + rows_below): this pass's
+// hiddens of the level below go into its ring for later passes.
+__global__ void shorten_gather_kernel(Dims dm, SeqState st, int batch, int level_out, const float* __restrict__ x_below,
+                                      float* __restrict__ ring, bf16* __restrict__ out, int rows_out) {
   ptx::grid_dep_launch();
   ptx::grid_dep_wait();
+  const int lb = level_out - 1, rs = fm_ring(lb), d = dm.d;
+  if ((int)blockIdx.x >= rows_out) {
+    const int row = blockIdx.x - rows_out;
+    int b, p;
+    if (!fm_row_map(dm, st, batch, lb, row, b, p)) return;
+    float* dst = ring + ((size_t)b * rs + (p % rs)) * d;
+    const float* src = x_below + (size_t)row * d;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = src[i];
+    return;
+  }
   const int row = blockIdx.x;
   int b, v;
   const bool valid = fm_row_map(dm, st, batch, level_out, row, b, v);
-  const int rs = fm_ring(level_out - 1), d = dm.d;
+  const int p0 = valid ? fm_first_pos(st, b, lb) : 0, m_below = fm_rows_per_seq(dm, lb);
   for (int part = 0; part < 3; ++part) {
     const int pos = 3 * v - 2 + part;
     const bool ok = valid && pos >= 0;
-    const float* src = ring + ((size_t)b * rs + ((pos + rs) % rs)) * d;
+    const float* src = (ok && pos >= p0) ? x_below + ((size_t)b * m_below + (pos - p0)) * d
+                                         : ring + ((size_t)b * rs + ((pos + rs) % rs)) * d;
     for (int i = threadIdx.x; i < d; i += blockDim.x)
       store_hi_lo(out + (size_t)row * 6 * d + part * d + i, ok ? src[i] : 0.f, 3 * d);
   }
 }
 
-// a7/a9 upsample, residual half: x[row] = h_ring[b][p] + tri_ring[b][p/3][(p%3)*d ...]; the row is
-// then handed to the first layer of the stack above (operand row and sum of squares)
+// a7/a9 upsample, residual half, fused with the ring store of the upsampled triples.  Blocks
+// [0, rows): x[row] = h[b][p] + tri[b][p/3][(p%3)*d ...], where h is the pre-shorten hidden of the
+// position (kept in the carry ring by the shorten step of this pass) and the triple comes from
+// `tri_new` if its parent row belongs to this pass, else from the ring; the row is then handed to
+// the first layer of the stack above (operand row and sum of squares).  Blocks [rows, rows +
+// rows_up): this pass's triples go into the ring.
 __global__ void upsample_add_kernel(Dims dm, SeqState st, int batch, int level, const float* __restrict__ h_ring,
-                                    const float* __restrict__ tri_ring, float* __restrict__ x, const float* __restrict__ g,
-                                    bf16* __restrict__ a_out, float* __restrict__ ssq) {
+                                    const float* __restrict__ tri_new, float* __restrict__ tri_ring, float* __restrict__ x,
+                                    const float* __restrict__ g, bf16* __restrict__ a_out, float* __restrict__ ssq, int rows) {
   ptx::grid_dep_launch();
   ptx::grid_dep_wait();
+  const int rs = fm_ring(level), rsu = fm_ring(level + 1), d = dm.d;
+  if ((int)blockIdx.x >= rows) {
+    const int row = blockIdx.x - rows;
+    int b, p;
+    if (!fm_row_map(dm, st, batch, level + 1, row, b, p)) return;
+    float* dst = tri_ring + ((size_t)b * rsu + (p % rsu)) * 3 * d;
+    const float* src = tri_new + (size_t)row * 3 * d;
+    for (int i = threadIdx.x; i < 3 * d; i += blockDim.x) dst[i] = src[i];
+    return;
+  }
   const int row = blockIdx.x;
   int b, p;
   const bool valid = fm_row_map(dm, st, batch, level, row, b, p);
-  const int rs = fm_ring(level), rsu = fm_ring(level + 1), d = dm.d;
   const float* h = h_ring + ((size_t)b * rs + (p % rs)) * d;
-  const float* t = tri_ring + ((size_t)b * rsu + ((p / 3) % rsu)) * 3 * d + (p % 3) * d;
+  const int up = p / 3, p0u = valid ? fm_first_pos(st, b, level + 1) : 0;
+  const float* t = (valid && up >= p0u) ? tri_new + ((size_t)b * fm_rows_per_seq(dm, level + 1) + (up - p0u)) * 3 * d + (p % 3) * d
+                                        : tri_ring + ((size_t)b * rsu + (up % rsu)) * 3 * d + (p % 3) * d;
   for (int i = threadIdx.x; i < d; i += blockDim.x) x[(size_t)row * d + i] = valid ? h[i] + t[i] : 0.f;
   __syncthreads();
   stack_entry_row(x + (size_t)row * d, row, d, g, a_out, ssq);
