@@ -453,7 +453,8 @@ tc::Epi epi_plain(void* out, int ldo) {
 // 128), A: [a_rows_alloc, a_parts * K] bf16 (rows padded to 16; a_parts = 2: [hi | lo] terms).  The
 // K split (= cluster size) depends on the shapes only.
 void gemm(fm_ctx* c, const bf16* W, size_t w_rows_alloc, int w_row0, const bf16* A, size_t a_rows_alloc, int a_row0,
-          int M, int K, int R, const int* n_active, int mode, tc::Epi e, int a_parts = 1) {
+          int M, int K, int R, const int* n_active, int mode, tc::Epi e, int a_parts = 1, int stacked = 1, int z_rows = 0,
+          int z_w_rows = 0) {
   if (R <= 0) return;
   (void)w_rows_alloc;
   if (w_row0 % tc::BM != 0) { c->launch_error = FM_ERR_UNSUPPORTED; return; }
@@ -463,7 +464,7 @@ void gemm(fm_ctx* c, const bf16* W, size_t w_rows_alloc, int w_row0, const bf16*
   // N tiles), which keeps the K split, and with it the cluster reduction, small.
   const int Rpad = round_up(R, 16);
   const int N = Rpad <= 32 ? Rpad : 32;
-  const int n_tiles = (Rpad + N - 1) / N;
+  const int n_tiles = stacked > 1 ? stacked : (Rpad + N - 1) / N;   // stacked problems share a launch through grid.z
   int split = 1;
   while (split * 2 <= tc::MAX_SPLIT && split * 2 <= slabs && tiles * n_tiles * split * 2 <= c->split_target) split *= 2;
   const int tA = tmap_for(c, A, a_rows_alloc, (uint64_t)K, N, (uint32_t)a_parts);
@@ -471,12 +472,13 @@ void gemm(fm_ctx* c, const bf16* W, size_t w_rows_alloc, int w_row0, const bf16*
   int stages = tc::pick_stages(N, (slabs + split - 1) / split, a_parts);
   if (c->stage_cap > 0 && stages > c->stage_cap) stages = c->stage_cap;
   const long pi = prof_open(c, PROF_GEMM, 2.0 * M * K);            // algorithmic bytes: the weight matrix once
-  tc::Args g{W, c->tmaps + tA, M, K, N, R, split, stages, a_parts, w_row0 / tc::BM, a_row0, n_active, c->st.status};
+  tc::Args g{W, c->tmaps + tA, M, K, N, R, split, stages, a_parts, w_row0 / tc::BM, a_row0, stacked > 1 ? z_rows : 0,
+             stacked > 1 ? z_w_rows / tc::BM : 0, n_active, c->st.status};
   e.row0 = 0;
   const int smem = tc::smem_bytes(N, stages, a_parts);
   const dim3 grid(tiles, split, n_tiles), cl(1, split, 1);
   c->cur_class = PROF_GEMM;
-  if (c->only_class == PROF_GEMM) c->class_bytes += 2.0 * M * K;
+  if (c->only_class == PROF_GEMM) c->class_bytes += 2.0 * M * K * (stacked > 1 ? stacked : 1);
   switch (mode) {
     case tc::EPI_F32: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_F32>, grid, 128, smem, g, e); break;
     case tc::EPI_BF16: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_BF16>, grid, 128, smem, g, e); break;
@@ -601,9 +603,14 @@ void draft(fm_ctx* c, float* logits_out, float* margin_out, const GenOut* gen) {
     const int* na = c->st.n_active + 3;
     const size_t MB = dm.max_batch;
     LAUNCH(c, draft_prep_kernel, dim3(B, dm.NH), 256, 0, dm, c->st, B, c->zc, c->zv, c->zf, c->head_g, c->dh_a);
-    for (int h = 0; h < dm.NH; ++h)
-      gemm(c, c->headA, (size_t)dm.NH * dpad, h * dpad, c->dh_a, (size_t)dm.NH * MB + 16, h * (int)MB, d, d, B, na, tc::EPI_F32,
-           epi_plain(c->dh_y + (size_t)h * MB * d, d));
+    if (B <= 32) {                                               // the NH head matrices as one launch
+      gemm(c, c->headA, (size_t)dm.NH * dpad, 0, c->dh_a, (size_t)dm.NH * MB + 16, 0, d, d, B, na, tc::EPI_F32, epi_plain(c->dh_y, d), 1,
+           dm.NH, (int)MB, dpad);
+    } else {
+      for (int h = 0; h < dm.NH; ++h)
+        gemm(c, c->headA, (size_t)dm.NH * dpad, h * dpad, c->dh_a, (size_t)dm.NH * MB + 16, h * (int)MB, d, d, B, na, tc::EPI_F32,
+             epi_plain(c->dh_y + (size_t)h * MB * d, d));
+    }
     launch_pdl(c, dim3(1, 1, 1), draft_residual_kernel, dim3(B, dm.NH), 128, 0, dm, c->st, B, (const float*)c->zc, (const float*)c->zv,
                (const float*)c->zf, (const float*)c->dh_y, c->feat, c->up_in_v, c->up_in_f);
     gemm(c, c->U_fv, pad128(3 * d), 0, c->up_in_f, align_up((size_t)dm.Ef * MB, 16), 0, 3 * d, d, dm.Ef * B, na, tc::EPI_BF16,

@@ -53,6 +53,8 @@ struct Args {
   int stages;                    // depth of the shared-memory ring (2..MAX_STAGES)
   int a_parts;                   // 1: plain bf16 operand rows, 2: hi + lo terms
   int w_tile0, a_row0;           // first M tile inside W (stacked matrices), first operand row
+  int z_rows, z_w_tiles;         // z_rows > 0: blockIdx.z indexes stacked problems instead of N tiles: problem z
+                                 // uses weight tiles from w_tile0 + z*z_w_tiles and rows from z*z_rows (n_store rows each)
   const int* n_active;           // skip when *n_active == 0 (may be null); must not change during a pass
   int* status;
 };
@@ -216,8 +218,9 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tile_m = blockIdx.x;
   // token rows of this CTA: N tile blockIdx.z of the launch's rows
-  const int row_lo = (int)blockIdx.z * g.N;
-  const int ns = min(g.N, g.n_store - row_lo);               // rows of this tile that exist
+  const int row_lo = (int)blockIdx.z * (g.z_rows > 0 ? g.z_rows : g.N);
+  const int ns = g.z_rows > 0 ? min(g.N, g.n_store) : min(g.N, g.n_store - row_lo);   // rows of this tile that exist
+  const int w_tile = g.w_tile0 + (int)blockIdx.z * g.z_w_tiles;
   const int row0 = e.row0 + row_lo;                        // first output row
   const int a_row = g.a_row0 + row_lo;                     // first operand row
   const int S = g.split;
@@ -239,7 +242,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
     ptx::prefetch_tmap(g.tmA);
     // The weight slabs of the first stages do not depend on the previous kernel: request them at
     // once, so that they travel while the rest of the prologue runs.
-    const bf16* wsrc = g.W + ((size_t)(g.w_tile0 + tile_m) * slabs + s0) * (BM * BK);
+    const bf16* wsrc = g.W + ((size_t)(w_tile + tile_m) * slabs + s0) * (BM * BK);
     const int pre = n_slabs < STAGES ? n_slabs : STAGES;
     for (int i = 0; i < pre; ++i) {
       ptx::mbar_expect_tx(full + i, BM * 128 + g.a_parts * g.N * 128);
@@ -271,7 +274,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   }
   if (warp == 0 && lane == 0) {
     // ---- producer: stream the rest of this CTA's K range through the stage ring
-    const bf16* wsrc = g.W + ((size_t)(g.w_tile0 + tile_m) * slabs + s0) * (BM * BK);
+    const bf16* wsrc = g.W + ((size_t)(w_tile + tile_m) * slabs + s0) * (BM * BK);
     const int pre = n_slabs < STAGES ? n_slabs : STAGES;
     for (int i = pre; i < n_slabs; ++i) {
       const int st = i % STAGES;
