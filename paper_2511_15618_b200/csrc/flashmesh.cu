@@ -496,6 +496,8 @@ __global__ void row_count_kernel(Dims dm, SeqState st, int batch) {
   if (threadIdx.x == 0 && blockIdx.x == 0) count_rows(dm, st, batch);
 }
 
+// threads of a kernel that walks over one row of d values: one element per thread up to 512
+inline int row_threads(int d) { return d >= 512 ? 512 : (d >= 256 ? 256 : 128); }
 inline int accept_threads(int batch) { return batch >= 32 ? 1024 : 32 * (batch < 1 ? 1 : batch); }
 
 void attention(fm_ctx* c, int level, const LayerDev& L) {
@@ -564,26 +566,26 @@ void forward(fm_ctx* c, float* logits_out) {
   // The launch that opens a pass is a full barrier: the per-pass state (rows, lengths, row counts
   // -- every call that changes them ends with a row count -- and candidates) is final before any
   // later kernel's prologue can run.
-  LAUNCH(c, embed_kernel, Rc, 128, 0, dm, c->st, B, c->E, c->xc, c->layers[0][0].g1, c->a_norm, c->ssq);
+  LAUNCH(c, embed_kernel, Rc, row_threads(d), 0, dm, c->st, B, c->E, c->xc, c->layers[0][0].g1, c->a_norm, c->ssq);
   c->ssq_n = 1;
   run_stack(c, 0, c->xc, nullptr, nullptr, false);
-  launch_pdl(c, dim3(1, 1, 1), shorten_gather_kernel, Rv + Rc, 128, 0, dm, c->st, B, 1, (const float*)c->xc, c->hc_ring, c->a_cat, Rv);
+  launch_pdl(c, dim3(1, 1, 1), shorten_gather_kernel, dim3(Rv + Rc, 3), row_threads(d), 0, dm, c->st, B, 1, (const float*)c->xc, c->hc_ring, c->a_cat, Rv);
   tc::Epi es{};
   es.x = c->xv; es.ldx = d; es.add = 0; es.gain = c->layers[1][0].g1; es.a_out = c->a_norm; es.lda = 2 * d; es.lo_off = d;
   es.ssq_out = c->ssq; es.ld_ssq_out = c->ssq_ld;
   gemm(c, c->S_cv, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rv, na + 1, tc::EPI_RESID, es, 2);
   run_stack(c, 1, c->xv, nullptr, nullptr, false);
-  launch_pdl(c, dim3(1, 1, 1), shorten_gather_kernel, Rf + Rv, 128, 0, dm, c->st, B, 2, (const float*)c->xv, c->hv_ring, c->a_cat, Rf);
+  launch_pdl(c, dim3(1, 1, 1), shorten_gather_kernel, dim3(Rf + Rv, 3), row_threads(d), 0, dm, c->st, B, 2, (const float*)c->xv, c->hv_ring, c->a_cat, Rf);
   es.x = c->xf; es.gain = c->layers[2][0].g1;
   gemm(c, c->S_vf, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rf, na + 2, tc::EPI_RESID, es, 2);
   run_stack(c, 2, c->xf, c->zf, nullptr, true);                    // leaves bf16(xf) in a_norm
   gemm(c, c->U_fv, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rf, na + 2, tc::EPI_F32, epi_plain(c->tmp3d, 3 * d), 2);
-  launch_pdl(c, dim3(1, 1, 1), upsample_add_kernel, Rv + Rf, 128, 0, dm, c->st, B, 1, (const float*)c->hv_ring, (const float*)c->tmp3d,
+  launch_pdl(c, dim3(1, 1, 1), upsample_add_kernel, Rv + Rf, row_threads(d), 0, dm, c->st, B, 1, (const float*)c->hv_ring, (const float*)c->tmp3d,
              c->trif_ring, c->xv, (const float*)c->layers[3][0].g1, c->a_norm, c->ssq, Rv);
   c->ssq_n = 1;
   run_stack(c, 3, c->xv, c->zv, nullptr, true);                    // leaves bf16(xv) in a_norm
   gemm(c, c->U_vc, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rv, na + 1, tc::EPI_F32, epi_plain(c->tmp3d, 3 * d), 2);
-  launch_pdl(c, dim3(1, 1, 1), upsample_add_kernel, Rc + Rv, 128, 0, dm, c->st, B, 0, (const float*)c->hc_ring, (const float*)c->tmp3d,
+  launch_pdl(c, dim3(1, 1, 1), upsample_add_kernel, Rc + Rv, row_threads(d), 0, dm, c->st, B, 0, (const float*)c->hc_ring, (const float*)c->tmp3d,
              c->triv_ring, c->xc, (const float*)c->layers[4][0].g1, c->a_norm, c->ssq, Rc);
   c->ssq_n = 1;
   run_stack(c, 4, c->xc, c->zc, c->g_out, true);                   // leaves bf16(xc * g_out) and its sums of squares

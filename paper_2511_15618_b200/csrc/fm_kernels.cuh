@@ -129,6 +129,7 @@ __global__ void shorten_gather_kernel(Dims dm, SeqState st, int batch, int level
   ptx::grid_dep_wait();
   const int lb = level_out - 1, rs = fm_ring(lb), d = dm.d;
   if ((int)blockIdx.x >= rows_out) {
+    if (blockIdx.y != 0) return;
     const int row = blockIdx.x - rows_out;
     int b, p;
     if (!fm_row_map(dm, st, batch, lb, row, b, p)) return;
@@ -141,7 +142,8 @@ __global__ void shorten_gather_kernel(Dims dm, SeqState st, int batch, int level
   int b, v;
   const bool valid = fm_row_map(dm, st, batch, level_out, row, b, v);
   const int p0 = valid ? fm_first_pos(st, b, lb) : 0, m_below = fm_rows_per_seq(dm, lb);
-  for (int part = 0; part < 3; ++part) {
+  {
+    const int part = blockIdx.y;                     // grid.y = 3: one of the three concatenated hiddens
     const int pos = 3 * v - 2 + part;
     const bool ok = valid && pos >= 0;
     const float* src = (ok && pos >= p0) ? x_below + ((size_t)b * m_below + (pos - p0)) * d
