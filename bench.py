@@ -201,8 +201,14 @@ def run_ours(args):
         _, _, kv = dev.accept()
         sb = dev.verify_bytes(kv.cpu().numpy().tolist())
         peak, _ = _peaks()
+        cand, _, _ = dev.draft()
+        dev.verify(cand)
+        g_ms, g_n, g_b = dev.profile_class(0, 20)
+        a_ms, a_n, _ = dev.profile_class(1, 20)
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": emitted / (ms * 1e-3), "unit": "tokens/s", "workload": args.workload,
+                              "gemm": {"launches": g_n, "us_per_launch": 1e3 * g_ms / max(1, g_n), "weight_bytes": g_b},
+                              "attention": {"launches": a_n, "us_per_launch": 1e3 * a_ms / max(1, a_n)},
                               "batch": B, "ms_per_step": ms / max(1, steps), "steps": steps, "gpu_launches": launches,
                               "mean_accept_len": emitted / max(1, steps * B),
                               "verify_step_frac_of_hbm_peak": sb / (ms / max(1, steps) * 1e-3) / 1e9 / peak,

@@ -14,7 +14,9 @@
  *
  * Conventions
  *   - Every call returns FM_OK (0) or a negative FM_ERR_* code; nothing throws.  On an error
- *     return no decoding state has been changed.
+ *     return no decoding state has been changed, except after FM_ERR_CUDA or FM_ERR_TIMEOUT:
+ *     then nothing more is enqueued and the sequences must be started again with fm_prefill
+ *     (or the context destroyed).
  *   - Pointers are marked HOST or DEV.  DEV pointers are caller-owned device memory that must
  *     stay valid until the work enqueued by the call has finished on the context's stream.
  *   - All calls except fm_create / fm_destroy / fm_generate only enqueue work on the

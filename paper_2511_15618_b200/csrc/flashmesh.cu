@@ -75,6 +75,7 @@ struct fm_ctx {
   float* ssq;
   int ssq_n, ssq_ld;    // slots the last producer filled, floats between slots
   bool use_pdl;
+  bool debug_sync;      // FM_DEBUG_SYNC: wait for and check every launch
   // prefill temporaries
   bf16* pre_a;
   float* pre_o;
@@ -228,7 +229,9 @@ void carve(fm_ctx* c, Carver& cv) {
     // about one CTA per SM when the cache is full; at most 16 chunks per group
     int G = (int)(((size_t)max_chunks * dm.Hkv * B * c->attn_mt[l] + 147) / 148);
     G = G < 1 ? 1 : (G > 16 ? 16 : G);
-    const int G_min = (max_chunks + 23) / 24;          // at most 24 groups: their states (and weights) are merged from shared memory
+    // the groups' states (and weights) are merged from shared memory: 24 groups at most, fewer for wide heads
+    const int g_cap = dm.dh == 64 ? AttnCfg<64, 128, 8>::MAX_GROUPS : AttnCfg<128, 64, 4>::MAX_GROUPS;
+    const int G_min = (max_chunks + g_cap - 1) / g_cap;
     G = G < G_min ? G_min : G;
     c->attn_G[l] = G;
     c->attn_max_groups[l] = (max_chunks + G - 1) / G;
@@ -303,11 +306,26 @@ int upload_f32(float* dst, const float* src, size_t n) {
 #define LAUNCH(ctx, kern, grid, block, smem, ...)                        \
   do {                                                                   \
     if ((ctx)->only_class >= 0 && (ctx)->cur_class != (ctx)->only_class) break; \
+    if ((ctx)->launch_error != FM_OK) break;                             \
     kern<<<grid, block, smem, (ctx)->stream>>>(__VA_ARGS__);             \
     (ctx)->launches++;                                                   \
+    if ((ctx)->debug_sync) debug_sync_check(ctx, #kern);                 \
   } while (0)
 
 enum ProfClass { PROF_GEMM = 0, PROF_ATTN = 1, PROF_OTHER = 2 };
+
+// Diagnostic mode (environment FM_DEBUG_SYNC): wait for every launch and name the first one that
+// ends with an error; nothing is launched after it.  Not used while a graph is being captured.
+void debug_sync_check(fm_ctx* c, const char* what) {
+  if (c->capturing || c->launch_error != FM_OK) return;
+  cudaError_t err = cudaStreamSynchronize(c->stream);
+  if (err == cudaSuccess) err = cudaGetLastError();
+  if (err != cudaSuccess) {
+    fprintf(stderr, "flashmesh: launch %ld (%s, class %d) ended with: %s\n", c->launches, what, c->cur_class,
+            cudaGetErrorString(err));
+    c->launch_error = FM_ERR_CUDA;
+  }
+}
 
 void prof_drain(fm_ctx* c) {
   if (c->prof_used == 0) return;
@@ -410,6 +428,7 @@ int tmap_for(fm_ctx* c, const void* base, uint64_t rows, uint64_t cols, uint32_t
 template <typename... KArgs, typename... CArgs>
 void launch_pdl(fm_ctx* c, dim3 cluster, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, CArgs&&... args) {
   if (c->only_class >= 0 && c->cur_class != c->only_class) return;
+  if (c->launch_error != FM_OK) return;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
@@ -439,6 +458,11 @@ void launch_pdl(fm_ctx* c, dim3 cluster, void (*kern)(KArgs...), dim3 grid, dim3
     if (c->launch_error == FM_OK) c->launch_error = FM_ERR_CUDA;
   }
   c->launches++;
+  if (c->debug_sync) {
+    char what[96];
+    snprintf(what, sizeof what, "grid %u %u %u block %u smem %zu cluster %u", grid.x, grid.y, grid.z, block.x, smem, cluster.y);
+    debug_sync_check(c, what);
+  }
 }
 
 tc::Epi epi_plain(void* out, int ldo) {
@@ -832,6 +856,8 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
   {
     const char* v = getenv("FM_NO_PDL");
     c->use_pdl = !(v != nullptr && v[0] == '1');
+    const char* ds = getenv("FM_DEBUG_SYNC");
+    c->debug_sync = ds != nullptr && ds[0] == '1';
     const char* t = getenv("FM_SPLIT_TARGET");
     c->split_target = t != nullptr && atoi(t) > 0 ? atoi(t) : 160;
     const char* sc = getenv("FM_STAGE_CAP");
@@ -934,6 +960,7 @@ int fm_prefill(fm_ctx* c, int32_t batch, const float* cond, const int32_t* promp
   }
   if (prompt_off[batch] > 0 && prompt == nullptr) return FM_ERR_INVALID_ARG;
   c->batch = batch;
+  c->launch_error = FM_OK;                         // a new start clears an earlier enqueue error
   c->plen_host.assign(batch, 0);
   for (int b = 0; b < batch; ++b) c->plen_host[b] = prompt_off[b + 1] - prompt_off[b];
   CUDA_OK(cudaMemcpyAsync(c->prompt_off_dev, prompt_off, (batch + 1) * sizeof(int), cudaMemcpyHostToDevice, c->stream));

@@ -50,6 +50,9 @@ struct AttnCfg {
   static constexpr int MERGE = (NW + 1) * STATE;            // the warps' states and the merged one, aliasing the ring
   static constexpr int WORK = RING > MERGE ? RING : MERGE;
   static constexpr int BYTES = WORK + 128 + 1024;           // + barriers + alignment slack
+  // groups the last CTA can merge: their states plus 16 x (groups + 1) weights are staged in WORK
+  static constexpr int MAX_GROUPS_FIT = (WORK - 64) / (STATE + 64);
+  static constexpr int MAX_GROUPS = MAX_GROUPS_FIT < 24 ? MAX_GROUPS_FIT : 24;
   static constexpr int THREADS = (NW + 1) * 32;
 };
 
@@ -89,7 +92,10 @@ __global__ void __launch_bounds__((NW + 1) * 32) attn_stream_kernel(const AttnAr
   const int n_groups = (n_chunks + a.G - 1) / a.G;
   const int group = dm.H / dm.Hkv;
   const int M = nq * group;
-  if (nq <= 0 || mt * 16 >= M || u >= n_groups) {  // nothing of the cache falls into this group yet
+  if (nq <= 0 || mt * 16 >= M || u >= n_groups || n_groups > CF::MAX_GROUPS) {
+    // nothing of the cache falls into this group yet; or more groups than the merge can stage
+    // (the host sizes G so that this never happens): report, write nothing
+    if (n_groups > CF::MAX_GROUPS && threadIdx.x == 0) atomicExch(a.st.status, -1);
     ptx::grid_dep_wait();                          // keep the launch chain ordered
     return;
   }

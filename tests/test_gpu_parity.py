@@ -61,6 +61,24 @@ def test_toy_lockstep_windows_and_mqa_and_eos():
     assert rep["done"]
 
 
+@pytest.mark.parametrize("prompt_faces", [100, 150])
+def test_toy_head_dim_128_long_cache_many_groups(prompt_faces):
+    """Head dimension 128 with a cache of 15 to 22 chunks: 100 faces give the largest number of
+    groups the last CTA can merge from shared memory (15, one chunk each), 150 faces give groups
+    of two chunks."""
+    from oracle.lockstep import run_lockstep
+    faces = 3
+    cfg = S.toy_config(d_model=128, n_heads=1, n_kv_heads=1, head_dim=128, d_ff=256, weight_std=0.1, draft_len=3,
+                       layers=(1, 1, 1, 1, 1), prompt_faces=(prompt_faces, prompt_faces), prompt_subdiv=2, gen_faces=faces,
+                       max_tokens=1 + 9 * (prompt_faces + faces) + 3 + 2)
+    w, conds, prompts = _setup(cfg, batch=1)
+    assert len(prompts[0]) == 9 * prompt_faces
+    dev = _dev(cfg, w)
+    rep = run_lockstep(cfg, w, conds, prompts, dev, faces, 60, tol=TOY_TOL, margin=TOY_MARGIN)
+    assert rep["done"] and rep["emitted"] == 9 * faces
+    assert dev.device_status() in (0, -1)
+
+
 def test_toy_teacher_drafts_vary_accept_lengths():
     from oracle.lockstep import run_lockstep
     cfg = S.toy_config(d_model=128, head_dim=64, d_ff=256, weight_std=0.1, draft_len=9, layers=(1, 1, 2, 1, 1), max_batch=2, gen_faces=8, max_tokens=1 + 9 * 8 + 9 + 2)
