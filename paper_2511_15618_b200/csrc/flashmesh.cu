@@ -97,6 +97,8 @@ struct fm_ctx {
   double class_bytes;   // weight bytes of the GEMM launches enqueued by fm_profile_class
   int split_target;     // CTAs a GEMM launch aims for (M tiles x K splits)
   int stage_cap;        // tuning knob: upper bound on the GEMM ring depth (0 = none)
+  int n_sm;                                  // SMs of the device
+  int split_target_deep;                     // the same for launches whose CTAs stream long K ranges
   int launch_error;     // first error met while enqueueing (capacity, descriptor creation)
   // one decode pass (draft, teacher edit, verify, accept) captured as a CUDA graph
   cudaGraph_t graph;
@@ -489,26 +491,46 @@ void gemm(fm_ctx* c, const bf16* W, size_t w_rows_alloc, int w_row0, const bf16*
   const int Rpad = round_up(R, 16);
   const int N = Rpad <= 32 ? Rpad : 32;
   const int n_tiles = stacked > 1 ? stacked : (Rpad + N - 1) / N;   // stacked problems share a launch through grid.z
+  // K split: up to about one CTA per SM; while a CTA would still stream more than 8 slabs (or the
+  // launch has several N tiles) up to two CTAs per SM, whose rings are then kept small enough to share it.
+  const bool tiled = n_tiles > 1 && stacked == 1;
   int split = 1;
-  while (split * 2 <= tc::MAX_SPLIT && split * 2 <= slabs && tiles * n_tiles * split * 2 <= c->split_target) split *= 2;
+  while (split * 2 <= tc::MAX_SPLIT && split * 2 <= slabs) {
+    const bool deep = tiled || slabs / split > 8;
+    if (tiles * n_tiles * split * 2 > (deep ? c->split_target_deep : c->split_target)) break;
+    split *= 2;
+  }
   const int tA = tmap_for(c, A, a_rows_alloc, (uint64_t)K, N, (uint32_t)a_parts);
   if (tA < 0) { c->launch_error = FM_ERR_CUDA; return; }
-  int stages = tc::pick_stages(N, (slabs + split - 1) / split, a_parts);
+  // only the residual and the QKV epilogue have side rows, and only when a thread gets more than two items
+  const bool side = (mode == tc::EPI_RESID || mode == tc::EPI_QKV) && tc::side_bytes(N, split) > 0;
+  const int side_b = side ? tc::side_bytes(N, split) : 0;
+  int stages = tc::pick_stages(N, (slabs + split - 1) / split, a_parts, side_b);
   if (c->stage_cap > 0 && stages > c->stage_cap) stages = c->stage_cap;
+  if (tiles * n_tiles * split > c->n_sm) {                 // two CTAs per SM: each at most 112 KB
+    const int fit = (112 * 1024 - tc::smem_bytes(N, 0, a_parts, side_b)) / tc::stage_bytes(N, a_parts);
+    stages = stages > fit ? (fit < 2 ? 2 : fit) : stages;
+  }
   const long pi = prof_open(c, PROF_GEMM, 2.0 * M * K);            // algorithmic bytes: the weight matrix once
   tc::Args g{W, c->tmaps + tA, M, K, N, R, split, stages, a_parts, w_row0 / tc::BM, a_row0, stacked > 1 ? z_rows : 0,
              stacked > 1 ? z_w_rows / tc::BM : 0, n_active, c->st.status};
   e.row0 = 0;
-  const int smem = tc::smem_bytes(N, stages, a_parts);
+  const int smem = tc::smem_bytes(N, stages, a_parts, side_b);
   const dim3 grid(tiles, split, n_tiles), cl(1, split, 1);
   c->cur_class = PROF_GEMM;
   if (c->only_class == PROF_GEMM) c->class_bytes += 2.0 * M * K * (stacked > 1 ? stacked : 1);
   switch (mode) {
-    case tc::EPI_F32: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_F32>, grid, 128, smem, g, e); break;
-    case tc::EPI_BF16: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_BF16>, grid, 128, smem, g, e); break;
-    case tc::EPI_GELU: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_GELU>, grid, 128, smem, g, e); break;
-    case tc::EPI_RESID: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_RESID>, grid, 128, smem, g, e); break;
-    default: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_QKV>, grid, 128, smem, g, e); break;
+    case tc::EPI_F32: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_F32, false>, grid, 128, smem, g, e); break;
+    case tc::EPI_BF16: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_BF16, false>, grid, 128, smem, g, e); break;
+    case tc::EPI_GELU: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_GELU, false>, grid, 128, smem, g, e); break;
+    case tc::EPI_RESID:
+      if (side) launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_RESID, true>, grid, 128, smem, g, e);
+      else launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_RESID, false>, grid, 128, smem, g, e);
+      break;
+    default:
+      if (side) launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_QKV, true>, grid, 128, smem, g, e);
+      else launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_QKV, false>, grid, 128, smem, g, e);
+      break;
   }
   c->cur_class = PROF_OTHER;
   prof_close(c, pi);
@@ -826,11 +848,13 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
       if (L.tmK < 0 || L.tmV < 0) { delete c; return FM_ERR_CUDA; }
     }
   TRYCUDA(cudaMemcpy(c->tmaps, c->tmaps_host.data(), c->tmaps_host.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice));
-  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
-  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
-  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_GELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
-  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
-  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_F32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_BF16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_GELU, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_RESID, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_QKV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_RESID, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_QKV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
   TRYCUDA(cudaFuncSetAttribute(attn_stream_kernel<64, 128, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<64, 128, 8>::BYTES));
   TRYCUDA(cudaFuncSetAttribute(attn_stream_kernel<128, 64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<128, 64, 4>::BYTES));
   std::vector<double> freq(dm.dh / 2);
@@ -860,6 +884,11 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
     c->debug_sync = ds != nullptr && ds[0] == '1';
     const char* t = getenv("FM_SPLIT_TARGET");
     c->split_target = t != nullptr && atoi(t) > 0 ? atoi(t) : 160;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    c->n_sm = sms > 0 ? sms : 148;
+    const char* tt = getenv("FM_SPLIT_TARGET_DEEP");
+    c->split_target_deep = tt != nullptr && atoi(tt) > 0 ? atoi(tt) : 296;
     const char* sc = getenv("FM_STAGE_CAP");
     c->stage_cap = sc != nullptr ? atoi(sc) : 4;        // measured: deeper rings cost more than they prefetch
   }

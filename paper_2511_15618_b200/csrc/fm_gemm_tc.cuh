@@ -157,20 +157,29 @@ __device__ inline uint32_t map_peer(uint32_t local_addr, uint32_t rank) {
 // Shared memory: ring of `stages` x ([128 x 64] weight slab + [N x 64] operand slab), then the
 // receive buffer of the cluster reduction [split][64/split][2][N + 4] fp32 = (N + 4) * 512 bytes
 // (peers write into it while this CTA may still be multiplying, so it never aliases the ring;
-// the 4 floats of padding spread the readers over the banks), then barriers.
+// the 4 floats of padding spread the readers over the banks), then the side rows [N][512 bytes]
+// (what the epilogue reads per row besides the product: the residual rows of the tile's 128
+// columns, or the rows' rotary angles; brought in by bulk copies while the MMAs run), then barriers.
 inline int stage_bytes(int N, int parts) { return BM * 128 + parts * (((N * 128 + 1023) / 1024) * 1024); }
+// The side rows exist only when a thread may get more than two items of the epilogue (N rows x
+// 64/split pair slots over 128 threads); otherwise the shared memory is better left to a
+// neighbouring kernel's CTA.
+__host__ __device__ inline int side_bytes(int N, int split) { return N * (64 / split) > 256 ? N * 512 : 0; }
 // as many stages as the CTA has slabs (its whole K range is then requested at once), at most 8
 // and what fits beside the receive buffer
-inline int pick_stages(int N, int n_slabs, int parts) {
-  int st = (200 * 1024 - (N + 4) * 512) / stage_bytes(N, parts);
+inline int pick_stages(int N, int n_slabs, int parts, int side_b) {
+  int st = (200 * 1024 - (N + 4) * 512 - side_b) / stage_bytes(N, parts);
   st = st > MAX_STAGES ? MAX_STAGES : st;
   st = st > n_slabs ? n_slabs : st;
   return st < 2 ? 2 : st;
 }
-inline int smem_bytes(int N, int stages, int parts) { return stages * stage_bytes(N, parts) + (N + 4) * 512 + 1024 + 256; }
+inline int smem_bytes(int N, int stages, int parts, int side_b) {
+  return stages * stage_bytes(N, parts) + (N + 4) * 512 + side_b + 1024 + 256;
+}
 
 inline int max_smem_bytes() {
-  const int a = smem_bytes(32, pick_stages(32, MAX_STAGES, 1), 1), b = smem_bytes(32, pick_stages(32, MAX_STAGES, 2), 2);
+  const int sb = side_bytes(32, 1);
+  const int a = smem_bytes(32, pick_stages(32, MAX_STAGES, 1, sb), 1, sb), b = smem_bytes(32, pick_stages(32, MAX_STAGES, 2, sb), 2, sb);
   return a > b ? a : b;
 }
 
@@ -192,7 +201,9 @@ __device__ inline void pair_cols(int q, bool head128, int& ca, int& cb) {
 
 // grid (M/128 tiles, split, N tiles of the token rows), cluster (1, split, 1); block 128.  Warp 0 lane 0 feeds TMA, warp 1
 // lane 0 issues MMAs, all four warps read the accumulator back (warp w owns TMEM lanes 32w..32w+31).
-template <int MODE>
+// SIDE: the launch has side rows (side_bytes(N, split) > 0); a separate instantiation, because the
+// mere presence of that path costs the few-row launches 0.4 us each (measured).
+template <int MODE, bool SIDE>
 __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e) {
   if (g.n_active != nullptr && *g.n_active == 0) {   // the whole grid leaves; keep the launch chain ordered
     ptx::grid_dep_launch();
@@ -206,11 +217,13 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   const int stage_bytes = BM * 128 + g.a_parts * b_bytes;
   const int NP = g.N + 4;
   float* recv = reinterpret_cast<float*>(sm + STAGES * stage_bytes);          // [S][PW][2][NP]
-  uint64_t* full = reinterpret_cast<uint64_t*>(sm + STAGES * stage_bytes + NP * 512);
+  float* side = recv + NP * 128;                                              // [N][128] fp32 (or [N][64] float2)
+  uint64_t* full = reinterpret_cast<uint64_t*>(sm + STAGES * stage_bytes + NP * 512 + (SIDE ? g.N * 512 : 0));
   uint64_t* empty = full + MAX_STAGES;
   uint64_t* accum = empty + MAX_STAGES;
   uint64_t* rbar = accum + 1;                                                 // partials of all ranks have arrived
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(rbar + 1);
+  uint64_t* sbar = rbar + 1;                                                  // side rows have arrived
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sbar + 1);
   __shared__ int s_fail;
   __shared__ float s_inv[256];
   __shared__ int s_rb[256], s_rp[256];
@@ -236,6 +249,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
     for (int i = 0; i < STAGES; ++i) { ptx::mbar_init(full + i, 1); ptx::mbar_init(empty + i, 1); }
     ptx::mbar_init(accum, 1);
     ptx::mbar_init(rbar, 1);
+    ptx::mbar_init(sbar, 1);
     ptx::fence_mbar_init();
     // rows are sent in groups of 16: groups x 16 rows x 128/S columns x S ranks x 4 bytes
     ptx::mbar_expect_tx(rbar, (uint32_t)((ns + 15) / 16) * 16u * 512u);
@@ -265,6 +279,13 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   // CTA of the cluster runs and has initialised them.
   if (S > 1) cluster_sync();
 
+  // side rows: residual rows of this tile's columns (EPI_RESID that adds), or the rows' rotary
+  // angles (EPI_QKV tiles that hold query or key heads)
+  // Only when a thread has more than two items: with fewer, loads straight into registers right
+  // after the dependency wait are quicker than the round through the copy engine (measured).
+  const bool want_side = (MODE == EPI_RESID && e.add != 0) ||
+                         (MODE == EPI_QKV && e.dm.theta != 0.f && (tile_m * BM) / e.dm.dh < e.dm.H + e.dm.Hkv);
+  const bool use_side = SIDE && want_side;
   if (warp == 0) {
     // ---- operand rows of the first stages (their weight slabs are already on their way): one
     // copy per slab brings the hi and the lo tile; lanes issue them side by side
@@ -304,7 +325,33 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
     // ---- warps 2 and 3, while the operands arrive: operand-row scales (the partial sums of
     // squares of a row are gathered by 8 lanes, each adding its slots in slot order, then combined by
     // a fixed shuffle tree) and row maps
+    if (MODE == EPI_QKV && warp == 3) {
+      // row maps, and the rows' rotary angles into the side buffer: positions are per-pass state
+      // and the table is constant, so nothing here waits for the previous kernel
+      const uint32_t row_bytes = (uint32_t)e.dm.dh * 4u;   // dh/2 (cos, sin) pairs
+      uint32_t total = 0;
+      for (int n0 = 0; n0 < ns; n0 += 32) {
+        const int n = n0 + lane;
+        int b = 0, p = 0;
+        const bool valid = n < ns && fm_row_map(e.dm, e.st, e.batch, e.level, row0 + n, b, p);
+        if (n < ns) { s_rb[n] = valid ? b : -1; s_rp[n] = p; }
+        total += (uint32_t)__popc(__ballot_sync(0xffffffffu, valid)) * row_bytes;
+      }
+      if (use_side) {
+        if (lane == 0) ptx::mbar_expect_tx(sbar, total);
+        __syncwarp();
+        for (int n = lane; n < ns; n += 32)
+          if (s_rb[n] >= 0) ptx::bulk_load(side + n * 128, e.rope_tab + (size_t)s_rp[n] * (e.dm.dh >> 1), row_bytes, sbar);
+      }
+    }
     ptx::grid_dep_wait();
+    if (MODE == EPI_RESID && use_side && warp == 2) {      // residual rows of this tile's columns
+      const int cols = min(BM, g.M - tile_m * BM);
+      if (lane == 0) ptx::mbar_expect_tx(sbar, (uint32_t)(ns * cols) * 4u);
+      __syncwarp();
+      for (int n = lane; n < ns; n += 32)
+        ptx::bulk_load(side + n * 128, e.x + (size_t)(row0 + n) * e.ldx + tile_m * BM, (uint32_t)cols * 4u, sbar);
+    }
     const int t = tid - 64;
     if (e.ssq_in != nullptr) {
       const int sub = t & 7;
@@ -329,14 +376,6 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
     } else {
       for (int n = t; n < ns; n += 64) s_inv[n] = 1.f;
     }
-    if (MODE == EPI_QKV) {
-      for (int n = t; n < ns; n += 64) {
-        int b, p;
-        const bool valid = fm_row_map(e.dm, e.st, e.batch, e.level, row0 + n, b, p);
-        s_rb[n] = valid ? b : -1;
-        s_rp[n] = p;
-      }
-    }
   }
   __syncwarp();
 
@@ -360,49 +399,48 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
       dbar = map_peer(ptx::smem_u32(rbar), (uint32_t)owner);
     }
   }
+  // A thread keeps its pair slot in every item (items advance by 128, a multiple of PW): its two
+  // columns, and with them the gains, are fixed.
   float pre_ga = 1.f, pre_gb = 1.f;
-  float2 pre_cs = make_float2(1.f, 0.f);
+  float2 pre_cs = make_float2(1.f, 0.f);                   // first item's rotary angle when the side rows are not used
   if (tid < items) {
-    const int n = tid >> lgPW, cc = tid & (PW - 1);
     int ca, cb;
-    pair_cols(z * PW + cc, head128, ca, cb);
+    pair_cols(z * PW + (tid & (PW - 1)), head128, ca, cb);
     const int ma = tile_m * BM + ca, mb = tile_m * BM + cb;
     if (MODE == EPI_RESID && e.gain != nullptr) {
       if (ma < g.M) pre_ga = e.gain[ma];
       if (mb < g.M) pre_gb = e.gain[mb];
     }
-    if (MODE == EPI_QKV && e.dm.theta != 0.f) {
+    if (MODE == EPI_QKV && want_side && !use_side) {
       int b, p;
-      const bool valid = fm_row_map(e.dm, e.st, e.batch, e.level, row0 + n, b, p);
+      const bool valid = fm_row_map(e.dm, e.st, e.batch, e.level, row0 + (tid >> lgPW), b, p);
       const int head = ma / e.dm.dh, i = ma - head * e.dm.dh;
       if (valid && ma < g.M && head < e.dm.H + e.dm.Hkv) pre_cs = e.rope_tab[(size_t)p * (e.dm.dh >> 1) + i];
     }
   }
   // Kernel parameters the tail needs, read into registers now: a first touch of the parameter
   // bank after the wait would sit on the critical path.
-  int k_row0 = row0, k_ldo = e.ldo, k_ldx = e.ldx, k_add = e.add, k_lda = e.lda, k_ldssq = e.ld_ssq_out;
+  int k_row0 = row0, k_ldo = e.ldo, k_ldx = e.ldx, k_lda = e.lda, k_ldssq = e.ld_ssq_out;
   int k_M = g.M, k_ns = ns, k_lo = e.lo_off;
   void* k_out = e.out;
   float* k_x = e.x;
-  const float* k_gain = e.gain;
   bf16* k_aout = e.a_out;
   float* k_ssqo = e.ssq_out;
   bf16 *k_q = e.q_out, *k_K = e.Kc, *k_V = e.Vc;
-  const float2* k_rope = e.rope_tab;
-  float k_qs = e.qscale, k_theta = e.dm.theta;
+  float k_qs = e.qscale;
   int k_H = e.dm.H, k_Hkv = e.dm.Hkv, k_dh = e.dm.dh, k_P = e.dm.P, k_cap = MODE == EPI_QKV ? e.dm.cap[e.level] : 1;
   int* k_status = g.status;
-  asm volatile("" : "+r"(k_row0), "+r"(k_ldo), "+r"(k_ldx), "+r"(k_add), "+r"(k_lda), "+r"(k_ldssq), "+r"(k_M), "+r"(k_ns), "+r"(k_lo));
-  asm volatile("" : "+l"(k_out), "+l"(k_x), "+l"(k_gain), "+l"(k_aout), "+l"(k_ssqo), "+l"(k_q), "+l"(k_K), "+l"(k_V), "+l"(k_rope), "+l"(k_status));
-  asm volatile("" : "+f"(k_qs), "+f"(k_theta), "+r"(k_H), "+r"(k_Hkv), "+r"(k_dh), "+r"(k_P), "+r"(k_cap));
+
+  asm volatile("" : "+r"(k_row0), "+r"(k_ldo), "+r"(k_ldx), "+r"(k_lda), "+r"(k_ldssq), "+r"(k_M), "+r"(k_ns), "+r"(k_lo));
+  asm volatile("" : "+l"(k_out), "+l"(k_x), "+l"(k_aout), "+l"(k_ssqo), "+l"(k_q), "+l"(k_K), "+l"(k_V), "+l"(k_status));
+  asm volatile("" : "+f"(k_qs), "+r"(k_H), "+r"(k_Hkv), "+r"(k_dh), "+r"(k_P), "+r"(k_cap));
   ptx::grid_dep_wait();                                    // everything below touches activations
-  float pre_xa = 0.f, pre_xb = 0.f;
-  if (MODE == EPI_RESID && k_add && tid < items) {
-    const int n = tid >> lgPW, cc = tid & (PW - 1);
+  float pre_xa = 0.f, pre_xb = 0.f;                        // first item's residual values, same case
+  if (MODE == EPI_RESID && want_side && !use_side && tid < items) {
     int ca, cb;
-    pair_cols(z * PW + cc, head128, ca, cb);
+    pair_cols(z * PW + (tid & (PW - 1)), head128, ca, cb);
     const int ma = tile_m * BM + ca, mb = tile_m * BM + cb;
-    const float* xr = k_x + (size_t)(k_row0 + n) * k_ldx;
+    const float* xr = k_x + (size_t)(k_row0 + (tid >> lgPW)) * k_ldx;
     if (ma < k_M) pre_xa = xr[ma];
     if (mb < k_M) pre_xb = xr[mb];
   }
@@ -448,6 +486,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   bool arrived = true;
   if (S > 1) arrived = mbar_wait_cluster(rbar, 0);
   else __syncthreads();
+  if (use_side) arrived = ptx::mbar_wait(sbar, 0) && arrived;
   if (!ok || !arrived || s_fail) {
     if (tid == 0) atomicExch(k_status, -5);
   }
@@ -492,14 +531,14 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
       float* xr = k_x + row * k_ldx;
       float xa = 0.f, xb = 0.f;
       if (a_ok) {
-        xa = (first ? pre_xa : (k_add ? xr[ma] : 0.f)) + ya;
+        xa = (use_side ? side[n * 128 + ca] : (first ? pre_xa : (want_side ? xr[ma] : 0.f))) + ya;
         xr[ma] = xa;
-        if (k_aout != nullptr) store_hi_lo(k_aout + row * k_lda + ma, xa * (first ? pre_ga : (k_gain != nullptr ? k_gain[ma] : 1.f)), k_lo);
+        if (k_aout != nullptr) store_hi_lo(k_aout + row * k_lda + ma, xa * pre_ga, k_lo);
       }
       if (b_ok) {
-        xb = (first ? pre_xb : (k_add ? xr[mb] : 0.f)) + yb;
+        xb = (use_side ? side[n * 128 + cb] : (first ? pre_xb : (want_side ? xr[mb] : 0.f))) + yb;
         xr[mb] = xb;
-        if (k_aout != nullptr) store_hi_lo(k_aout + row * k_lda + mb, xb * (first ? pre_gb : (k_gain != nullptr ? k_gain[mb] : 1.f)), k_lo);
+        if (k_aout != nullptr) store_hi_lo(k_aout + row * k_lda + mb, xb * pre_gb, k_lo);
       }
       if (k_ssqo != nullptr) {
         // per-row sums of squares of this rank's columns: a fixed shuffle tree over the L lanes that
@@ -518,8 +557,9 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
         const int slots = k_P + k_cap;
         if (head < H + Hkv) {
           float2 cs = make_float2(1.f, 0.f);
-          if (first) cs = pre_cs;
-          else if (k_theta != 0.f && valid) cs = k_rope[(size_t)p * half + i];
+          if (use_side) { if (valid) cs = reinterpret_cast<const float2*>(side)[n * 64 + i]; }
+          else if (first) cs = pre_cs;
+          else if (want_side && valid) cs = e.rope_tab[(size_t)p * half + i];
           const float y1 = ya * cs.x - yb * cs.y, y2 = yb * cs.x + ya * cs.y;
           if (head < H) {
             bf16* q = k_q + (row * H + head) * dh;
