@@ -69,7 +69,7 @@ def rank_sequences(rank, batch_per_rank):
 # DRAM traffic of the dominant kernel per launch from ncu (dram__bytes_read.sum +
 # dram__bytes_write.sum; profiles/gemm_traffic_medium.md), keyed by workload; None where the kernel
 # changed since the capture or none was taken.
-NCU_TRAFFIC = {"medium": 6.47e6}      # bytes per GEMM launch, mean over the four projections of a layer
+NCU_TRAFFIC = {"medium": 6.46e6}      # bytes per GEMM launch, mean over the four projections of a layer
 
 
 class ClockSampler:
