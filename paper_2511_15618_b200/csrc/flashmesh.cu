@@ -228,13 +228,26 @@ void carve(fm_ctx* c, Carver& cv) {
   for (int l = 0; l < 3; ++l) {
     const int max_chunks = (dm.P + dm.cap[l] + c->attn_chunk - 1) / c->attn_chunk;
     c->attn_mt[l] = (fm_rows_per_seq(dm, l) * (dm.H / dm.Hkv) + 15) / 16;
-    // about one CTA per SM when the cache is full; at most 16 chunks per group
-    int G = (int)(((size_t)max_chunks * dm.Hkv * B * c->attn_mt[l] + 147) / 148);
-    G = G < 1 ? 1 : (G > 16 ? 16 : G);
-    // the groups' states (and weights) are merged from shared memory: 24 groups at most, fewer for wide heads
+    // Chunks per group: the number of groups (1 .. what the merge can stage: 24, fewer for wide
+    // heads) that minimises waves x (chunks per CTA + a CTA's fixed cost), with the cache full.
+    // The fixed cost (pipeline start, merge of the warps, and with several groups the partials,
+    // the ticket and the last CTA's merge) was measured at batch 16 as about 5 chunk times:
+    // 87 / 70 / 63 / 61 us per launch with at most 8 / 16 / 32 / 64 chunks per group.
     const int g_cap = dm.dh == 64 ? AttnCfg<64, 128, 8>::MAX_GROUPS : AttnCfg<128, 64, 4>::MAX_GROUPS;
-    const int G_min = (max_chunks + g_cap - 1) / g_cap;
-    G = G < G_min ? G_min : G;
+    const size_t tiles_l = (size_t)dm.Hkv * B * c->attn_mt[l];
+    int G = max_chunks;
+    double best = 0.0;
+    for (int ng = 1; ng <= g_cap && ng <= max_chunks; ++ng) {
+      const int Gc = (max_chunks + ng - 1) / ng, groups = (max_chunks + Gc - 1) / Gc;
+      const size_t waves = (tiles_l * groups + 147) / 148;
+      const double cost = (double)waves * (Gc + (groups == 1 ? 3 : 6));
+      if (ng == 1 || cost < best) { best = cost; G = Gc; }
+    }
+    const char* gm = getenv("FM_ATTN_G");                 // tuning knob: chunks per group, all levels
+    if (gm != nullptr && atoi(gm) > 0) {
+      const int G_min = (max_chunks + g_cap - 1) / g_cap;
+      G = atoi(gm) < G_min ? G_min : atoi(gm);
+    }
     c->attn_G[l] = G;
     c->attn_max_groups[l] = (max_chunks + G - 1) / G;
     const size_t need = B * dm.Hkv * (size_t)c->attn_mt[l] * c->attn_max_groups[l] * 16 * (dm.dh + 2);

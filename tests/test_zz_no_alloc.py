@@ -57,11 +57,14 @@ def test_static_scratch_verify_matches_fm_verify_twice_in_a_row():
     assert int(n_acc[0]) >= 1
 
 
-def test_static_scratch_rejects_a_configuration_that_needs_more_than_the_array():
+def test_static_scratch_rejects_a_configuration_that_needs_more_than_the_array(monkeypatch):
     from paper_2511_15618_b200 import FlashMesh, fm_verify_static_scratch
     import torch
 
-    # many sequences and kv-heads with long caches: the group partials outgrow the fixed array
+    # many sequences and kv-heads with long caches cut into many groups (the tuning knob asks for
+    # short groups; the library then takes the largest number of groups it can merge): the group
+    # partials outgrow the fixed array
+    monkeypatch.setenv("FM_ATTN_G", "8")
     cfg = S.get_config("tiny").with_(max_batch=16, max_tokens=100000)
     w = S.make_weights(cfg)
     dev = FlashMesh(cfg, w)
