@@ -165,6 +165,8 @@ def run_ours(args):
         seq = np.concatenate([np.asarray(prompts[b], np.int32), pt[b]])
         truth[b, :len(seq)] = seq
     keep = (S.accept_schedule(cfg.seed + rank, B, 4096, D, MEAN_DRAFTS) - 1).astype(np.int32)
+    if args.pin_accept > 0:               # every pass accepts exactly this many tokens (main + drafts)
+        keep[:] = min(D, args.pin_accept - 1)
     truth_d = torch.as_tensor(truth).cuda()
     keep_d = torch.as_tensor(keep).cuda()
 
@@ -412,6 +414,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-batched", action="store_true", help="skip the batch-16 add-on of the default run")
     ap.add_argument("--timed-only", action="store_true", help="stop after the timed passes (for profiler captures)")
+    ap.add_argument("--pin-accept", type=int, default=0,
+                    help="teacher drafts with the true acceptance pinned to this many tokens per pass (1 .. D+1); 0 = seeded schedule")
     args = ap.parse_args()
     args.warmup = max(3, args.warmup) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
