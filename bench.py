@@ -282,6 +282,22 @@ def run_ours(args):
                         "frac_of_hbm_peak": step_bytes / (step_ms * 1e-3) / 1e9 / peak, "kv_len": kv_len[0],
                         "note": "whole pass (draft heads + verify + accept) against the verify bytes"},
     }
+    # ---- the correction stage between draft and verify (an integer kernel, outside the timed passes):
+    # random labels on the drafts of the current state, 200 calls between two events
+    cand, _, _ = dev.draft()
+    lab = torch.randint(0, 3, cand.shape, dtype=torch.int32, device=cand.device)
+    for _ in range(5):
+        dev.correct(cand.clone(), lab)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    work = [cand.clone() for _ in range(200)]
+    e0.record()
+    for w_ in work:
+        dev.correct(w_, lab)
+    e1.record()
+    torch.cuda.synchronize()
+    line["correct_stage"] = {"us_per_call": 1e3 * e0.elapsed_time(e1) / 200, "batch": B, "slots_per_row": D + 1,
+                             "note": "fm_correct on random labels; host bound (binding call + launch per call); not part of the timed passes"}
     if rank == 0:
         if world == 1 and args.workload == "medium" and not args.no_batched:
             # the metric also asks for batch 16: the batched-ragged workload, timed passes only

@@ -147,6 +147,25 @@ int fm_set_max_faces(fm_ctx* ctx, const int32_t* max_faces /*HOST*/);
  * [batch, D] (top-1 minus top-2 of the masked draft logits) or NULL. */
 int fm_draft(fm_ctx* ctx, int32_t* cand /*DEV*/, float* draft_logits /*DEV*/, float* draft_margin /*DEV*/);
 
+/* Correct (Sec. 3.2 "Correction Mechanism"): edit the drafts of a candidate row in place, between
+ * fm_draft and fm_verify.  A point is a vertex whose three coordinate tokens (z, y, x) are all
+ * drafts of this pass (slot s of sequence b holds mesh token L[b] - 1 + s; slot 0 is the main
+ * token and is never touched; vertices that are only partly in the row, or that hold a token that
+ * is not a coordinate bin, are left alone).  labels: DEV int32 [batch, D+1]; labels[b][s] is the
+ * label of the point that starts at slot s: FM_LABEL_HISTORICAL, FM_LABEL_NEW or FM_LABEL_INTRA
+ * (other slots are not read; the label head that would produce them is not part of the library).
+ * In sequence order, every FM_LABEL_INTRA point that has no identical point in the row is
+ * replaced by the nearest (squared distance between bin indices, ties to the earliest) earlier
+ * FM_LABEL_NEW point of another face, if there is one; then the points of every face are sorted
+ * ascending by (z, y, x) among the slots they occupy.  Only rows the next pass feeds
+ * (the first nrow slots of an unfinished sequence) are considered.
+ * cand: DEV int32 in/out [batch, D+1].  Errors: INVALID_ARG (null pointer), BAD_STATE (before
+ * fm_prefill), UNSUPPORTED (more than 48 slots per row; cannot happen while FM_MAX_DRAFT is 24). */
+#define FM_LABEL_HISTORICAL 0
+#define FM_LABEL_NEW 1
+#define FM_LABEL_INTRA 2
+int fm_correct(fm_ctx* ctx, int32_t* cand /*DEV*/, const int32_t* labels /*DEV*/);
+
 /* Verify (Sec. 3.3): one forward pass over main + D candidates, causal among themselves,
  * through all five level stacks.  cand: DEV int32 in [batch, D+1]; cand[b][0] must be the
  * pending main token.  Rows fed per sequence = min(D+1, tokens left).  argmax: DEV int32 out

@@ -87,6 +87,8 @@ def load_library():
     lib.fm_set_max_faces.argtypes = [vp, C.POINTER(C.c_int32)]
     lib.fm_draft.restype = C.c_int
     lib.fm_draft.argtypes = [vp, vp, f32p, f32p]
+    lib.fm_correct.restype = C.c_int
+    lib.fm_correct.argtypes = [vp, vp, vp]
     lib.fm_verify.restype = C.c_int
     lib.fm_verify.argtypes = [vp, vp, vp, f32p, f32p]
     lib.fm_verify_static_scratch.restype = C.c_int
@@ -147,6 +149,10 @@ def fm_set_max_faces(ctx, max_faces):
 
 def fm_draft(ctx, cand_ptr, draft_logits_ptr=None, draft_margin_ptr=None):
     return load_library().fm_draft(ctx, cand_ptr, draft_logits_ptr, draft_margin_ptr)
+
+
+def fm_correct(ctx, cand_ptr, labels_ptr):
+    return load_library().fm_correct(ctx, cand_ptr, labels_ptr)
 
 
 def fm_verify(ctx, cand_ptr, argmax_ptr=None, logits_ptr=None, margin_ptr=None):
@@ -339,6 +345,14 @@ class FlashMesh:
                              dm.data_ptr() if dm is not None and D > 0 else None), "fm_draft")
         self._after(cand, dl, dm)
         return cand, dl, dm
+
+    def correct(self, cand, labels):
+        """Edit the drafts of `cand` (int32 [B, D+1], device) in place with the per-point labels
+        (int32 [B, D+1], device); returns `cand`."""
+        self._before()
+        self._check(fm_correct(self.ctx, cand.data_ptr(), labels.data_ptr()), "fm_correct")
+        self._after(cand, labels)
+        return cand
 
     def verify(self, cand, want_logits=False):
         t = self.torch

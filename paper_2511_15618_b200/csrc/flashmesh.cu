@@ -1061,6 +1061,16 @@ int fm_draft(fm_ctx* c, int32_t* cand, float* draft_logits, float* draft_margin)
   return FM_OK;
 }
 
+int fm_correct(fm_ctx* c, int32_t* cand, const int32_t* labels) {
+  if (c == nullptr || cand == nullptr || labels == nullptr) return FM_ERR_INVALID_ARG;
+  if (c->phase < 1) return FM_ERR_BAD_STATE;
+  if (c->dm.R1 > 3 * FM_CORRECT_MAX_POINTS) return FM_ERR_UNSUPPORTED;
+  LAUNCH(c, correct_kernel, (c->batch + 63) / 64, 64, 0, c->dm, c->st, c->batch, cand, labels);
+  CUDA_OK(cudaGetLastError());
+  if (c->launch_error != FM_OK) return c->launch_error;
+  return FM_OK;
+}
+
 int fm_verify(fm_ctx* c, const int32_t* cand, int32_t* argmax, float* logits, float* margin) {
   if (c == nullptr || cand == nullptr) return FM_ERR_INVALID_ARG;
   if (c->phase < 1) return FM_ERR_BAD_STATE;

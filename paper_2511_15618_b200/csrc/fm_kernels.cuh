@@ -495,3 +495,79 @@ __global__ void copy_f32_kernel(const float* __restrict__ src, float* __restrict
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) dst[i] = src[i];
 }
+
+// ------------------------------------------------------------------------------------------
+// Correction of the drafts (Sec. 3.2), one thread per sequence: a row has at most 16 points.
+// Slot s of a row is mesh token L - 1 + s; a point is a vertex (3 slots, mesh token index a
+// multiple of 3) made of drafts only, inside the rows the next pass feeds.
+// ------------------------------------------------------------------------------------------
+constexpr int FM_CORRECT_MAX_POINTS = 16;
+
+__device__ inline bool vertex_less(const int* a, const int* b) {       // (z, y, x) order
+  if (a[0] != b[0]) return a[0] < b[0];
+  if (a[1] != b[1]) return a[1] < b[1];
+  return a[2] < b[2];
+}
+
+__global__ void correct_kernel(Dims dm, SeqState st, int batch, int* __restrict__ cand, const int* __restrict__ labels) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= batch) return;
+  const int n = st.nrow[b];
+  if (n <= 0) return;
+  int* row = cand + (size_t)b * dm.R1;
+  const int* lab = labels + (size_t)b * dm.R1;
+  const int first = st.L[b] - 1;                 // mesh token index of slot 0
+  int slot[FM_CORRECT_MAX_POINTS], face[FM_CORRECT_MAX_POINTS], kind[FM_CORRECT_MAX_POINTS];
+  bool usable[FM_CORRECT_MAX_POINTS];
+  int m = 0;
+  for (int s = 1; s + 2 < n && m < FM_CORRECT_MAX_POINTS; ++s) {
+    const int j = first + s;
+    if (j % 3 != 0) continue;
+    slot[m] = s;
+    face[m] = j / 9;
+    kind[m] = lab[s];
+    usable[m] = row[s] >= 0 && row[s] < dm.n_bins && row[s + 1] >= 0 && row[s + 1] < dm.n_bins && row[s + 2] >= 0 &&
+                row[s + 2] < dm.n_bins;
+    ++m;
+  }
+  // intra-batch points in sequence order; each sees the corrections before it
+  for (int k = 0; k < m; ++k) {
+    if (kind[k] != 2 || !usable[k]) continue;
+    const int z = row[slot[k]], y = row[slot[k] + 1], x = row[slot[k] + 2];
+    bool twin = false;
+    for (int q = 0; q < m; ++q)
+      if (q != k && usable[q] && row[slot[q]] == z && row[slot[q] + 1] == y && row[slot[q] + 2] == x) twin = true;
+    if (twin) continue;
+    int src = -1;
+    long long best = 0;
+    for (int q = 0; q < k; ++q) {
+      if (kind[q] != 1 || !usable[q] || face[q] == face[k]) continue;
+      const long long dz = row[slot[q]] - z, dy = row[slot[q] + 1] - y, dx = row[slot[q] + 2] - x;
+      const long long dist = dz * dz + dy * dy + dx * dx;
+      if (src < 0 || dist < best) { src = q; best = dist; }
+    }
+    if (src >= 0) {
+      row[slot[k]] = row[slot[src]];
+      row[slot[k] + 1] = row[slot[src] + 1];
+      row[slot[k] + 2] = row[slot[src] + 2];
+    }
+  }
+  // z-y-x order inside every face, among the slots its usable points occupy (a face has at most
+  // three): exchange sort on the triples
+  for (int k0 = 0; k0 < m;) {
+    int k1 = k0;
+    while (k1 < m && face[k1] == face[k0]) ++k1;
+    for (int i = k0; i < k1; ++i) {
+      if (!usable[i]) continue;
+      for (int j = i + 1; j < k1; ++j) {
+        if (!usable[j]) continue;
+        int* a = row + slot[i];
+        int* c = row + slot[j];
+        if (vertex_less(c, a)) {
+          for (int t = 0; t < 3; ++t) { const int tmp = a[t]; a[t] = c[t]; c[t] = tmp; }
+        }
+      }
+    }
+    k0 = k1;
+  }
+}
