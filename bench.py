@@ -139,6 +139,8 @@ def run_ours(args):
     if world > 1:
         dist.barrier()
     cfg = S.get_config(args.workload)
+    if args.draft_len >= 0:               # cost curve of the pass against the number of drafts
+        cfg = cfg.with_(draft_len=args.draft_len)
     B, D = cfg.batch, cfg.draft_len
     K, W = args.steps, args.warmup
     start_faces = int(cfg.gen_faces * args.start_frac)
@@ -310,6 +312,24 @@ def run_ours(args):
                 line["batch16"] = json.loads(r.stdout.strip().splitlines()[-1])
             except Exception:
                 line["batch16"] = {"error": (r.stderr or r.stdout)[-300:]}
+        if world == 1 and args.draft_len < 0 and not args.no_batched:
+            # T_ori of Sec. 4.1: the same model decoding one token per pass (D = 0, so the vertex and
+            # face stacks only run at multiples of 3 and 9), same kernels, same cache fill
+            try:
+                dev.close()
+                del dev
+                torch.cuda.empty_cache()
+            except NameError:
+                pass
+            r = subprocess.run([sys.executable, os.path.abspath(__file__), "--workload", args.workload, "--steps", "90", "--warmup", "9",
+                                "--draft-len", "0", "--timed-only", "--no-cpu"], capture_output=True, text=True)
+            try:
+                p0 = json.loads(r.stdout.strip().splitlines()[-1])
+                line["plain_decoding"] = {"tokens_per_s": p0["value"], "ms_per_token": p0["ms_per_step"], "draft_len": 0,
+                                          "speed_up": line["value"] / p0["value"],
+                                          "note": "S = T_ori * m / T_ours (Sec. 4.1) with T_ori from this run"}
+            except Exception:
+                line["plain_decoding"] = {"error": (r.stderr or r.stdout)[-300:]}
         if world == 1 and not args.no_cpu:
             line["cpu_baseline"] = cpu_baseline(args.workload, budget_s=args.cpu_seconds)
         print(json.dumps(line), flush=True)
@@ -430,6 +450,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-batched", action="store_true", help="skip the batch-16 add-on of the default run")
     ap.add_argument("--timed-only", action="store_true", help="stop after the timed passes (for profiler captures)")
+    ap.add_argument("--draft-len", type=int, default=-1, help="override the workload's number of drafts D (0 = plain decoding)")
     ap.add_argument("--pin-accept", type=int, default=0,
                     help="teacher drafts with the true acceptance pinned to this many tokens per pass (1 .. D+1); 0 = seeded schedule")
     args = ap.parse_args()
