@@ -353,7 +353,7 @@ def run_e2e(dev, cfg, truth, keep, prompts, steps):
     torch.cuda.synchronize()
     t0 = time.perf_counter()
     for s in range(steps):
-        dev.draft()                                           # heads run; their drafts are replaced below
+        dev.draft(reuse=True)                                 # heads run; their drafts are replaced below
         for b in range(B):
             n = L[b] - 1
             k = int(keep[s % keep.shape[0], b])
@@ -362,8 +362,8 @@ def run_e2e(dev, cfg, truth, keep, prompts, steps):
                 row[k + 1] = (row[k + 1] + 1) % cfg.n_bins
             cand_h[b] = torch.from_numpy(row)
         cand_d.copy_(cand_h, non_blocking=True)
-        dev.verify(cand_d)
-        n_acc, em, _ = dev.accept()
+        dev.verify(cand_d, reuse=True)                        # same buffers every pass: replayed as one graph
+        n_acc, em, _ = dev.accept(reuse=True)
         nacc_h.copy_(n_acc, non_blocking=True)
         em_h.copy_(em, non_blocking=True)
         torch.cuda.synchronize()

@@ -19,6 +19,10 @@
  *     (or the context destroyed).
  *   - Pointers are marked HOST or DEV.  DEV pointers are caller-owned device memory that must
  *     stay valid until the work enqueued by the call has finished on the context's stream.
+ *   - fm_draft and fm_verify launch their kernels one by one the first time they see a set of
+ *     pointer arguments, capture them into a CUDA graph when the same pointers come again, and
+ *     replay that graph afterwards: a host that drives the loop call by call should pass the same
+ *     buffers every pass.  (A stream that cannot be captured keeps the plain launches.)
  *   - All calls except fm_create / fm_destroy / fm_generate only enqueue work on the
  *     context's stream and return; fm_generate polls a completion flag and returns when every
  *     sequence has finished.

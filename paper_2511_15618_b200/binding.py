@@ -314,6 +314,18 @@ class FlashMesh:
     def _empty(self, shape, dtype):
         return self.torch.empty(shape, dtype=dtype, device=self.device)
 
+    def _out(self, name, shape, dtype, reuse):
+        """An output buffer: a fresh one, or with `reuse` the same one on every call (the library
+        replays a call whose pointers repeat as one CUDA graph; the next call overwrites it)."""
+        if not reuse:
+            return self._empty(shape, dtype)
+        key = (name, tuple(shape), dtype)
+        if not hasattr(self, "_held"):
+            self._held = {}
+        if key not in self._held:
+            self._held[key] = self._empty(shape, dtype)
+        return self._held[key]
+
     def prefill(self, cond, prompts):
         """cond: [B,P,d] float32 (tensor or array); prompts: list of int sequences."""
         t = self.torch
@@ -334,11 +346,11 @@ class FlashMesh:
         self._check(fm_set_max_faces(self.ctx, list(max_faces)), "fm_set_max_faces")
         self._after()
 
-    def draft(self, want_logits=False):
+    def draft(self, want_logits=False, reuse=False):
         t = self.torch
         B, D = self.batch, self.D
-        cand = self._empty((B, D + 1), t.int32)
-        dl = self._empty((B, D, self.V), t.float32) if want_logits else None
+        cand = self._out("cand", (B, D + 1), t.int32, reuse)
+        dl = self._out("dl", (B, D, self.V), t.float32, reuse) if want_logits else None
         dm = self._empty((B, max(D, 1)), t.float32)[:, :D].contiguous() if want_logits else None
         self._before()
         self._check(fm_draft(self.ctx, cand.data_ptr(), dl.data_ptr() if dl is not None else None,
@@ -354,27 +366,27 @@ class FlashMesh:
         self._after(cand, labels)
         return cand
 
-    def verify(self, cand, want_logits=False):
+    def verify(self, cand, want_logits=False, reuse=False):
         t = self.torch
         B, D = self.batch, self.D
         cand = self._dev(cand, t.int32)
-        o = self._empty((B, D + 1), t.int32)
-        mg = self._empty((B, D + 1), t.float32)
-        lg = self._empty((B, D + 1, self.V), t.float32) if want_logits else None
+        o = self._out("o", (B, D + 1), t.int32, reuse)
+        mg = self._out("mg", (B, D + 1), t.float32, reuse)
+        lg = self._out("lg", (B, D + 1, self.V), t.float32, reuse) if want_logits else None
         self._before()
         self._check(fm_verify(self.ctx, cand.data_ptr(), o.data_ptr(), lg.data_ptr() if lg is not None else None,
                               mg.data_ptr()), "fm_verify")
         self._after(cand, o, lg, mg)
         return o, lg, mg
 
-    def accept(self, force_len=None, force_tok=None):
+    def accept(self, force_len=None, force_tok=None, reuse=False):
         t = self.torch
         B, D = self.batch, self.D
         fl = self._dev(force_len, t.int32) if force_len is not None else None
         ft = self._dev(force_tok, t.int32) if force_tok is not None else None
-        n_acc = self._empty((B,), t.int32)
-        em = self._empty((B, D + 1), t.int32)
-        kv = self._empty((B, 3), t.int32)
+        n_acc = self._out("n_acc", (B,), t.int32, reuse)
+        em = self._out("em", (B, D + 1), t.int32, reuse)
+        kv = self._out("kv", (B, 3), t.int32, reuse)
         self._before()
         self._check(fm_accept(self.ctx, fl.data_ptr() if fl is not None else None,
                               ft.data_ptr() if ft is not None else None, n_acc.data_ptr(), em.data_ptr(),

@@ -106,6 +106,15 @@ struct fm_ctx {
   int graph_batch;
   int64_t graph_launches;
   bool capturing, graph_unavailable;
+  // Stepwise calls repeated with the same pointer arguments are replayed as CUDA graphs.
+  struct CallGraph {
+    const void* key[4] = {nullptr, nullptr, nullptr, nullptr};
+    int batch = -1;
+    bool valid = false, failed = false;
+    int64_t launches = 0;
+    cudaGraphExec_t exec = nullptr;
+  } cg_verify, cg_draft;
+  bool call_graphs_off;   // plain launches only (diagnostic modes, calls that swap scratch buffers)
   int batch;
   bool gen_fresh;       // no fm_generate call since the last fm_prefill
   std::vector<int> plen_host;
@@ -727,6 +736,66 @@ void drop_graph(fm_ctx* c) {
   c->graph = nullptr;
 }
 
+void drop_call_graph(fm_ctx::CallGraph& g) {
+  if (g.exec != nullptr) cudaGraphExecDestroy(g.exec);
+  g.exec = nullptr;
+  g.valid = false;
+  g.batch = -1;
+}
+
+// Runs `body` (which only enqueues work on the context's stream).  The first time a set of caller
+// pointers is seen the kernels are launched one by one (this also creates every descriptor the
+// path needs); when the same pointers come again the launches are captured into a graph, and
+// from then on the graph is replayed: a pass is 180 launches, and a host that drives the loop
+// call by call would otherwise pay for each of them.  All state the kernels read lives in device
+// memory, so the same graph serves every pass.
+template <typename F>
+void run_cached(fm_ctx* c, fm_ctx::CallGraph& g, const void* k0, const void* k1, const void* k2, const void* k3, F&& body) {
+  const bool off = c->call_graphs_off || c->graph_unavailable || c->debug_sync || c->prof_on || g.failed;
+  const bool same = g.valid && g.batch == c->batch && g.key[0] == k0 && g.key[1] == k1 && g.key[2] == k2 && g.key[3] == k3;
+  if (off) { body(); return; }
+  if (same && g.exec != nullptr) {
+    if (cudaGraphLaunch(g.exec, c->stream) != cudaSuccess) { cudaGetLastError(); c->launch_error = FM_ERR_CUDA; }
+    c->launches += g.launches;
+    return;
+  }
+  if (!same) {
+    drop_call_graph(g);
+    g.key[0] = k0; g.key[1] = k1; g.key[2] = k2; g.key[3] = k3;
+    g.batch = c->batch;
+    g.valid = true;
+    body();
+    return;
+  }
+  // same pointers as last time and no graph yet: capture
+  if (cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+    cudaGetLastError();
+    g.failed = true;
+    body();
+    return;
+  }
+  const int64_t l0 = c->launches;
+  c->capturing = true;
+  body();
+  c->capturing = false;
+  g.launches = c->launches - l0;
+  c->launches = l0;
+  cudaGraph_t gr = nullptr;
+  if (cudaStreamEndCapture(c->stream, &gr) != cudaSuccess || gr == nullptr || c->launch_error != FM_OK ||
+      cudaGraphInstantiate(&g.exec, gr, 0) != cudaSuccess) {
+    cudaGetLastError();
+    if (gr != nullptr) cudaGraphDestroy(gr);
+    g.exec = nullptr;
+    g.failed = true;
+    c->launch_error = FM_OK;
+    body();                                          // nothing ran during the failed capture
+    return;
+  }
+  cudaGraphDestroy(gr);
+  if (cudaGraphLaunch(g.exec, c->stream) != cudaSuccess) { cudaGetLastError(); c->launch_error = FM_ERR_CUDA; }
+  c->launches += g.launches;
+}
+
 // Capture the pass once per batch size.  All state the kernels read lives in device memory, so the
 // same graph serves every pass.  Streams that cannot be captured (the legacy default stream) fall
 // back to plain launches of the same kernels.
@@ -895,6 +964,8 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
     c->use_pdl = !(v != nullptr && v[0] == '1');
     const char* ds = getenv("FM_DEBUG_SYNC");
     c->debug_sync = ds != nullptr && ds[0] == '1';
+    const char* ncg = getenv("FM_NO_CALL_GRAPH");
+    c->call_graphs_off = ncg != nullptr && ncg[0] == '1';
     const char* t = getenv("FM_SPLIT_TARGET");
     c->split_target = t != nullptr && atoi(t) > 0 ? atoi(t) : 160;
     int dev = 0, sms = 148;
@@ -982,6 +1053,8 @@ int fm_destroy(fm_ctx* c) {
   cudaStreamSynchronize(c->stream);
   for (auto& e : c->prof_ev) cudaEventDestroy(e);
   drop_graph(c);
+  drop_call_graph(c->cg_verify);
+  drop_call_graph(c->cg_draft);
   if (c->host_done != nullptr) cudaFreeHost(c->host_done);
   delete c;
   return FM_OK;
@@ -1053,9 +1126,11 @@ int fm_set_max_faces(fm_ctx* c, const int32_t* max_faces) {
 int fm_draft(fm_ctx* c, int32_t* cand, float* draft_logits, float* draft_margin) {
   if (c == nullptr) return FM_ERR_INVALID_ARG;
   if (c->phase < 1) return FM_ERR_BAD_STATE;
-  draft(c, draft_logits, draft_margin, nullptr);
-  const int n = c->batch * c->dm.R1;
-  if (cand != nullptr) LAUNCH(c, copy_i32_kernel, (n + 127) / 128, 128, 0, c->st.cand, cand, n);
+  run_cached(c, c->cg_draft, cand, draft_logits, draft_margin, nullptr, [&] {
+    draft(c, draft_logits, draft_margin, nullptr);
+    const int n = c->batch * c->dm.R1;
+    if (cand != nullptr) LAUNCH(c, copy_i32_kernel, (n + 127) / 128, 128, 0, c->st.cand, cand, n);
+  });
   CUDA_OK(cudaGetLastError());
   if (c->launch_error != FM_OK) return c->launch_error;
   return FM_OK;
@@ -1074,11 +1149,13 @@ int fm_correct(fm_ctx* c, int32_t* cand, const int32_t* labels) {
 int fm_verify(fm_ctx* c, const int32_t* cand, int32_t* argmax, float* logits, float* margin) {
   if (c == nullptr || cand == nullptr) return FM_ERR_INVALID_ARG;
   if (c->phase < 1) return FM_ERR_BAD_STATE;
-  const int n = c->batch * c->dm.R1;
-  LAUNCH(c, verify_load_kernel, (n + 127) / 128, 128, 0, c->dm, c->st, c->batch, cand);
-  forward(c, logits);
-  if (argmax != nullptr) LAUNCH(c, copy_i32_kernel, (n + 127) / 128, 128, 0, c->st.o, argmax, n);
-  if (margin != nullptr) LAUNCH(c, copy_f32_kernel, (n + 127) / 128, 128, 0, c->st.margin, margin, n);
+  run_cached(c, c->cg_verify, cand, argmax, logits, margin, [&] {
+    const int n = c->batch * c->dm.R1;
+    LAUNCH(c, verify_load_kernel, (n + 127) / 128, 128, 0, c->dm, c->st, c->batch, cand);
+    forward(c, logits);
+    if (argmax != nullptr) LAUNCH(c, copy_i32_kernel, (n + 127) / 128, 128, 0, c->st.o, argmax, n);
+    if (margin != nullptr) LAUNCH(c, copy_f32_kernel, (n + 127) / 128, 128, 0, c->st.margin, margin, n);
+  });
   CUDA_OK(cudaGetLastError());
   if (c->launch_error != FM_OK) return c->launch_error;
   c->phase = 2;
@@ -1118,7 +1195,10 @@ int fm_verify_static_scratch(fm_ctx* c, const int32_t* cand, int32_t* argmax, fl
   int* saved_ticket = c->attn_ticket;
   c->attn_part = reinterpret_cast<float*>(base);
   c->attn_ticket = reinterpret_cast<int*>(base + ticket_off);
+  const bool was_off = c->call_graphs_off;
+  c->call_graphs_off = true;                       // the scratch pointers differ from the cached graph's
   const int rc = fm_verify(c, cand, argmax, logits, margin);
+  c->call_graphs_off = was_off;
   c->attn_part = saved_part;
   c->attn_ticket = saved_ticket;
   return rc;

@@ -130,6 +130,38 @@ def test_generate_speculative_equals_plain_on_device():
     assert (teach == plain).all() and st2.steps == 288 // 4 and st2.accept_hist[4] == 72
 
 
+def test_stepwise_calls_replayed_as_graphs_give_the_same_results(monkeypatch):
+    """fm_draft / fm_verify with the same pointer arguments every pass are captured and replayed as
+    CUDA graphs from the second call on; results must be those of the plain launches, bit for bit."""
+    import torch
+    cfg = S.get_config("tiny")
+    w, conds, prompts = _setup(cfg)
+
+    def run(dev, reuse):
+        dev.prefill(np.stack(conds), prompts)
+        out = []
+        for step in range(10):
+            cand, dl, _ = dev.draft(want_logits=True, reuse=reuse)
+            o, lg, mg = dev.verify(cand, want_logits=True, reuse=reuse)
+            out.append((cand.clone(), dl.clone(), o.clone(), lg.clone(), mg.clone()))
+            dev.accept(force_len=np.array([1 + step % (cfg.draft_len + 1)], dtype=np.int32), reuse=reuse)
+        return out
+
+    dev_g = _dev(cfg, w)
+    l0 = dev_g.launch_count()
+    got = run(dev_g, True)
+    n_graph = dev_g.launch_count() - l0
+    monkeypatch.setenv("FM_NO_CALL_GRAPH", "1")
+    dev_p = _dev(cfg, w)
+    l0 = dev_p.launch_count()
+    want = run(dev_p, False)
+    assert dev_p.launch_count() - l0 == n_graph          # a replayed pass counts the launches it holds
+    for a, b in zip(got, want):
+        for x, y in zip(a, b):
+            assert torch.equal(x, y)
+    assert dev_g.device_status() == 0
+
+
 def test_error_codes():
     from paper_2511_15618_b200 import FmError
     cfg = S.toy_config(d_model=128, head_dim=64, d_ff=256, weight_std=0.1, )
