@@ -189,13 +189,25 @@ __device__ inline void store_hi_lo(bf16* p, float v, int lo_off) {
   if (lo_off > 0) p[lo_off] = __float2bfloat16(v - __bfloat162float(hi));
 }
 
+// two neighbouring values as [hi, hi] and [lo, lo] pairs: one 4-byte store each
+__device__ inline void store_hi_lo2(bf16* p, float a, float b, int lo_off) {
+  const __nv_bfloat162 hi = __floats2bfloat162_rn(a, b);
+  *reinterpret_cast<__nv_bfloat162*>(p) = hi;
+  if (lo_off > 0)
+    *reinterpret_cast<__nv_bfloat162*>(p + lo_off) = __floats2bfloat162_rn(a - __bfloat162float(hi.x), b - __bfloat162float(hi.y));
+}
+
 __device__ inline float gelu_erf_f(float x) { return 0.5f * x * (1.f + erff(x * 0.70710678118654752f)); }
 
 // Pair slot q (0..63) of a 128-column tile -> its two columns.  Rotary pairs are (i, i + dh/2)
 // inside a head, so with heads of 64 a tile holds two heads with 32 pairs each, with heads of
 // 128 one head with 64 pairs.  The other epilogues use the same map (any bijection would do).
+// Epilogues without rotation pair neighbouring columns (2q, 2q + 1), so that a thread's two values
+// leave in one store.
+template <bool ROT>
 __device__ inline void pair_cols(int q, bool head128, int& ca, int& cb) {
-  if (head128) { ca = q; cb = q + 64; }
+  if (!ROT) { ca = 2 * q; cb = ca + 1; }
+  else if (head128) { ca = q; cb = q + 64; }
   else { ca = (q >> 5) * 64 + (q & 31); cb = ca + 32; }
 }
 
@@ -390,8 +402,8 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   uint32_t dst0 = 0, dbar = 0;
   float* recv_own;                                         // S == 1: this thread's row run in the local buffer
   {
-    const int q = head128 ? (tid & 63) : ((tid >> 6) * 32 + (tid & 31));
-    const int h = head128 ? (tid >> 6) : ((tid >> 5) & 1);
+    const int q = MODE != EPI_QKV ? (tid >> 1) : (head128 ? (tid & 63) : ((tid >> 6) * 32 + (tid & 31)));
+    const int h = MODE != EPI_QKV ? (tid & 1) : (head128 ? (tid >> 6) : ((tid >> 5) & 1));
     const int owner = q >> lgPW, cc = q & (PW - 1);
     recv_own = recv + (((size_t)z * PW + cc) * 2 + h) * NP;
     if (S > 1) {
@@ -405,7 +417,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   float2 pre_cs = make_float2(1.f, 0.f);                   // first item's rotary angle when the side rows are not used
   if (tid < items) {
     int ca, cb;
-    pair_cols(z * PW + (tid & (PW - 1)), head128, ca, cb);
+    pair_cols<MODE == EPI_QKV>(z * PW + (tid & (PW - 1)), head128, ca, cb);
     const int ma = tile_m * BM + ca, mb = tile_m * BM + cb;
     if (MODE == EPI_RESID && e.gain != nullptr) {
       if (ma < g.M) pre_ga = e.gain[ma];
@@ -438,7 +450,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   float pre_xa = 0.f, pre_xb = 0.f;                        // first item's residual values, same case
   if (MODE == EPI_RESID && want_side && !use_side && tid < items) {
     int ca, cb;
-    pair_cols(z * PW + (tid & (PW - 1)), head128, ca, cb);
+    pair_cols<MODE == EPI_QKV>(z * PW + (tid & (PW - 1)), head128, ca, cb);
     const int ma = tile_m * BM + ca, mb = tile_m * BM + cb;
     const float* xr = k_x + (size_t)(k_row0 + (tid >> lgPW)) * k_ldx;
     if (ma < k_M) pre_xa = xr[ma];
@@ -497,7 +509,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
     const bool active = it < items, first = it0 == 0;
     const int n = active ? it >> lgPW : 0, cc = active ? it & (PW - 1) : 0;
     int ca, cb;
-    pair_cols(z * PW + cc, head128, ca, cb);
+    pair_cols<MODE == EPI_QKV>(z * PW + cc, head128, ca, cb);
     float va[MAX_SPLIT], vb[MAX_SPLIT];
 #pragma unroll
     for (int r = 0; r < MAX_SPLIT; ++r) {                  // all loads first, then the sums in rank order
@@ -517,28 +529,35 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
     const size_t row = (size_t)(k_row0 + n);
     if (MODE == EPI_F32) {
       float* o = reinterpret_cast<float*>(k_out) + row * k_ldo;
-      if (a_ok) o[ma] = ya;
-      if (b_ok) o[mb] = yb;
+      if (b_ok && (k_ldo & 1) == 0) *reinterpret_cast<float2*>(o + ma) = make_float2(ya, yb);
+      else {
+        if (a_ok) o[ma] = ya;
+        if (b_ok) o[mb] = yb;
+      }
     } else if (MODE == EPI_BF16) {
       bf16* o = reinterpret_cast<bf16*>(k_out) + row * k_ldo;
-      if (a_ok) store_hi_lo(o + ma, ya, k_lo);
-      if (b_ok) store_hi_lo(o + mb, yb, k_lo);
+      if (b_ok) store_hi_lo2(o + ma, ya, yb, k_lo);
+      else if (a_ok) store_hi_lo(o + ma, ya, k_lo);
     } else if (MODE == EPI_GELU) {
       bf16* o = reinterpret_cast<bf16*>(k_out) + row * k_ldo;
-      if (a_ok) store_hi_lo(o + ma, gelu_erf_f(ya), k_lo);
-      if (b_ok) store_hi_lo(o + mb, gelu_erf_f(yb), k_lo);
+      if (b_ok) store_hi_lo2(o + ma, gelu_erf_f(ya), gelu_erf_f(yb), k_lo);
+      else if (a_ok) store_hi_lo(o + ma, gelu_erf_f(ya), k_lo);
     } else if (MODE == EPI_RESID) {
       float* xr = k_x + row * k_ldx;
       float xa = 0.f, xb = 0.f;
-      if (a_ok) {
+      if (b_ok) {                                          // both columns (M is even wherever the residual is used)
+        float2 x0 = make_float2(0.f, 0.f);
+        if (use_side) x0 = *reinterpret_cast<const float2*>(side + n * 128 + ca);
+        else if (first) x0 = make_float2(pre_xa, pre_xb);
+        else if (want_side) x0 = *reinterpret_cast<const float2*>(xr + ma);
+        xa = x0.x + ya;
+        xb = x0.y + yb;
+        *reinterpret_cast<float2*>(xr + ma) = make_float2(xa, xb);
+        if (k_aout != nullptr) store_hi_lo2(k_aout + row * k_lda + ma, xa * pre_ga, xb * pre_gb, k_lo);
+      } else if (a_ok) {
         xa = (use_side ? side[n * 128 + ca] : (first ? pre_xa : (want_side ? xr[ma] : 0.f))) + ya;
         xr[ma] = xa;
         if (k_aout != nullptr) store_hi_lo(k_aout + row * k_lda + ma, xa * pre_ga, k_lo);
-      }
-      if (b_ok) {
-        xb = (use_side ? side[n * 128 + cb] : (first ? pre_xb : (want_side ? xr[mb] : 0.f))) + yb;
-        xr[mb] = xb;
-        if (k_aout != nullptr) store_hi_lo(k_aout + row * k_lda + mb, xb * pre_gb, k_lo);
       }
       if (k_ssqo != nullptr) {
         // per-row sums of squares of this rank's columns: a fixed shuffle tree over the L lanes that
