@@ -374,15 +374,15 @@ __global__ void __launch_bounds__((NW + 1) * 32) attn_stream_kernel(const AttnAr
   const float4* src4 = reinterpret_cast<const float4*>(a.part + pt * a.max_groups * gstride);
   float4* dst4 = reinterpret_cast<float4*>(sm);
   const int n4 = n_groups * (int)(gstride / 4);
-  for (int i0 = 0; i0 < n4; i0 += CF::THREADS * 8) {
-    float4 v[8];
+  for (int i0 = 0; i0 < n4; i0 += CF::THREADS * 10) {    // 10 loads per thread: 9 groups of heads of 64 in one trip
+    float4 v[10];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
+    for (int k = 0; k < 10; ++k) {
       const int i = i0 + k * CF::THREADS + threadIdx.x;
       if (i < n4) v[k] = __ldcg(src4 + i);
     }
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
+    for (int k = 0; k < 10; ++k) {
       const int i = i0 + k * CF::THREADS + threadIdx.x;
       if (i < n4) dst4[i] = v[k];
     }
