@@ -391,19 +391,19 @@ __global__ void __launch_bounds__((NW + 1) * 32) attn_stream_kernel(const AttnAr
   const float* base = reinterpret_cast<const float*>(sm);
   // per row: common maximum, each group's weight (in group order) and the normaliser
   float* wgt = reinterpret_cast<float*>(sm) + (size_t)n_groups * gstride;      // [16][n_groups + 1]
-  if ((int)threadIdx.x < rows_here) {
-    const int i = threadIdx.x;
+  // (one warp per row, one lane per group: there are at most 24 groups; the normaliser is summed
+  // by shuffles in group order)
+  for (int i = warp; i < rows_here; i += NW + 1) {
     const float* pr = base + (size_t)i * (DH + 2);
-    float mm = -INFINITY;
-    for (int ck = 0; ck < n_groups; ++ck) mm = fmaxf(mm, pr[ck * gstride + DH]);
+    const float mc = lane < n_groups ? pr[lane * gstride + DH] : -INFINITY;
+    const float lc = lane < n_groups ? pr[lane * gstride + DH + 1] : 0.f;
+    const float mm = warp_max(mc);
+    const float sc = mc == -INFINITY ? 0.f : exp2f(mc - mm);
+    if (lane < n_groups) wgt[i * (n_groups + 1) + lane] = sc;
     float lsum = 0.f;
-    for (int ck = 0; ck < n_groups; ++ck) {
-      const float mc = pr[ck * gstride + DH];
-      const float sc = mc == -INFINITY ? 0.f : exp2f(mc - mm);
-      wgt[i * (n_groups + 1) + ck] = sc;
-      lsum += sc * pr[ck * gstride + DH + 1];
-    }
-    wgt[i * (n_groups + 1) + n_groups] = lsum;
+    for (int ck = 0; ck < n_groups; ++ck)
+      lsum = fmaf(__shfl_sync(0xffffffffu, sc, ck), __shfl_sync(0xffffffffu, lc, ck), lsum);
+    if (lane == 0) wgt[i * (n_groups + 1) + n_groups] = lsum;
   }
   __syncthreads();
   for (int e = threadIdx.x; e < rows_here * DH; e += CF::THREADS) {
