@@ -406,16 +406,25 @@ __global__ void __launch_bounds__((NW + 1) * 32) attn_stream_kernel(const AttnAr
     if (lane == 0) wgt[i * (n_groups + 1) + n_groups] = lsum;
   }
   __syncthreads();
-  for (int e = threadIdx.x; e < rows_here * DH; e += CF::THREADS) {
-    const int i = e / DH, c = e - i * DH;
+  for (int e = threadIdx.x; e < rows_here * (DH / 2); e += CF::THREADS) {     // two neighbouring columns per thread
+    const int i = e / (DH / 2), c = 2 * (e - i * (DH / 2));
     const float* pr = base + (size_t)i * (DH + 2) + c;
     const float* wr = wgt + i * (n_groups + 1);
-    float acc = 0.f;
+    float acc0 = 0.f, acc1 = 0.f;
 #pragma unroll 4
-    for (int ck = 0; ck < n_groups; ++ck) acc += wr[ck] * pr[ck * gstride];   // group order
+    for (int ck = 0; ck < n_groups; ++ck) {                                     // group order
+      const float2 v = *reinterpret_cast<const float2*>(pr + ck * gstride);
+      acc0 += wr[ck] * v.x;
+      acc1 += wr[ck] * v.y;
+    }
     const int idx = mt * 16 + i;
     const int r = group == 1 ? idx : idx / group, gh = idx - r * group;
-    attn::store_out(a.out, ((size_t)(b * m_rows + r) * 2 * dm.H + hk * group + gh) * DH + c, acc / wr[n_groups], dm.H * DH);
+    const size_t at = ((size_t)(b * m_rows + r) * 2 * dm.H + hk * group + gh) * DH + c;
+    const float o0 = acc0 / wr[n_groups], o1 = acc1 / wr[n_groups];
+    const __nv_bfloat162 hi = __floats2bfloat162_rn(o0, o1);
+    *reinterpret_cast<__nv_bfloat162*>(a.out + at) = hi;
+    *reinterpret_cast<__nv_bfloat162*>(a.out + at + dm.H * DH) =
+        __floats2bfloat162_rn(o0 - __bfloat162float(hi.x), o1 - __bfloat162float(hi.y));
   }
   if (threadIdx.x == 0) a.ticket[pt] = 0;
 }
