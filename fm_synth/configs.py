@@ -58,8 +58,10 @@ class ModelConfig:
         return self.n_bins + 2
 
     @property
-    def n_face_heads(self) -> int:      # Ef = ceil(D / 9)
-        return max(1, -(-self.draft_len // 9))
+    def n_face_heads(self) -> int:
+        # face head e drafts the face e - 1 after the one that holds the pending token; a draft
+        # can reach face (8 + D) // 9 after it, and only offsets >= 7 ever leave the next two points
+        return 1 if self.draft_len < 7 else (self.draft_len + 8) // 9 + 1
 
     def with_(self, **kw) -> "ModelConfig":
         return replace(self, **kw)

@@ -9,7 +9,8 @@ Draw order (numpy `default_rng(seed)`, `standard_normal(float32) * weight_std`):
   for each stack in (coord_down, vertex_down, face, vertex_up, coord_up),
     for each layer: g1[d], Wqkv[(H+2Hkv)*dh, d], Wo[d, H*dh], g2[d], W1[d_ff,d], W2[d,d_ff];
   S_cv[d,3d], S_vf[d,3d], U_fv[3d,d], U_vc[3d,d]; g_out[d], W_out[V,d];
-  draft heads: (gain[d], A[d,d]) for coordinate heads 1,2; vertex heads 1,2; face heads 1..Ef.
+  draft heads: (gain[d], A[d,d]) for coordinate heads 1,2; vertex heads 1,2; face heads 1..Ef
+  (Ef = ModelConfig.n_face_heads).
 Gains are exactly 1 when `gain_std == 0` (nothing is drawn for them then), else
 1 + gain_std * N(0,1) in float32 (gains are not rounded to bfloat16).
 """

@@ -15,7 +15,7 @@ What it follows (FlashMesh, arXiv 2511.15618, Sec. 3.2 "Correction Mechanism"):
 The label head itself (a linear layer on point features) needs trained weights to mean anything:
 labels are inputs here.
 
-Readings taken where the section is silent (each is listed in the design notes):
+Readings taken where the section is silent:
   R1  a "point" of a candidate row is a vertex whose three coordinate tokens (z, y, x) are all
       drafts of this pass; vertices that contain the main token or already accepted tokens, or
       that are cut off by the end of the row, are left alone.  A vertex with a token that is not a

@@ -15,7 +15,7 @@ What it follows (FlashMesh, arXiv 2511.15618):
     drafts up to the first mismatch, continue from the backbone's output there.
   * Supp. "Optimizations", rules (A) and (B): one draft source per future position.
 
-Readings taken where the paper is silent (each is listed in the design notes): pre-norm
+Readings taken where the paper is silent: pre-norm
 RMSNorm, GELU(erf) FFN without biases, rotate-half RoPE on the level-local index,
 conditioning folded in as per-layer prefix keys/values visible to every query,
 right-aligned linear shortening of 3 concatenated hiddens, linear upsampling added to the
@@ -97,17 +97,36 @@ def masked_top2(cfg, logits, target_index):
 def draft_source(n, j, draft_len):
     """Which head predicts draft offset j (target t_{n+j}) when the pending main token is t_n.
 
-    Rule (B): offsets 1 and 2 come from the coordinate heads.  Later offsets inside the
-    current face come from the vertex (point) heads; offsets in a later face come from the
-    face heads (rule (A): the higher level wins).  Returns (level, head, slot):
-    level 0 -> coordinate head `head` (1-based); level 1 -> vertex head `head`, slot r of its
-    3 upsampled features; level 2 -> face head `head`, slot r of its 9 features."""
+    Supp. "Optimizations".  The levels fire at their own rows: the point level where a vertex
+    starts (n % 3 == 0), the face level where a face starts (n % 9 == 0); rows in between
+    reuse the most recent predictions of those levels (Supp. "Integrating the three levels").
+    With v* = n // 3 and f* = n // 9 the most recent point-level row is 3 v*, the most recent
+    face-level row 9 f*.
+      * Rule (B): offsets 1 and 2 always come from the coordinate heads; the higher levels
+        drop the point that holds the main token.
+      * The point level then covers the next two whole points, vertices v*+1 and v*+2,
+        wherever the face boundary lies (worked step (1): predicting the first coordinate
+        of a face's last vertex, the point level gives the six tokens of the next face's
+        first two vertices; step (2): one token later those predictions are reused).
+      * Rule (A): where the most recent point-level row was also a face-level row
+        (v* % 3 == 0) the point-level predictions were removed, and the face level covers
+        the rest of the face it started: face head 1 predicts the face that holds t_n.
+      * Targets beyond vertex v*+2 (the paper's 9-9 model stops there and drafts 8, 7 or 6
+        tokens depending on the row; a fixed draft length needs a source for them) come from
+        the face level: face head e predicts face f* + e - 1.
+    Every offset has exactly one source (no averaging).  Returns (level, head, slot):
+    level 0 -> coordinate head `head` (1-based); level 1 -> vertex head `head` (vertex
+    v* + head), slot r of its 3 upsampled features; level 2 -> face head `head` (face
+    f* + head - 1), slot r of its 9 features."""
     p = n + j
     if j <= 2:
         return (0, j, 0)
-    if p // 9 == n // 9:
-        return (1, p // 3 - n // 3, p % 3)
-    return (2, p // 9 - n // 9, p % 9)
+    ev = p // 3 - n // 3
+    if ev <= 2:
+        if (n // 3) % 3 == 0 and p // 9 == n // 9:
+            return (2, 1, p % 9)
+        return (1, ev, p % 3)
+    return (2, p // 9 - n // 9 + 1, p % 9)
 
 
 # ---------------------------------------------------------------------------------------------
@@ -348,8 +367,11 @@ class OracleSeq:
         return rms_norm(hc2, w["g_out"], cfg.norm_eps) @ w["W_out"].T
 
     # -- the six operations -------------------------------------------------------------------
-    def prefill(self, cond, prompt, max_faces=None):
-        """Consume BOS + prompt; afterwards L = 1 + len(prompt) and the first main token is pending."""
+    def prefill(self, cond, prompt, max_faces=None, chunk=None):
+        """Consume BOS + prompt; afterwards L = 1 + len(prompt) and the first main token is pending.
+        `chunk` feeds the inputs that many rows at a time (same result as one dense pass: the
+        cached rows of a later chunk see the earlier ones through the caches); long prompts
+        need it to keep the score matrices small.  Returns the logits of the last chunk."""
         cfg = self.cfg
         self._alloc(cond)
         self.L = 0
@@ -358,8 +380,10 @@ class OracleSeq:
         if max_faces is not None:
             self.t_end = self.prompt_len + 9 * max_faces
         u = [cfg.bos] + [int(t) for t in prompt]
-        logits = self.forward_rows(u)
-        self.L = len(u)
+        step = len(u) if not chunk else int(chunk)
+        for i in range(0, len(u), step):
+            logits = self.forward_rows(u[i:i + step])
+            self.L = min(len(u), i + step)
         self.main, self.main_margin = masked_top2(cfg, logits[-1], self.L - 1)
         if self.L - 1 >= self.t_end:
             self.done = True
@@ -390,7 +414,7 @@ class OracleSeq:
             tri = w["U_vc"] @ head(zv, w["heads_v"][e - 1])           # Eq. 2: one vertex -> 3 coordinates
             for r in range(3):
                 feats[(1, e, r)] = tri[r * d:(r + 1) * d]
-        for e in range(1, cfg.n_face_heads + 1):
+        for e in range(1, cfg.n_face_heads + 1):                       # head e drafts face f* + e - 1
             tri = w["U_fv"] @ head(zf, w["heads_f"][e - 1])           # one face -> 3 vertices
             for rv in range(3):
                 sub = w["U_vc"] @ tri[rv * d:(rv + 1) * d]             # each vertex -> 3 coordinates

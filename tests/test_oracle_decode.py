@@ -61,7 +61,7 @@ def test_speculative_equals_plain_equals_bruteforce(D):
     assert all(a == D + 1 for a in acc[:-1]) and 1 <= acc[-1] <= D + 1  # all drafts right: a = D+1
     assert len(acc) == -(-len(brute) // (D + 1))
     rnd, acc = run(_teacher(truth, upto=0, corrupt_rng=np.random.default_rng(D)))
-    assert rnd == brute and len(set(acc)) > 1 or D == 1
+    assert rnd == brute and (len(set(acc)) > 1 or D == 1)
 
 
 def test_accept_length_is_exactly_the_number_of_leading_matches():
@@ -141,26 +141,46 @@ def test_eos_inside_accepted_drafts_clips_the_accept():
 
 # ------------------------------------------------------------------ draft source assignment
 def test_draft_sources_match_the_papers_worked_example():
+    """Supp. "Optimizations": the row rule (A) names and the two worked steps, at the phases of
+    the face the paper's indices put them at (a face row, then 6 and 7 tokens into the face)."""
     rows = [tuple(int(x) for x in ln.split()) for ln in open(os.path.join(GOLDEN, "draft_coverage_9_9.txt"))
             if ln.strip() and not ln.startswith("#")]
-    assert len(rows) == 15
+    assert len(rows) == 23 and {r[0] for r in rows} == {0, 6, 7}
     for n, j, level in rows:
-        assert O.draft_source(n, j, 9)[0] == level
+        for faces_before in (0, 1, 5):                # the assignment depends on the phase only
+            assert O.draft_source(n + 9 * faces_before, j, 9)[0] == level
 
 
-@pytest.mark.parametrize("D", [3, 9, 12])
+def test_draft_sources_at_every_phase_of_the_face():
+    """All nine phases, offsets 1..9, against the table worked out by hand from the rules."""
+    table = {}
+    for ln in open(os.path.join(GOLDEN, "draft_sources_all_phases_D9.txt")):
+        if ln.strip() and not ln.startswith("#"):
+            f = ln.split()
+            table[int(f[0])] = f[1:]
+    assert sorted(table) == list(range(9)) and all(len(v) == 9 for v in table.values())
+    name = {0: "c", 1: "v", 2: "f"}
+    for n in range(0, 45):
+        for j in range(1, 10):
+            level, head, _ = O.draft_source(n, j, 9)
+            assert name[level] + (str(head) if level else "") == table[n % 9][j - 1], (n, j)
+
+
+@pytest.mark.parametrize("D", [3, 9, 12, 24, 27])
 def test_every_offset_has_one_valid_source(D):
-    Ef = max(1, -(-D // 9))
+    cfg = S.toy_config(draft_len=D)
     for n in range(0, 40):
         for j in range(1, D + 1):
             level, head, slot = O.draft_source(n, j, D)
             p = n + j
             if level == 0:
                 assert j in (1, 2) and head == j
-            elif level == 1:
-                assert 1 <= head <= 2 and 3 * (n // 3 + head) + slot == p and p // 9 == n // 9
-            else:
-                assert 1 <= head <= Ef and 9 * (n // 9 + head) + slot == p
+            elif level == 1:                          # the vertex `head` after the one that holds t_n
+                assert 1 <= head <= 2 and 3 * (n // 3 + head) + slot == p
+                assert (n // 3) % 3 != 0 or p // 9 != n // 9      # never where rule (A) keeps the face level
+            else:                                     # face head e drafts face f* + e - 1
+                assert 1 <= head <= cfg.n_face_heads and 9 * (n // 9 + head - 1) + slot == p
+                assert head > 1 or (n // 3) % 3 == 0
 
 
 def test_draft_features_follow_the_head_formula_in_special_cases():
@@ -170,19 +190,33 @@ def test_draft_features_follow_the_head_formula_in_special_cases():
     for hs in (w["heads_c"], w["heads_v"], w["heads_f"]):
         for h in hs:
             h["A"][:] = 0.0
-    seq = O.OracleSeq(cfg, w)
-    seq.prefill(cond, _prompt(cfg, 1), max_faces=4)       # n = 9: phase 0
-    _, dl, _ = seq.draft()
-    n, d = seq.L - 1, cfg.d_model
     W, g = w["W_out"].astype(np.float64), w["g_out"].astype(np.float64)
     out = lambda f: W @ (f / np.sqrt(np.mean(f * f) + cfg.norm_eps) * g)
+    d = cfg.d_model
+    U_vc, U_fv = w["U_vc"].astype(np.float64), w["U_fv"].astype(np.float64)
+    seq = O.OracleSeq(cfg, w)
+    seq.prefill(cond, _prompt(cfg, 1), max_faces=4)       # n = 9: a face row
+    _, dl, _ = seq.draft()
+    n = seq.L - 1
+    assert n == 9
     assert np.allclose(dl[0], out(seq.zc[n])) and np.allclose(dl[1], out(seq.zc[n]))
-    tri = w["U_vc"].astype(np.float64) @ seq.zv[n // 3]
+    ftri = U_fv @ seq.zf[n // 9]                           # every face head sees the same z_f
+    for j in range(3, 9):                                  # rule (A): the face level, slots 3..8 of this face
+        sub = U_vc @ ftri[(j // 3) * d:(j // 3 + 1) * d]
+        assert np.allclose(dl[j - 1], out(sub[(j % 3) * d:(j % 3 + 1) * d]))
+    assert np.allclose(dl[8], out((U_vc @ ftri[:d])[:d]))  # offset 9: next face, slot 0
+    # three tokens on (force the accept): a point-level row inside the face
+    cand, _, _ = seq.draft()
+    seq.verify(cand)
+    seq.accept(force_len=3)
+    _, dl, _ = seq.draft()
+    n = seq.L - 1
+    assert n == 12
+    tri = U_vc @ seq.zv[n // 3]
     for j in range(3, 9):                                  # both vertex heads see the same z_v
         assert np.allclose(dl[j - 1], out(tri[(j % 3) * d:(j % 3 + 1) * d]))
-    ftri = w["U_fv"].astype(np.float64) @ seq.zf[n // 9]
-    sub = w["U_vc"].astype(np.float64) @ ftri[:d]
-    assert np.allclose(dl[8], out(sub[:d]))                # offset 9 -> next face, slot 0
+    ftri = U_fv @ seq.zf[n // 9]
+    assert np.allclose(dl[8], out((U_vc @ ftri[d:2 * d])[:d]))     # offset 9 -> t_21: next face, slot 3
 
 
 def test_head_residual_and_linear_term():

@@ -218,6 +218,19 @@ def test_cached_rows_equal_dense_forward_and_single_steps(window):
     assert np.abs(np.concatenate(rows) - full).max() < 1e-9
 
 
+@pytest.mark.parametrize("chunk", [1, 7, 16])
+def test_chunked_prefill_equals_the_dense_forward(chunk):
+    cfg, w, cond = _setup(layers=(1, 2, 2, 1, 2), window=(11, 5, 2))
+    u = _tokens(cfg, 37)
+    full = O.forward_full(cfg, w, cond, u)
+    seq = O.OracleSeq(cfg, w)
+    last = seq.prefill(cond, u[1:], chunk=chunk)
+    assert seq.L == 37 and np.abs(last - full[-last.shape[0]:]).max() < 1e-9
+    nxt = seq.forward_rows([u[5]])                    # the state after a chunked prefill decodes on correctly
+    assert np.abs(nxt[0] - O.forward_full(cfg, w, cond, u + [u[5]])[-1]).max() < 1e-9
+    assert seq.main == O.masked_top2(cfg, full[-1], 36)[0]
+
+
 def test_rejected_rows_leave_no_trace():
     cfg, w, cond = _setup(draft_len=9)
     u = _tokens(cfg, 30)
