@@ -38,11 +38,7 @@ def _peaks():
 
 
 def _fill_prompt(cfg, seq, n_faces):
-    """Seeded mesh tokens standing in for an already generated prefix: the sorted faces of a
-    twice-subdivided icosphere, repeated until n_faces faces."""
-    base = S.make_prompt(cfg.with_(prompt_faces=(320, 320), prompt_subdiv=2), seq)
-    reps = -(-n_faces * 9 // len(base))
-    return [int(t) for t in np.tile(base, reps)[:9 * n_faces]]
+    return S.fill_prompt(cfg, seq, n_faces)
 
 
 def reduce_over_ranks(maxed, summed, device):

@@ -9,8 +9,8 @@ sharing any code of the method itself.
 from .configs import CONFIGS, ModelConfig, get_config, toy_config
 from .weights import make_weights, round_to_bf16, stack_names
 from .inputs import (make_condition, make_prompt, icosphere_faces,
-                     accept_schedule, stop_lengths)
+                     accept_schedule, stop_lengths, fill_prompt)
 
 __all__ = ["CONFIGS", "ModelConfig", "get_config", "toy_config", "make_weights",
            "round_to_bf16", "stack_names", "make_condition", "make_prompt",
-           "icosphere_faces", "accept_schedule", "stop_lengths"]
+           "icosphere_faces", "accept_schedule", "stop_lengths", "fill_prompt"]

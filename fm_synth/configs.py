@@ -39,6 +39,7 @@ class ModelConfig:
     cond_kind: str = "gauss"            # gauss | sphere | solids
     cond_points: int = 0
     weight_std: float = 0.02
+    out_std: float = 0.0                # std of the output matrix W_out; 0 => weight_std
     gain_std: float = 0.0               # 0 => RMSNorm gains exactly 1
 
     @property

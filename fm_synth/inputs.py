@@ -134,6 +134,14 @@ def make_prompt(cfg: ModelConfig, seq: int = 0) -> np.ndarray:
     return np.array(out[:n_faces], dtype=np.int32).reshape(-1)
 
 
+def fill_prompt(cfg: ModelConfig, seq: int, n_faces: int) -> list:
+    """Seeded mesh tokens standing in for an already generated prefix of `n_faces` faces: the
+    sorted faces of a twice-subdivided icosphere, repeated as often as needed."""
+    base = make_prompt(cfg.with_(prompt_faces=(320, 320), prompt_subdiv=2), seq)
+    reps = -(-n_faces * 9 // len(base))
+    return [int(t) for t in np.tile(base, reps)[:9 * n_faces]]
+
+
 # ----------------------------------------------------------------------------------------
 # acceptance schedules and stop lengths (stand-ins for trained draft heads / real meshes)
 # ----------------------------------------------------------------------------------------

@@ -11,6 +11,8 @@ Draw order (numpy `default_rng(seed)`, `standard_normal(float32) * weight_std`):
   S_cv[d,3d], S_vf[d,3d], U_fv[3d,d], U_vc[3d,d]; g_out[d], W_out[V,d];
   draft heads: (gain[d], A[d,d]) for coordinate heads 1,2; vertex heads 1,2; face heads 1..Ef
   (Ef = ModelConfig.n_face_heads).
+`W_out` alone is scaled by `out_std` when that is set (toy models keep sharp attention with
+std-0.1 matrices but logits on the scale of the workloads').
 Gains are exactly 1 when `gain_std == 0` (nothing is drawn for them then), else
 1 + gain_std * N(0,1) in float32 (gains are not rounded to bfloat16).
 """
@@ -36,9 +38,9 @@ def make_weights(cfg: ModelConfig, seed: int | None = None) -> dict:
     rng = np.random.default_rng(cfg.seed if seed is None else seed)
     d, H, Hkv, dh, dff, V = cfg.d_model, cfg.n_heads, cfg.n_kv_heads, cfg.head_dim, cfg.d_ff, cfg.vocab
 
-    def mat(o, i):
+    def mat(o, i, std=None):
         w = rng.standard_normal((o, i), dtype=np.float32)
-        w *= np.float32(cfg.weight_std)
+        w *= np.float32(cfg.weight_std if std is None else std)
         return round_to_bf16(w)
 
     def gain():
@@ -64,7 +66,7 @@ def make_weights(cfg: ModelConfig, seed: int | None = None) -> dict:
     w["U_fv"] = mat(3 * d, d)
     w["U_vc"] = mat(3 * d, d)
     w["g_out"] = gain()
-    w["W_out"] = mat(V, d)
+    w["W_out"] = mat(V, d, cfg.out_std if cfg.out_std > 0 else None)
     w["heads_c"] = [{"g": gain(), "A": mat(d, d)} for _ in range(2)]
     w["heads_v"] = [{"g": gain(), "A": mat(d, d)} for _ in range(2)]
     w["heads_f"] = [{"g": gain(), "A": mat(d, d)} for _ in range(cfg.n_face_heads)]

@@ -12,6 +12,14 @@
  * coordinates form a vertex, three vertices a face; shortening and upsampling layers with
  * residuals between levels) with a KV cache at each level.
  *
+ * Where the paper is silent the model is read as follows: pre-norm RMSNorm blocks, FFN =
+ * W2 gelu_erf(W1 x) without biases, rotate-half rotary embedding on the level-local index,
+ * conditioning as per-layer prefix keys/values (every layer projects rms(c) with its own K/V
+ * matrices; un-rotated, visible to every query, sharing the softmax with the causal keys),
+ * shortening = linear on the concatenation of hiddens 3v-2, 3v-1, 3v (zeros below 0), upsampling
+ * = linear d -> 3d whose slot r is added to the pre-shorten hidden of position 3v+r,
+ * longest-matching-prefix acceptance, masked argmax with ties to the lowest id.
+ *
  * Conventions
  *   - Every call returns FM_OK (0) or a negative FM_ERR_* code; nothing throws.  On an error
  *     return no decoding state has been changed, except after FM_ERR_CUDA or FM_ERR_TIMEOUT:
@@ -55,12 +63,11 @@ extern "C" {
 #define FM_ERR_UNSUPPORTED  -6   /* shape outside what the kernels were built for              */
 
 #define FM_MAX_FACE_HEADS 4
-#define FM_MAX_DRAFT      24
+#define FM_MAX_DRAFT      27
 
 typedef struct fm_ctx fm_ctx;    /* opaque; owns nothing but pinned host flags */
 
-/* Model and capacity description (the hourglass of the supplement; every reading the paper
- * leaves open is fixed in the oracle's header and repeated here where it shapes a field). */
+/* Model and capacity description (the hourglass of the supplement, read as stated above). */
 typedef struct fm_config {
   int32_t d_model, n_heads, n_kv_heads, head_dim, d_ff;
   int32_t layers[5];          /* coord_down, vertex_down, face, vertex_up, coord_up          */
@@ -97,7 +104,9 @@ typedef struct fm_weights {
   const float* W_out;                     /* [V, d]                                           */
   const float* head_c_g[2];  const float* head_c_A[2];   /* coordinate draft heads, A [d,d]  */
   const float* head_v_g[2];  const float* head_v_A[2];   /* vertex (point) draft heads       */
-  const float* head_f_g[FM_MAX_FACE_HEADS]; const float* head_f_A[FM_MAX_FACE_HEADS]; /* ceil(D/9) used */
+  const float* head_f_g[FM_MAX_FACE_HEADS]; const float* head_f_A[FM_MAX_FACE_HEADS];
+                              /* face head e (1-based) drafts the face e-1 after the one that holds the
+                                 pending token; D < 7 uses 1 head, otherwise (D+8)/9 + 1 */
 } fm_weights;
 
 /* Optional device-side draft editor for fm_generate: the place where the paper's Correct
@@ -164,7 +173,7 @@ int fm_draft(fm_ctx* ctx, int32_t* cand /*DEV*/, float* draft_logits /*DEV*/, fl
  * ascending by (z, y, x) among the slots they occupy.  Only rows the next pass feeds
  * (the first nrow slots of an unfinished sequence) are considered.
  * cand: DEV int32 in/out [batch, D+1].  Errors: INVALID_ARG (null pointer), BAD_STATE (before
- * fm_prefill), UNSUPPORTED (more than 48 slots per row; cannot happen while FM_MAX_DRAFT is 24). */
+ * fm_prefill), UNSUPPORTED (more than 48 slots per row; cannot happen while FM_MAX_DRAFT is 27). */
 #define FM_LABEL_HISTORICAL 0
 #define FM_LABEL_NEW 1
 #define FM_LABEL_INTRA 2
@@ -193,8 +202,9 @@ int fm_verify(fm_ctx* ctx, const int32_t* cand /*DEV*/, int32_t* argmax /*DEV*/,
  *   - Limit: the scratch one pass needs (it grows with max_batch * n_kv_heads and with the cache
  *     capacity) must fit in FM_STATIC_SCRATCH_BYTES, else FM_ERR_CAPACITY is returned and nothing
  *     is enqueued.
- *   - The first call on a device looks up the array's device address (with the context's device
- *     current); make that first call before any stream capture is begun.
+ *   - Every GPU has its own copy of the array: the device the context was created on must be the
+ *     current device at every call (FM_ERR_BAD_STATE otherwise).  The first call on a device looks
+ *     up the array's device address; make that first call before any stream capture is begun.
  *   - All contexts and all calls share the one array.  It keeps the previous call's contents (the
  *     call clears the counters that must start at zero), and two calls whose kernels overlap on
  *     the GPU -- different streams, different contexts -- race on it: serialise them. */
@@ -249,13 +259,33 @@ int fm_profile_begin(fm_ctx* ctx);
 int fm_profile_class(fm_ctx* ctx, int32_t cls, int32_t reps, fm_profile* out /*HOST*/);
 int fm_profile_end(fm_ctx* ctx, fm_profile* out /*HOST*/);
 
+/* How the attention kernel cuts a level's cache (no counterpart in the paper; for reports and
+ * tests): slots per chunk, chunks per group (one CTA streams one group; fixed when the context is
+ * created) and the number of groups the full cache has.  A (sequence, kv-head) whose cache holds n
+ * slots, prefix included, is read by ceil(ceil(n / chunk) / chunks_per_group) CTAs, whose partial
+ * results go through the scratch buffers when there is more than one.  level: 0 coordinate,
+ * 1 vertex, 2 face.  HOST out pointers, any may be NULL. */
+int fm_attention_layout(const fm_ctx* ctx, int32_t level, int32_t* chunk_slots, int32_t* chunks_per_group,
+                        int32_t* max_groups);
+
 /* Number of kernels launched by this context since creation (for launch accounting). */
 int64_t fm_launch_count(const fm_ctx* ctx);
 
+/* Self-check of the give-up path of the device-side waits (no counterpart in the paper).  Every
+ * wait inside the kernels (on a shared-memory barrier that a copy, a tensor-core commit or a peer
+ * CTA completes) polls for a bounded number of clock cycles, then records FM_ERR_TIMEOUT in the
+ * device status word and lets the kernel finish without touching the data.  This call enqueues one
+ * thread that runs the same wait, limited to `limit_cycles` (1 .. 1e8), on a barrier that nothing
+ * completes: afterwards fm_device_status returns FM_ERR_TIMEOUT, and fm_prefill clears it.  The
+ * kernel always ends by itself. */
+int fm_selftest_wait_timeout(fm_ctx* ctx, int64_t limit_cycles);
+
 const char* fm_strerror(int code);
 /* Device status word: 0, or FM_ERR_TIMEOUT if a bounded wait inside a kernel gave up, or
- * FM_ERR_INVALID_ARG if a kernel met an out-of-range token id (it then used PAD).  Synchronises
- * the stream. */
+ * FM_ERR_INVALID_ARG if a kernel met an out-of-range token id (it then used PAD), or
+ * FM_ERR_CAPACITY if the attention kernel was asked to merge more cache groups than it can stage
+ * (it then wrote nothing; fm_create sizes the groups so that this does not happen).  The word is
+ * cleared by fm_prefill.  Synchronises the stream. */
 int fm_device_status(fm_ctx* ctx);
 
 #ifdef __cplusplus

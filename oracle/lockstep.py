@@ -19,15 +19,22 @@ def _np(x):
 
 
 def run_lockstep(cfg, w, conds, prompts, dev, max_faces, max_steps, *, tol=2e-2, margin=0.1, truth=None,
-                 keep_rng=None, check_drafts=True, dtype=np.float64):
+                 keep_rng=None, check_drafts=True, dtype=np.float64, prefill_chunk=None, seq_max_tokens=None):
     """Returns a report dict; raises AssertionError on a parity failure.
 
     truth: optional per-sequence known continuation (mesh tokens, prompt included) used to
-    overwrite drafts so that accept lengths vary (keep_rng draws how many are kept)."""
+    overwrite drafts so that accept lengths vary (keep_rng draws how many are kept).
+    prefill_chunk: the oracle consumes the prompts that many rows at a time (long prompts).
+    seq_max_tokens: per-sequence cache capacity of the oracle's sequences (default: cfg's)."""
     B, D, V = len(prompts), cfg.draft_len, cfg.vocab
-    seqs = [OracleSeq(cfg, w, dtype) for _ in range(B)]
+    seqs = []
     for b in range(B):
-        seqs[b].prefill(conds[b], prompts[b], max_faces=max_faces[b] if hasattr(max_faces, "__len__") else max_faces)
+        c = cfg if seq_max_tokens is None else cfg.with_(max_tokens=int(seq_max_tokens[b]))
+        # the first sequence converts the weights to `dtype`; the others share those arrays
+        seqs.append(OracleSeq(c, w if b == 0 else seqs[0].w, dtype))
+    for b in range(B):
+        seqs[b].prefill(conds[b], prompts[b], max_faces=max_faces[b] if hasattr(max_faces, "__len__") else max_faces,
+                        chunk=prefill_chunk)
     dev.prefill(np.stack(conds), prompts)
     dev.set_max_faces([max_faces[b] if hasattr(max_faces, "__len__") else max_faces for b in range(B)])
     rep = dict(steps=0, emitted=0, overrides=0, max_logit_err=0.0, max_draft_err=0.0, rows=0, low_margin_rows=0,

@@ -12,7 +12,7 @@ import os
 import numpy as np
 
 FM_MAX_FACE_HEADS = 4
-FM_MAX_DRAFT = 24
+FM_MAX_DRAFT = 27
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB = None
@@ -105,8 +105,12 @@ def load_library():
     lib.fm_profile_end.argtypes = [vp, C.POINTER(FmProfile)]
     lib.fm_profile_class.restype = C.c_int
     lib.fm_profile_class.argtypes = [vp, i32, i32, C.POINTER(FmProfile)]
+    lib.fm_attention_layout.restype = C.c_int
+    lib.fm_attention_layout.argtypes = [vp, i32, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     lib.fm_launch_count.restype = C.c_int64
     lib.fm_launch_count.argtypes = [vp]
+    lib.fm_selftest_wait_timeout.restype = C.c_int
+    lib.fm_selftest_wait_timeout.argtypes = [vp, C.c_int64]
     lib.fm_strerror.restype = C.c_char_p
     lib.fm_strerror.argtypes = [C.c_int]
     lib.fm_device_status.restype = C.c_int
@@ -196,8 +200,19 @@ def fm_profile_class(ctx, cls, reps):
     return rc, p
 
 
+def fm_attention_layout(ctx, level):
+    """(slots per chunk, chunks per group, groups of the full cache) of a level's attention."""
+    a, b, c = C.c_int32(), C.c_int32(), C.c_int32()
+    rc = load_library().fm_attention_layout(ctx, int(level), C.byref(a), C.byref(b), C.byref(c))
+    return rc, (a.value, b.value, c.value)
+
+
 def fm_launch_count(ctx):
     return int(load_library().fm_launch_count(ctx))
+
+
+def fm_selftest_wait_timeout(ctx, limit_cycles):
+    return int(load_library().fm_selftest_wait_timeout(ctx, int(limit_cycles)))
 
 
 def fm_device_status(ctx):
@@ -270,7 +285,7 @@ class FlashMesh:
             base = (self.workspace.data_ptr() + 255) // 256 * 256
             # a stream of its own: the legacy default stream cannot be captured into a CUDA graph
             self.stream = stream if stream is not None else torch.cuda.Stream(self.device)
-            fw, self._keep = make_weights(weights, (self.D + 8) // 9 if self.D else 0)
+            fw, self._keep = make_weights(weights, 0 if self.D == 0 else (1 if self.D < 7 else (self.D + 8) // 9 + 1))
             rc, self.ctx = fm_create(self.cfg, fw, base, nbytes, self.stream.cuda_stream)
         if rc != 0:
             raise FmError(rc, "fm_create")

@@ -10,6 +10,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
 #include <utility>
 #include <vector>
@@ -98,6 +99,8 @@ struct fm_ctx {
   int split_target;     // CTAs a GEMM launch aims for (M tiles x K splits)
   int stage_cap;        // tuning knob: upper bound on the GEMM ring depth (0 = none)
   int n_sm;                                  // SMs of the device
+  int device;                                // ordinal of the device the context was created on
+  size_t attn_ticket_n;                      // entries of attn_ticket
   int split_target_deep;                     // the same for launches whose CTAs stream long K ranges
   int launch_error;     // first error met while enqueueing (capacity, descriptor creation)
   // one decode pass (draft, teacher edit, verify, accept) captured as a CUDA graph
@@ -138,7 +141,7 @@ int check_config(const fm_config* c) {
   if (c->draft_len > FM_MAX_DRAFT) return FM_ERR_UNSUPPORTED;
   if (c->d_model % 64 != 0 || c->d_ff % 64 != 0 || (c->n_heads * c->head_dim) % 128 != 0) return FM_ERR_UNSUPPORTED;
   if (c->head_dim != 64 && c->head_dim != 128) return FM_ERR_UNSUPPORTED;
-  if ((c->draft_len + 8) / 9 > FM_MAX_FACE_HEADS) return FM_ERR_UNSUPPORTED;
+  if (c->draft_len >= 7 && (c->draft_len + 8) / 9 + 1 > FM_MAX_FACE_HEADS) return FM_ERR_UNSUPPORTED;
   if (c->max_tokens < c->draft_len + 2) return FM_ERR_INVALID_ARG;
   return FM_OK;
 }
@@ -158,7 +161,9 @@ Dims make_dims(const fm_config& c) {
   }
   dm.max_batch = c.max_batch; dm.max_tokens = c.max_tokens; dm.allow_eos = c.allow_eos;
   dm.eps = c.norm_eps; dm.theta = c.rope_theta;
-  dm.Ef = dm.D > 0 ? (dm.D + 8) / 9 : 1; dm.NH = 4 + dm.Ef;
+  // face head e drafts face f* + e - 1 (f* holds the pending token); offsets below 7 never leave
+  // the next two points, a draft of D tokens reaches face f* + (8 + D) / 9
+  dm.Ef = dm.D >= 7 ? (dm.D + 8) / 9 + 1 : 1; dm.NH = 4 + dm.Ef;
   return dm;
 }
 
@@ -266,6 +271,7 @@ void carve(fm_ctx* c, Carver& cv) {
   }
   c->attn_part = cv.take<float>(part_max);
   c->attn_ticket = cv.take<int>(ticket_max);
+  c->attn_ticket_n = ticket_max;
   int n_layers = 0;
   for (int s = 0; s < 5; ++s) n_layers += c->cfg.layers[s];
   c->tmaps_cap = (size_t)6 * n_layers + 128;
@@ -971,6 +977,7 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     c->n_sm = sms > 0 ? sms : 148;
+    c->device = dev;
     const char* tt = getenv("FM_SPLIT_TARGET_DEEP");
     c->split_target_deep = tt != nullptr && atoi(tt) > 0 ? atoi(tt) : 296;
     const char* sc = getenv("FM_STAGE_CAP");
@@ -1076,6 +1083,10 @@ int fm_prefill(fm_ctx* c, int32_t batch, const float* cond, const int32_t* promp
   if (prompt_off[batch] > 0 && prompt == nullptr) return FM_ERR_INVALID_ARG;
   c->batch = batch;
   c->launch_error = FM_OK;                         // a new start clears an earlier enqueue error
+  // ... and whatever a kernel that gave up on a bounded wait left behind: the status word, and
+  // the tickets of attention tiles whose last CTA never came to reset them
+  CUDA_OK(cudaMemsetAsync(c->st.status, 0, sizeof(int), c->stream));
+  CUDA_OK(cudaMemsetAsync(c->attn_ticket, 0, c->attn_ticket_n * sizeof(int), c->stream));
   c->plen_host.assign(batch, 0);
   for (int b = 0; b < batch; ++b) c->plen_host[b] = prompt_off[b + 1] - prompt_off[b];
   CUDA_OK(cudaMemcpyAsync(c->prompt_off_dev, prompt_off, (batch + 1) * sizeof(int), cudaMemcpyHostToDevice, c->stream));
@@ -1178,15 +1189,22 @@ int fm_verify_static_scratch(fm_ctx* c, const int32_t* cand, int32_t* argmax, fl
   const size_t ticket_off = align_up(part_floats * sizeof(float), 256);
   if (ticket_off + tickets * sizeof(int) > (size_t)FM_STATIC_SCRATCH_BYTES) return FM_ERR_CAPACITY;
   // Device address of the static array, looked up once per device with that device current (the
-  // array's name is only a host-side handle; a kernel must be given this address).
+  // array's name is only a host-side handle; a kernel must be given this address).  Every GPU
+  // holds its own copy of the array, so the address must be the one of the context's device:
+  // the call is refused when another device is current.
   static void* dev_addr[64] = {nullptr};
+  static std::mutex dev_addr_lock;
   int dev = -1;
   CUDA_OK(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return FM_ERR_UNSUPPORTED;
-  if (dev_addr[dev] == nullptr) {
-    void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_static_attn_scratch) != cudaSuccess || p == nullptr) return FM_ERR_CUDA;
-    dev_addr[dev] = p;
+  if (dev != c->device) return FM_ERR_BAD_STATE;
+  {
+    std::lock_guard<std::mutex> hold(dev_addr_lock);
+    if (dev_addr[dev] == nullptr) {
+      void* p = nullptr;
+      if (cudaGetSymbolAddress(&p, g_static_attn_scratch) != cudaSuccess || p == nullptr) return FM_ERR_CUDA;
+      dev_addr[dev] = p;
+    }
   }
   unsigned char* base = static_cast<unsigned char*>(dev_addr[dev]);
   // tickets must start at zero; the array keeps whatever the last call (of any context) left
@@ -1312,7 +1330,22 @@ double fm_verify_bytes(const fm_ctx* c, int32_t batch, const int32_t* kv_len) {
   return bytes;
 }
 
+int fm_attention_layout(const fm_ctx* c, int32_t level, int32_t* chunk_slots, int32_t* chunks_per_group, int32_t* max_groups) {
+  if (c == nullptr || level < 0 || level > 2) return FM_ERR_INVALID_ARG;
+  if (chunk_slots != nullptr) *chunk_slots = c->attn_chunk;
+  if (chunks_per_group != nullptr) *chunks_per_group = c->attn_G[level];
+  if (max_groups != nullptr) *max_groups = c->attn_max_groups[level];
+  return FM_OK;
+}
+
 int64_t fm_launch_count(const fm_ctx* c) { return c ? c->launches : 0; }
+
+int fm_selftest_wait_timeout(fm_ctx* c, int64_t limit_cycles) {
+  if (c == nullptr || limit_cycles < 1 || limit_cycles > 100000000ll) return FM_ERR_INVALID_ARG;
+  LAUNCH(c, wait_timeout_probe_kernel, 1, 32, 0, c->st.status, (long long)limit_cycles);
+  CUDA_OK(cudaGetLastError());
+  return FM_OK;
+}
 
 int fm_device_status(fm_ctx* c) {
   if (c == nullptr) return FM_ERR_INVALID_ARG;

@@ -95,7 +95,7 @@ __global__ void __launch_bounds__((NW + 1) * 32) attn_stream_kernel(const AttnAr
   if (nq <= 0 || mt * 16 >= M || u >= n_groups || n_groups > CF::MAX_GROUPS) {
     // nothing of the cache falls into this group yet; or more groups than the merge can stage
     // (the host sizes G so that this never happens): report, write nothing
-    if (n_groups > CF::MAX_GROUPS && threadIdx.x == 0) atomicExch(a.st.status, -1);
+    if (n_groups > CF::MAX_GROUPS && threadIdx.x == 0) atomicExch(a.st.status, -3);   // capacity
     ptx::grid_dep_wait();                          // keep the launch chain ordered
     return;
   }
@@ -283,6 +283,7 @@ __global__ void __launch_bounds__((NW + 1) * 32) attn_stream_kernel(const AttnAr
   __syncthreads();
   if (s_fail) {                                              // a bounded wait gave up: report, write nothing
     if (threadIdx.x == 0) atomicExch(a.st.status, -5);
+    ptx::drain_delay();                                      // chunks already requested may still be landing
     return;
   }
   // Merge of the NW warps' states, in warp order.  First every warp publishes its row maxima and

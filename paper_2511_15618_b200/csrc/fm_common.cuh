@@ -8,8 +8,8 @@ typedef __nv_bfloat16 bf16;
 
 // Ring sizes (entries per sequence) of the hourglass carry state, indexed by level-local
 // position modulo the size.  A verify pass touches coordinate positions L-2 .. L+D, vertices
-// ceil(L/3)-2 .. floor((L+D)/3) and faces ceil(L/9)-1 .. floor((L+D)/9); with D <= 24 these
-// spans are at most 27, 11 and 4 entries.
+// ceil(L/3)-2 .. floor((L+D)/3) and faces ceil(L/9)-1 .. floor((L+D)/9); with D <= 27 these
+// spans are at most 30, 12 and 5 entries.
 constexpr int FM_RING_C = 32;
 constexpr int FM_RING_V = 16;
 constexpr int FM_RING_F = 8;

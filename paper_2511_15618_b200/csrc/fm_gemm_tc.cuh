@@ -600,6 +600,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   fence_before();
   __syncthreads();
   fence_after();
+  if (s_fail) ptx::drain_delay();                          // a wait gave up: stages already requested may still be landing
   if (warp == 0) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(ncols) : "memory");
   }

@@ -428,17 +428,18 @@ __global__ void draft_residual_kernel(Dims dm, SeqState st, int batch, const flo
   }
 }
 
-// feature row that serves draft offset j of sequence b (single source per offset):
-// offsets 1,2 -> coordinate heads; later offsets in the current face -> vertex head
-// floor(p/3)-v*; offsets in a later face -> face head floor(p/9)-f*.
+// Feature row that serves draft offset j of sequence b (single source per offset; supplement,
+// "Optimizations"): offsets 1,2 -> coordinate heads (rule B); targets in the next two vertices
+// v*+1, v*+2 -> vertex head floor(p/3) - v*, wherever the face boundary lies, except where the
+// latest vertex row was also a face row (v* % 3 == 0): there the face level keeps the rest of
+// its own face (rule A), face head 1; targets beyond two vertices -> face head
+// floor(p/9) - f* + 1 (head e drafts face f* + e - 1).
 __device__ inline int draft_feature_row(int n, int j, int b, int B) {
   const int p = n + j;
   if (j <= 2) return (j - 1) * B + b;
-  if (p / 9 == n / 9) {
-    const int e = p / 3 - n / 3;
-    return 2 * B + 3 * ((e - 1) * B + b) + p % 3;
-  }
-  const int e = p / 9 - n / 9, s = p % 9;
+  const int ev = p / 3 - n / 3;
+  if (ev <= 2 && !((n / 3) % 3 == 0 && p / 9 == n / 9)) return 2 * B + 3 * ((ev - 1) * B + b) + p % 3;
+  const int e = p / 9 - n / 9 + 1, s = p % 9;
   return 2 * B + 3 * (2 * B + 3 * ((e - 1) * B + b) + s / 3) + s % 3;
 }
 
@@ -484,6 +485,18 @@ __global__ void draft_pick_kernel(Dims dm, SeqState st, int batch, const float* 
     }
     st.cand[b * dm.R1 + j] = tok;
     if (margin_out) margin_out[b * dm.D + j - 1] = t.v1 - t.v2;
+  }
+}
+
+// Self-check of the bounded waits: one thread waits on a barrier of its own that nothing ever
+// completes (no copy is in flight, nobody else knows the barrier), with a short limit; the wait
+// must come back false, and the kernel then reports it the way the GEMM and attention kernels do.
+__global__ void wait_timeout_probe_kernel(int* status, long long limit_cycles) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&bar, 1);
+    ptx::fence_mbar_init();
+    if (!ptx::mbar_wait(&bar, 0, limit_cycles)) atomicExch(status, -5);
   }
 }
 

@@ -41,6 +41,14 @@ __device__ inline bool mbar_wait(uint64_t* bar, uint32_t parity, long long limit
   return true;
 }
 
+// Give-up path of a kernel whose bounded wait ran out: before the CTA leaves (and its shared
+// memory can be handed to another CTA) let bulk copies it has already requested land.  They take
+// microseconds; this waits about a millisecond, once, on a path that is never taken in a healthy run.
+__device__ inline void drain_delay(long long cycles = 2000000ll) {
+  const long long t0 = clock64();
+  while (clock64() - t0 < cycles) {}
+}
+
 // ---------------------------------------------------------------- TMA
 __device__ inline void prefetch_tmap(const CUtensorMap* m) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");

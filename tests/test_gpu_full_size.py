@@ -13,7 +13,7 @@ pytestmark = pytest.mark.gpu
 
 def _setup(workload, start_faces, passes):
     import torch
-    from bench import MEAN_DRAFTS, _fill_prompt
+    from bench import MEAN_DRAFTS
     from paper_2511_15618_b200 import FlashMesh
     cfg = S.get_config(workload)
     B, D = cfg.batch, cfg.draft_len
@@ -25,7 +25,7 @@ def _setup(workload, start_faces, passes):
     prompts = []
     for b in range(B):
         f = start_faces if B == 1 else max(1, int(start_faces * rng.uniform(0.5, 1.0)))
-        prompts.append(_fill_prompt(cfg, b, f))
+        prompts.append(S.fill_prompt(cfg, b, f))
     dev = FlashMesh(cfg, w, max_tokens=max_tokens)
     del w
     keep = (S.accept_schedule(cfg.seed, B, 4096, D, MEAN_DRAFTS) - 1).astype(np.int32)
