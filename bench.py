@@ -63,9 +63,9 @@ def rank_sequences(rank, batch_per_rank):
 
 
 # DRAM traffic of the dominant kernel per launch from ncu (dram__bytes_read.sum +
-# dram__bytes_write.sum; profiles/gemm_traffic_medium.md), keyed by workload; None where the kernel
-# changed since the capture or none was taken.
-NCU_TRAFFIC = {"medium": 6.46e6}      # bytes per GEMM launch, mean over the four projections of a layer
+# dram__bytes_write.sum), keyed by workload, each with the summary under profiles/ that holds the
+# capture; None where the kernel changed since the capture or none was taken.
+NCU_TRAFFIC = {}
 
 
 class ClockSampler:
@@ -259,7 +259,9 @@ def run_ours(args):
         "mean_accept_len": emitted / max(1, steps * B * world),
         "natural_accept_len": st_nat.emitted / max(1, st_nat.steps * B),
         "natural_tokens_per_s": st_nat.emitted / (st_nat.ms * 1e-3),
-        "plain_tokens_per_s": B / (t_ori_ms * 1e-3), "plain_ms_per_step": t_ori_ms,
+        # the same D-draft pass with acceptance forced to one token (NOT T_ori of Sec. 4.1, which is
+        # the D = 0 run reported under "plain_decoding")
+        "single_accept_tokens_per_s": B / (t_ori_ms * 1e-3), "single_accept_ms_per_step": t_ori_ms,
         "clocks": clocks,
         "e2e": {"value": e2e["tokens"] / e2e["seconds"], "unit": "tokens/s",
                 "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
@@ -269,7 +271,8 @@ def run_ours(args):
         "roofline": {"bound": "hbm", "kernel": "tc::gemm_tc_kernel (all GEMM launches of one verify pass, timed alone as a graph)",
                      "achieved": gemm_gbs, "peak": peak, "unit": "GB/s", "frac": gemm_gbs / peak,
                      "peak_kind": peak_kind + " copy bandwidth (burst figure: the kernel is timed alone)",
-                     "traffic": NCU_TRAFFIC.get(args.workload),
+                     "traffic": NCU_TRAFFIC.get(args.workload, {}).get("bytes_per_launch"),
+                     "traffic_source": NCU_TRAFFIC.get(args.workload, {}).get("summary"),
                      "algorithmic_bytes_per_launch": gemm_bytes / max(1, gemm_n),
                      "launches_per_pass": int(gemm_n), "us_per_launch": gemm_ms * 1e3 / max(1, gemm_n),
                      "second_kernel": {"kernel": "attn_stream_kernel (all attention launches of one verify pass)",
@@ -451,6 +454,16 @@ def main():
                     help="teacher drafts with the true acceptance pinned to this many tokens per pass (1 .. D+1); 0 = seeded schedule")
     args = ap.parse_args()
     args.warmup = max(3, args.warmup) if args.impl == "ours" else args.warmup
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.gpus > 1 and world == 1 and "RANK" not in os.environ:
+        # started plainly with --gpus N: run the N replicas as N ranks, one per GPU
+        port = 29500 + os.getpid() % 2000
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        sys.exit(subprocess.run(cmd).returncode)
+    if args.gpus != world:
+        sys.exit(f"bench.py: --gpus {args.gpus} but WORLD_SIZE is {world}: launch one rank per GPU "
+                 f"(python -m torch.distributed.run --nproc-per-node {args.gpus} ... bench.py --gpus {args.gpus})")
     if args.impl == "reference":
         run_reference(args)
     else:
