@@ -19,7 +19,6 @@
 #include "fm_common.cuh"
 #include "fm_gemm_tc.cuh"
 #include "fm_kernels.cuh"
-#include "fm_mlp_fused.cuh"
 
 namespace {
 
@@ -28,7 +27,6 @@ constexpr int PREFILL_CHUNK = 256;      // conditioning rows projected per launc
 
 struct LayerDev {
   bf16 *Wqkv, *Wo, *W1, *W2;
-  bf16* W1p;                            // W1 again, dealt out per CTA for the fused feed-forward launch (or null)
   float *g1, *g2;
   bf16 *K, *V;                          // [max_batch, Hkv, P + cap, dh]
   int tmK, tmV;                         // tensor-map indices
@@ -105,10 +103,6 @@ struct fm_ctx {
   size_t attn_ticket_n;                      // entries of attn_ticket
   int split_target_deep;                     // the same for launches whose CTAs stream long K ranges
   int launch_error;     // first error met while enqueueing (capacity, descriptor creation)
-  // fused feed-forward launch for single-sequence passes (fm_mlp_fused.cuh); mlp_FB == 0: not available
-  int mlp_FB, mlp_CS;
-  float* mlp_part;
-  int* mlp_ticket;
   // one decode pass (draft, teacher edit, verify, accept) captured as a CUDA graph
   cudaGraph_t graph;
   cudaGraphExec_t graph_exec;
@@ -173,19 +167,6 @@ Dims make_dims(const fm_config& c) {
   return dm;
 }
 
-// Whether the feed-forward half runs as one fused launch on single-sequence passes: decided from
-// the shapes (and the device's SM count) alone, so that the workspace size is known up front.
-void decide_mlp(fm_ctx* c) {
-  int sms = 148, dev = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  if (sms <= 0) sms = 148;
-  const char* on = getenv("FM_FUSED_MLP");          // opt-in while the launch is slower than the two it replaces
-  c->mlp_FB = c->mlp_CS = 0;
-  if (on == nullptr || on[0] != '1') return;
-  if (c->dm.R1 > 16) return;
-  mlp::shape(c->dm.d, c->dm.dff, sms, c->mlp_FB, c->mlp_CS);
-}
-
 // bump allocator; with base == nullptr it only measures
 struct Carver {
   char* base; size_t off;
@@ -211,7 +192,6 @@ void carve(fm_ctx* c, Carver& cv) {
       L.Wo = cv.take<bf16>(align_up(d, 128) * hd);
       L.W1 = cv.take<bf16>(align_up((size_t)dm.dff, 128) * d);
       L.W2 = cv.take<bf16>(align_up(d, 128) * dm.dff);
-      L.W1p = c->mlp_FB > 0 ? cv.take<bf16>((size_t)dm.dff * d) : nullptr;
       L.g1 = cv.take<float>(d);
       L.g2 = cv.take<float>(d);
       L.K = cv.take<bf16>(kvn);
@@ -289,10 +269,6 @@ void carve(fm_ctx* c, Carver& cv) {
     const size_t tk = B * dm.Hkv * (size_t)c->attn_mt[l];
     ticket_max = tk > ticket_max ? tk : ticket_max;
   }
-  if (c->mlp_FB > 0) {
-    c->mlp_part = cv.take<float>((size_t)(dm.dff / (c->mlp_FB * c->mlp_CS)) * (d / 128) * 16 * 128);
-    c->mlp_ticket = cv.take<int>(d / 128);
-  }
   c->attn_part = cv.take<float>(part_max);
   c->attn_ticket = cv.take<int>(ticket_max);
   c->attn_ticket_n = ticket_max;
@@ -343,28 +319,6 @@ int upload_packed(bf16* dst, const float* src, size_t M, size_t K, std::vector<u
       else { u += 0x7fffu + ((u >> 16) & 1u); h = (uint16_t)(u >> 16); }
       const size_t kb = k / 64, c = (k % 64) / 8, e = k % 8;
       tmp[((t * slabs + kb) * 128 + r) * 64 + ((c ^ (r & 7)) * 8) + e] = h;
-    }
-  }
-  CUDA_OK(cudaMemcpy(dst, tmp.data(), tmp.size() * 2, cudaMemcpyHostToDevice));
-  return FM_OK;
-}
-// fp32 host matrix [M, K] -> blocks of FB rows, one block per CTA of the fused feed-forward launch:
-// [block g][K slab k][FB rows x 64 columns] with the same row pitch and swizzle as upload_packed
-// (row r at r*128 bytes, 16-byte chunk c at c ^ (r & 7)).  M must be a multiple of FB.
-int upload_dealt(bf16* dst, const float* src, size_t M, size_t K, size_t FB, std::vector<uint16_t>& tmp) {
-  if (src == nullptr) return FM_ERR_INVALID_ARG;
-  const size_t slabs = K / 64;
-  tmp.assign(M * K, 0);
-  for (size_t m = 0; m < M; ++m) {
-    const size_t gidx = m / FB, r = m % FB;
-    for (size_t k = 0; k < K; ++k) {
-      uint32_t u;
-      memcpy(&u, src + m * K + k, 4);
-      uint16_t h;
-      if ((u & 0x7fffffffu) > 0x7f800000u) h = 0x7fc0;
-      else { u += 0x7fffu + ((u >> 16) & 1u); h = (uint16_t)(u >> 16); }
-      const size_t kb = k / 64, cc = (k % 64) / 8, e = k % 8;
-      tmp[((gidx * slabs + kb) * FB + r) * 64 + ((cc ^ (r & 7)) * 8) + e] = h;
     }
   }
   CUDA_OK(cudaMemcpy(dst, tmp.data(), tmp.size() * 2, cudaMemcpyHostToDevice));
@@ -636,34 +590,6 @@ void attention(fm_ctx* c, int level, const LayerDev& L) {
 
 inline size_t pad128(size_t v) { return align_up(v, 128); }
 
-// x += W2 gelu(W1 rms(x)) as one launch (single-sequence passes; fm_mlp_fused.cuh).  On entry
-// c->a_norm / c->ssq hold the operand rows and their statistics as the output projection left them.
-void mlp_fused(fm_ctx* c, const LayerDev& L, float* x, int rows, const int* na, const float* gain, bool want_a) {
-  const Dims& dm = c->dm;
-  const size_t Rc_alloc = align_up((size_t)dm.max_batch * dm.R1, 16);
-  const int N = rows <= 8 ? 8 : 16;
-  const int tA = tmap_for(c, c->a_norm, Rc_alloc, (uint64_t)dm.d, N, 2u);
-  if (tA < 0) { c->launch_error = FM_ERR_CUDA; return; }
-  const int FB = c->mlp_FB, CS = c->mlp_CS, NC = dm.dff / (FB * CS);
-  mlp::Args g{};
-  g.W1p = L.W1p; g.W2 = L.W2; g.tmA = c->tmaps + tA;
-  g.d = dm.d; g.dff = dm.dff; g.N = N; g.rows = rows;
-  g.FB = FB; g.CS = CS; g.NC = NC;
-  g.ssq_in = c->ssq; g.ssq_n = c->ssq_n; g.ld_ssq = c->ssq_ld; g.inv_d = 1.f / dm.d; g.eps = dm.eps;
-  g.x = x; g.gain = gain;
-  g.a_out = want_a ? c->a_norm : nullptr;
-  g.ssq_out = want_a ? c->ssq : nullptr; g.ld_ssq_out = c->ssq_ld;
-  g.part = c->mlp_part; g.ticket = c->mlp_ticket; g.n_active = na; g.status = c->st.status;
-  const double bytes = 2.0 * 2.0 * dm.d * dm.dff;
-  const long pi = prof_open(c, PROF_GEMM, bytes);
-  c->cur_class = PROF_GEMM;
-  if (c->only_class == PROF_GEMM) c->class_bytes += bytes;
-  launch_pdl(c, dim3(CS, 1, 1), mlp::mlp_fused_kernel, dim3(CS, NC, 1), mlp::THREADS, (size_t)mlp::plan(dm.d, N, FB, CS).total, g);
-  c->cur_class = PROF_OTHER;
-  prof_close(c, pi);
-  if (want_a) c->ssq_n = dm.d / 128;
-}
-
 // One stack of pre-norm blocks on the rows of its level (a2/a4/a6/a8/a10): five launches per
 // layer.  On entry c->a_norm holds bf16(x * g1 of the first layer) and c->ssq the rows' sums of
 // squares; on exit, if `want_a`, c->a_norm holds bf16(x * next_gain) (gain 1 when null) and c->ssq
@@ -692,18 +618,13 @@ void run_stack(fm_ctx* c, int s, float* x, float* stash_ring, const float* next_
     eo.x = x; eo.ldx = d; eo.add = 1; eo.gain = L.g2; eo.a_out = c->a_norm; eo.lda = 2 * d; eo.lo_off = d;
     eo.ssq_out = c->ssq; eo.ld_ssq_out = c->ssq_ld;
     gemm(c, L.Wo, pad128(d), 0, c->a_attn, Rc_alloc, 0, d, hd, rows, na, tc::EPI_RESID, eo, 2);
-    const bool last = l == nl - 1;
-    const float* gain_after = last ? next_gain : c->layers[s][l + 1].g1;
-    if (c->mlp_FB > 0 && c->batch == 1 && L.W1p != nullptr) {       // single sequence: one launch for the feed-forward half
-      mlp_fused(c, L, x, rows, na, gain_after, !(last && !want_a));
-      continue;
-    }
     tc::Epi e1 = epi_plain(c->a_ff, 2 * dm.dff);
     e1.lo_off = dm.dff;
     e1.ssq_in = c->ssq; e1.ssq_n = c->ssq_n; e1.ld_ssq = c->ssq_ld; e1.inv_d_in = 1.f / d; e1.eps = dm.eps;
     gemm(c, L.W1, pad128(dm.dff), 0, c->a_norm, Rc_alloc, 0, dm.dff, d, rows, na, tc::EPI_GELU, e1, 2);
     tc::Epi e2 = eo;
-    e2.gain = gain_after;
+    const bool last = l == nl - 1;
+    e2.gain = last ? next_gain : c->layers[s][l + 1].g1;
     if (last && !want_a) { e2.a_out = nullptr; e2.ssq_out = nullptr; }
     gemm(c, L.W2, pad128(d), 0, c->a_ff, Rc_alloc, 0, d, dm.dff, rows, na, tc::EPI_RESID, e2, 2);
   }
@@ -943,7 +864,6 @@ size_t fm_workspace_bytes(const fm_config* cfg) {
   fm_ctx tmp{};
   tmp.cfg = *cfg;
   tmp.dm = make_dims(*cfg);
-  decide_mlp(&tmp);
   Carver cv{nullptr, 0};
   carve(&tmp, cv);
   return cv.off;
@@ -968,7 +888,6 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
   c->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   c->ws = static_cast<char*>(dev_workspace);
   c->ws_bytes = need;
-  decide_mlp(c);
   Carver cv{c->ws, 0};
   carve(c, cv);
   const Dims& dm = c->dm;
@@ -988,7 +907,6 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
       TRY(upload_packed(L.Wo, hw.Wo, d, hd, tmp));
       TRY(upload_packed(L.W1, hw.W1, (size_t)dm.dff, d, tmp));
       TRY(upload_packed(L.W2, hw.W2, d, (size_t)dm.dff, tmp));
-      if (L.W1p != nullptr) TRY(upload_dealt(L.W1p, hw.W1, (size_t)dm.dff, d, (size_t)c->mlp_FB, tmp));
       TRY(upload_f32(L.g1, hw.g1, d));
       TRY(upload_f32(L.g2, hw.g2, d));
     }
@@ -1025,9 +943,6 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
   TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_QKV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
   TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_RESID, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
   TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_QKV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
-  if (c->mlp_FB > 0)
-    TRYCUDA(cudaFuncSetAttribute(mlp::mlp_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 mlp::plan(dm.d, 16, c->mlp_FB, c->mlp_CS).total));
   TRYCUDA(cudaFuncSetAttribute(attn_stream_kernel<64, 128, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<64, 128, 8>::BYTES));
   TRYCUDA(cudaFuncSetAttribute(attn_stream_kernel<128, 64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<128, 64, 4>::BYTES));
   std::vector<double> freq(dm.dh / 2);
@@ -1172,7 +1087,6 @@ int fm_prefill(fm_ctx* c, int32_t batch, const float* cond, const int32_t* promp
   // the tickets of attention tiles whose last CTA never came to reset them
   CUDA_OK(cudaMemsetAsync(c->st.status, 0, sizeof(int), c->stream));
   CUDA_OK(cudaMemsetAsync(c->attn_ticket, 0, c->attn_ticket_n * sizeof(int), c->stream));
-  if (c->mlp_FB > 0) CUDA_OK(cudaMemsetAsync(c->mlp_ticket, 0, (c->dm.d / 128) * sizeof(int), c->stream));
   c->plen_host.assign(batch, 0);
   for (int b = 0; b < batch; ++b) c->plen_host[b] = prompt_off[b + 1] - prompt_off[b];
   CUDA_OK(cudaMemcpyAsync(c->prompt_off_dev, prompt_off, (batch + 1) * sizeof(int), cudaMemcpyHostToDevice, c->stream));
