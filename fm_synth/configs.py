@@ -40,6 +40,12 @@ class ModelConfig:
     cond_points: int = 0
     weight_std: float = 0.02
     out_std: float = 0.0                # std of the output matrix W_out; 0 => weight_std
+    # --- draft modules ---
+    draft_heads: str = "reduced"        # "reduced": SP = h + A rms(h), HF = the backbone's upsample matrices;
+                                        # "full": SP-Block with attention, HF-Blocks after every upsample
+    draft_levels: str = "three"         # "three": coordinate + point + face level; "coord": D coordinate heads only
+    hf_ff: int = 0                      # hidden width of the HF-Blocks' feed-forward networks; 0 => d_model
+    avg_levels: int = 0                 # 1: average the levels' distributions where several predict a position
     gain_std: float = 0.0               # 0 => RMSNorm gains exactly 1
 
     @property
@@ -59,9 +65,19 @@ class ModelConfig:
         return self.n_bins + 2
 
     @property
+    def n_coord_heads(self) -> int:
+        return 2 if self.draft_levels == "three" else self.draft_len
+
+    @property
+    def hf_width(self) -> int:
+        return self.hf_ff if self.hf_ff > 0 else self.d_model
+
+    @property
     def n_face_heads(self) -> int:
         # face head e drafts the face e - 1 after the one that holds the pending token; a draft
         # can reach face (8 + D) // 9 after it, and only offsets >= 7 ever leave the next two points
+        if self.draft_levels != "three":
+            return 0
         return 1 if self.draft_len < 7 else (self.draft_len + 8) // 9 + 1
 
     def with_(self, **kw) -> "ModelConfig":

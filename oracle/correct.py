@@ -12,8 +12,8 @@ What it follows (FlashMesh, arXiv 2511.15618, Sec. 3.2 "Correction Mechanism"):
   * finally the vertices are sorted again along z-y-x;
   * only draft tokens are touched, never the main token.
 
-The label head itself (a linear layer on point features) needs trained weights to mean anything:
-labels are inputs here.
+The label head itself (a linear layer on point features) is part of the draft modules
+(oracle/hourglass.py, OracleSeq.draft_labels); labels are inputs here.
 
 Readings taken where the section is silent:
   R1  a "point" of a candidate row is a vertex whose three coordinate tokens (z, y, x) are all
@@ -30,7 +30,15 @@ Readings taken where the section is silent:
   R6  re-sorting: inside each face, the points of the batch are sorted ascending by (z, y, x)
       among the slots they occupy (accepted vertices of the same face cannot move); faces are not
       reordered.
-  R7  historical points are not moved (the section gives no rule for them).
+  R7  historical points: the section defines the label (the point coincides with a vertex
+      generated before this batch) and gives no operation.  Without a history they are not moved.
+      With the accepted tokens given, the label is enforced the way the intra-batch rule enforces
+      its own: a historical point that equals no vertex of the history window is replaced by the
+      nearest vertex of the window (same distance, ties to the earliest).  The window holds the
+      complete accepted vertices of the face that contains the main token and of the face before
+      it (a shared vertex of a sorted mesh lies in a neighbouring face); the vertex that contains
+      the main token is not complete and is not in it.  Historical points are handled first, in
+      sequence order.
 
 Pins (tests/test_oracle_correct.py): a hand-worked case built like the section's figure (two
 displaced vertices snap to the vertices they should share, then the face is re-sorted); brute-force
@@ -58,11 +66,24 @@ def draft_points(L: int, n_cand: int):
     return out
 
 
-def correct_row(cand, labels, L: int, n_bins: int):
+def history_window(history, L: int, n_bins: int):
+    """Complete accepted vertices (z, y, x) of the face that holds the main token t_{L-1} and of
+    the face before it, oldest first (R7).  history[i] = mesh token t_i for i < L - 1."""
+    first = max(0, 3 * ((L - 1) // 9 - 1))           # first vertex of the previous face
+    out = []
+    for v in range(first, (L - 1) // 3):             # vertices whose three tokens precede the main token
+        c = tuple(int(history[3 * v + k]) for k in range(3))
+        if all(0 <= t < n_bins for t in c):
+            out.append(c)
+    return out
+
+
+def correct_row(cand, labels, L: int, n_bins: int, history=None):
     """Corrected copy of one sequence's candidate row.
 
     cand: D+1 token ids (main token first); labels: D+1 ints, labels[s] is the label of the
-    vertex that starts at slot s (read only at the slots `draft_points` returns)."""
+    vertex that starts at slot s (read only at the slots `draft_points` returns); history:
+    optional accepted mesh tokens t_0 .. t_{L-2} (R7)."""
     cand = [int(t) for t in cand]
     n = len(cand)
     starts = draft_points(L, n)
@@ -74,6 +95,18 @@ def correct_row(cand, labels, L: int, n_bins: int):
 
     def coords(s):
         return (cand[s], cand[s + 1], cand[s + 2])
+
+    # historical points against the accepted vertices (R7)
+    if history is not None:
+        window = history_window(history, L, n_bins)
+        for s, face, lab, ok in pts:
+            if lab != LABEL_HISTORICAL or not ok or not window:
+                continue
+            me = coords(s)
+            if me in window:
+                continue
+            dist = [sum((a - b) * (a - b) for a, b in zip(me, c)) for c in window]
+            cand[s:s + 3] = list(window[dist.index(min(dist))])
 
     # intra-batch points, in order (R3)
     for k, (s, face, lab, ok) in enumerate(pts):
@@ -105,6 +138,8 @@ def correct_row(cand, labels, L: int, n_bins: int):
     return cand
 
 
-def correct(cand_rows, label_rows, Ls, n_bins: int):
+def correct(cand_rows, label_rows, Ls, n_bins: int, histories=None):
     """All sequences of a pass: lists of rows, one L per sequence."""
-    return [correct_row(c, l, int(L), n_bins) for c, l, L in zip(cand_rows, label_rows, Ls)]
+    if histories is None:
+        histories = [None] * len(cand_rows)
+    return [correct_row(c, l, int(L), n_bins, h) for c, l, L, h in zip(cand_rows, label_rows, Ls, histories)]

@@ -14,6 +14,10 @@ What it follows (FlashMesh, arXiv 2511.15618):
   * Sec. 3.3: feed main + D drafts with causal masking, accept the main token, accept
     drafts up to the first mismatch, continue from the backbone's output there.
   * Supp. "Optimizations", rules (A) and (B): one draft source per future position.
+  * Sec. 3.1 Eq. 1-5 and Supp. "Three-Level Speculative Decoding": the full SP-Block and
+    HF-Blocks (`draft_heads == "full"`), the averaged merge of the levels (`avg_levels`), the
+    coordinate-only variant of the supplement's ablation (`draft_levels == "coord"`); Sec. 3.2:
+    the label head on the point-level features.
 
 Readings taken where the paper is silent: pre-norm
 RMSNorm, GELU(erf) FFN without biases, rotate-half RoPE on the level-local index,
@@ -94,8 +98,11 @@ def masked_top2(cfg, logits, target_index):
     return best, float(z[best] - np.max(rest))
 
 
-def draft_source(n, j, draft_len):
+def draft_source(n, j, draft_len, levels="three"):
     """Which head predicts draft offset j (target t_{n+j}) when the pending main token is t_n.
+
+    levels == "coord" is the variant of Supp. "Ablation on multi-level speculative decoding":
+    no point- or face-level modules, coordinate head j predicts offset j.  Otherwise:
 
     Supp. "Optimizations".  The levels fire at their own rows: the point level where a vertex
     starts (n % 3 == 0), the face level where a face starts (n % 9 == 0); rows in between
@@ -119,7 +126,7 @@ def draft_source(n, j, draft_len):
     v* + head), slot r of its 3 upsampled features; level 2 -> face head `head` (face
     f* + head - 1), slot r of its 9 features."""
     p = n + j
-    if j <= 2:
+    if j <= 2 or levels == "coord":
         return (0, j, 0)
     ev = p // 3 - n // 3
     if ev <= 2:
@@ -393,42 +400,151 @@ class OracleSeq:
         self.t_end = self.prompt_len + 9 * max_faces
         self.done = self.done or (self.L - 1 >= self.t_end)
 
-    def draft(self):
-        """Candidates [main, d_1..d_D] from the draft heads at the last accepted split nodes,
-        with the draft logits [D,V] and their top-2 margins."""
+    # -- draft modules (Sec. 3.1; Supp. "Three-Level Speculative Decoding") ----------------------
+    def _cache_attend(self, s, q, vis_pos):
+        """Attention of draft queries q[m,H,dh] (rotated) over the cache of the last layer of
+        stack s: the prefix keys and the accepted entries that the row at `vis_pos` sees
+        (positions max(0, vis_pos - W + 1) .. vis_pos).  Returns [m, H*dh]."""
+        cfg = self.cfg
+        l = len(self.w["stacks"][s]) - 1
+        W = cfg.window[STACK_LEVEL[s]]
+        lo = max(0, vis_pos - W + 1) if W > 0 else 0
+        keys = np.concatenate([self.KP[s][l], self.K[s][l][lo:vis_pos + 1]])
+        vals = np.concatenate([self.VP[s][l], self.V[s][l][lo:vis_pos + 1]])
+        mask = np.ones((q.shape[0], keys.shape[0]), dtype=bool)
+        return _attend(cfg, q, keys, vals, mask).reshape(q.shape[0], -1)
+
+    def _sp_block(self, z, hw, level, pos):
+        """Eq. 1: h^(d) = Linear(CA(SA(h_s), c)) + h_s for one head.  Reduced heads: the attention
+        is left out, h + A rms(h).  Full heads: the attention (self-attention and conditioning in
+        one softmax, as in every block of this model) reads the cache of the backbone's last
+        layer at this level -- the layer whose input the split-node hiddens are -- with the
+        head's own query and output projections: y = h + Wo Attn(Wq rms(h, ga)); then
+        h^(d) = h + A rms(y, g)."""
+        cfg = self.cfg
+        y = z
+        if cfg.draft_heads == "full":
+            s = (4, 3, 2)[level]
+            a = rms_norm(z, hw["ga"], cfg.norm_eps)
+            q = rope((hw["Wq"] @ a).reshape(1, cfg.n_heads, cfg.head_dim), [pos], cfg.rope_theta)
+            y = z + hw["Wo"] @ self._cache_attend(s, q, pos)[0]
+        return z + hw["A"] @ rms_norm(y, hw["g"], cfg.norm_eps)
+
+    def _hf_block(self, x, hw, level, qpos, vis_pos):
+        """Eq. 3-5: an upsampled feature for level position `qpos` queries the backbone's cache
+        at that level (its last layer, entries up to the last accepted position `vis_pos`) with
+        the offset's own W_q, and the offset's own FFN maps the attention output back:
+        x + FFN(Attn(W_q rms(x), K, V)).  Reduced heads: identity."""
+        cfg = self.cfg
+        if cfg.draft_heads != "full":
+            return x
+        s = (4, 3)[level]
+        a = rms_norm(x, hw["g"], cfg.norm_eps)
+        q = rope((hw["Wq"] @ a).reshape(1, cfg.n_heads, cfg.head_dim), [qpos], cfg.rope_theta)
+        o = self._cache_attend(s, q, vis_pos)[0]
+        return x + hw["W2"] @ gelu(hw["W1"] @ o)
+
+    def draft_features(self):
+        """Coordinate-level features of every head at the last accepted split nodes, keyed like
+        draft_source's result, and the point-level features they came from (for the label head):
+        points[(1, e, 0)] for vertex head e, points[(2, e, rv)] for vertex rv of face head e."""
         cfg, w, d = self.cfg, self.w, self.cfg.d_model
+        n = self.L - 1
+        vs, fs = n // 3, n // 9
+        feats, points = {}, {}
+        for k in range(1, cfg.n_coord_heads + 1):                      # coordinate level: SP only
+            feats[(0, k, 0)] = self._sp_block(self.zc[n], w["heads_c"][k - 1], 0, n)
+        if cfg.draft_levels != "three":
+            return feats, points
+        hf_vc = w.get("hf_vc", [None] * 6)
+        hf_fv = w.get("hf_fv", [None] * (3 * cfg.n_face_heads))
+        hf_fc = w.get("hf_fc", [None] * (9 * cfg.n_face_heads))
+        for e in (1, 2):                                               # point level: SP, upsample, one HF
+            yv = self._sp_block(self.zv[vs], w["heads_v"][e - 1], 1, vs)
+            points[(1, e, 0)] = yv
+            tri = w["U_vc"] @ yv                                       # Eq. 2: one vertex -> 3 coordinates
+            for r in range(3):
+                feats[(1, e, r)] = self._hf_block(tri[r * d:(r + 1) * d], hf_vc[3 * e + r - 3], 0, 3 * (vs + e) + r, n)
+        for e in range(1, cfg.n_face_heads + 1):                       # face level: SP, upsample, HF, upsample, HF
+            yf = self._sp_block(self.zf[fs], w["heads_f"][e - 1], 2, fs)       # head e drafts face f* + e - 1
+            tri = w["U_fv"] @ yf                                       # one face -> 3 vertices
+            for rv in range(3):
+                xv = self._hf_block(tri[rv * d:(rv + 1) * d], hf_fv[3 * (e - 1) + rv], 1, 3 * (fs + e - 1) + rv, vs)
+                points[(2, e, rv)] = xv
+                sub = w["U_vc"] @ xv                                   # each vertex -> 3 coordinates
+                for r in range(3):
+                    feats[(2, e, 3 * rv + r)] = self._hf_block(sub[r * d:(r + 1) * d], hf_fc[9 * (e - 1) + 3 * rv + r], 0,
+                                                               9 * (fs + e - 1) + 3 * rv + r, n)
+        return feats, points
+
+    def _all_sources(self, n, j):
+        """Every level that predicts offset j (Supp. "Integrating the three levels", before the
+        optimisation rules pick one): the coordinate head if there is one for j, the point level
+        for the next two vertices, the face level for the faces its heads draft (never the
+        vertex that holds the pending token: that one is the backbone's)."""
+        cfg = self.cfg
+        p = n + j
+        out = []
+        if j <= cfg.n_coord_heads:
+            out.append((0, j, 0))
+        if cfg.draft_levels == "three":
+            ev, ef = p // 3 - n // 3, p // 9 - n // 9 + 1
+            if 1 <= ev <= 2:
+                out.append((1, ev, p % 3))
+            if ev >= 1 and 1 <= ef <= cfg.n_face_heads:
+                out.append((2, ef, p % 9))
+        return out
+
+    def draft(self):
+        """Candidates [main, d_1..d_D] from the draft modules at the last accepted split nodes,
+        with the draft logits [D,V] and their top-2 margins.  With cfg.avg_levels the logits of
+        an offset are the logarithm of the mean of the levels' softmax distributions."""
+        cfg, w = self.cfg, self.w
         D = cfg.draft_len
         if self.done:
             return [cfg.pad] * (D + 1), np.zeros((D, cfg.vocab)), [0.0] * D
         n = self.L - 1
-        vs, fs = n // 3, n // 9
-        zc, zv, zf = self.zc[n], self.zv[vs], self.zf[fs]
+        feats, self.points = self.draft_features()
 
-        def head(z, hw):                       # Eq. 1 reduced to Linear + residual
-            return z + hw["A"] @ rms_norm(z, hw["g"], cfg.norm_eps)
+        def logits_of(f):
+            return w["W_out"] @ rms_norm(f, w["g_out"], cfg.norm_eps)
 
-        feats = {}
-        for k in (1, 2):
-            feats[(0, k, 0)] = head(zc, w["heads_c"][k - 1])
-        for e in (1, 2):
-            tri = w["U_vc"] @ head(zv, w["heads_v"][e - 1])           # Eq. 2: one vertex -> 3 coordinates
-            for r in range(3):
-                feats[(1, e, r)] = tri[r * d:(r + 1) * d]
-        for e in range(1, cfg.n_face_heads + 1):                       # head e drafts face f* + e - 1
-            tri = w["U_fv"] @ head(zf, w["heads_f"][e - 1])           # one face -> 3 vertices
-            for rv in range(3):
-                sub = w["U_vc"] @ tri[rv * d:(rv + 1) * d]             # each vertex -> 3 coordinates
-                for r in range(3):
-                    feats[(2, e, 3 * rv + r)] = sub[r * d:(r + 1) * d]
         cand, dl, margins = [self.main], [], []
         for j in range(1, D + 1):
-            f = feats[draft_source(n, j, D)]
-            logits = w["W_out"] @ rms_norm(f, w["g_out"], cfg.norm_eps)
+            if cfg.avg_levels:
+                probs = [softmax_rows(logits_of(feats[src])[None])[0] for src in self._all_sources(n, j)]
+                logits = np.log(np.mean(probs, axis=0))
+            else:
+                logits = logits_of(feats[draft_source(n, j, D, cfg.draft_levels)])
             tok, mg = masked_top2(cfg, logits, n + j)
             cand.append(tok)
             dl.append(logits)
             margins.append(mg)
         return cand, np.stack(dl) if D else np.zeros((0, cfg.vocab)), margins
+
+    def draft_labels(self):
+        """Sec. 3.2: a label head (a linear layer, here behind an RMSNorm) on the point-level
+        feature of every drafted point.  Slot s of the candidate row holds mesh token n + s; a
+        point starts at slot s >= 1 when (n + s) % 3 == 0 and its three tokens are drafts of the
+        row.  Its feature is the point-level feature in the pipeline of the head that drafts its
+        last coordinate.  Returns (labels[D+1] with -1 where no point starts, margins[D+1]).
+        Call after draft()."""
+        cfg, w = self.cfg, self.w
+        D = cfg.draft_len
+        labels, margins = [-1] * (D + 1), [0.0] * (D + 1)
+        if self.done or cfg.draft_levels != "three":
+            return labels, margins
+        n = self.L - 1
+        for s in range(1, D - 1):
+            if (n + s) % 3 != 0:
+                continue
+            level, head, slot = draft_source(n, s + 2, D)
+            f = self.points[(1, head, 0)] if level == 1 else self.points[(2, head, slot // 3)]
+            z = w["label"]["W"] @ rms_norm(f, w["label"]["g"], cfg.norm_eps)
+            best = int(np.argmax(z))
+            rest = np.delete(z, best)
+            labels[s], margins[s] = best, float(z[best] - rest.max())
+        return labels, margins
 
     def verify(self, cand):
         """One forward pass over the candidates (Sec. 3.3).  Rows fed = min(D+1, tokens left).

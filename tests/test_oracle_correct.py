@@ -124,3 +124,57 @@ def test_single_intra_point_takes_the_nearest_earlier_new_point_of_another_face(
     for f in range(3):
         want += sorted(tuple(int(t) for t in v) for v in expect[3 * f:3 * f + 3])
     assert out == [0] + [t for v in want for t in v]
+
+
+# ------------------------------------------------------------------ historical points (R7)
+def test_history_window_holds_the_complete_vertices_of_this_face_and_the_one_before():
+    from oracle.correct import history_window
+    hist = list(range(100))                              # token i has the value i: vertices are (3v, 3v+1, 3v+2)
+    # L = 23: main token is t_22, coordinate 1 of vertex 7 (face 2); complete vertices before it: 0..6;
+    # the window starts with the previous face (face 1 = vertices 3, 4, 5) and ends with vertex 6
+    assert history_window(hist, 23, 1000) == [(9, 10, 11), (12, 13, 14), (15, 16, 17), (18, 19, 20)]
+    assert history_window(hist, 1, 1000) == []           # right after BOS nothing is accepted
+    assert history_window(hist, 10, 1000) == [(0, 1, 2), (3, 4, 5), (6, 7, 8)]   # main = first token of face 1
+    assert history_window([5, 5, 1001, 1, 2, 3], 7, 1000) == [(1, 2, 3)]      # a vertex with a special token is skipped
+
+
+def test_historical_point_snaps_to_the_nearest_accepted_vertex_hand_worked():
+    # accepted: face 0 = (1,1,1) (4,4,4) (9,9,9); the main token opens face 1.  The drafted face has
+    # a point labelled historical at (4,5,4): distance 1 to (4,4,4), 27+... to the others -> (4,4,4);
+    # a historical point that already equals an accepted vertex stays; a new point is not touched.
+    hist = [1, 1, 1, 4, 4, 4, 9, 9, 9]
+    cand = [2, 2, 2, 4, 5, 4, 9, 9, 9, 7]               # main token 2, then slots 1.. : (2,2 | ...) see below
+    # L = 10: slot 0 is t_9 (first coordinate of vertex 3); slots 1,2 finish that vertex; points start at slots 3 and 6
+    labels = [0, 0, 0, H, 0, 0, H, 0, 0, 0]
+    out = correct_row(cand, labels, 10, BINS, history=hist)
+    assert out == [2, 2, 2, 4, 4, 4, 9, 9, 9, 7]
+    assert correct_row(cand, labels, 10, BINS) == cand                         # no history given: not moved
+    labels[3] = N
+    assert correct_row(cand, labels, 10, BINS, history=hist) == cand
+
+
+@pytest.mark.parametrize("seed", range(20))
+def test_historical_rule_brute_force(seed):
+    from oracle.correct import history_window
+    rng = np.random.default_rng(100 + seed)
+    L = int(rng.integers(1, 60))
+    n = int(rng.integers(4, 28))
+    hist = rng.integers(0, 6, size=L - 1).tolist()
+    cand = rng.integers(0, 6, size=n).tolist()
+    labels = rng.choice([H, N], size=n).tolist()          # no intra-batch points: only R7 and the sort act
+    out = correct_row(cand, labels, L, BINS, history=hist)
+    win = history_window(hist, L, BINS)
+    by_face = {}
+    for s in draft_points(L, n):
+        before = tuple(cand[s:s + 3])
+        if labels[s] == H and win and before not in win:
+            dmin = min(sum((a - b) ** 2 for a, b in zip(before, c)) for c in win)
+            want = next(c for c in win if sum((a - b) ** 2 for a, b in zip(before, c)) == dmin)
+        else:
+            want = before
+        by_face.setdefault((L - 1 + s) // 9, []).append((s, want))
+    for f, items in by_face.items():                      # then sorted inside the face
+        slots = [s for s, _ in items]
+        for s, v in zip(slots, sorted(w for _, w in items)):
+            assert tuple(out[s:s + 3]) == v
+    assert out[0] == cand[0]
