@@ -80,7 +80,23 @@ typedef struct fm_config {
   float   rope_theta;         /* 0 = no positional encoding                                  */
   float   norm_eps;
   int32_t allow_eos;          /* 0: EOS is masked everywhere (fixed-length runs)             */
+  /* draft modules (Sec. 3.1; supplement "Three-Level Speculative Decoding") */
+  int32_t draft_heads;        /* FM_HEADS_REDUCED: SP = h + A rms(h), HF = the upsample matrices alone;
+                                 FM_HEADS_FULL: SP-Blocks with attention (Eq. 1), an HF-Block after
+                                 every upsample (Eq. 2-5)                                     */
+  int32_t draft_levels;       /* FM_LEVELS_THREE: 2 coordinate heads + point level + face level;
+                                 FM_LEVELS_COORD: D coordinate heads, no point / face level (the
+                                 supplement's ablation on multi-level decoding)               */
+  int32_t hf_ff;              /* hidden width of the HF-Blocks' feed-forward networks (0 = d_model;
+                                 a multiple of 64)                                            */
+  int32_t avg_levels;         /* 1: where several levels predict a position their softmax
+                                 distributions are averaged (supplement, "Integrating the three
+                                 levels"); 0: one source per position ("Optimizations")       */
 } fm_config;
+#define FM_HEADS_REDUCED 0
+#define FM_HEADS_FULL    1
+#define FM_LEVELS_THREE  0
+#define FM_LEVELS_COORD  1
 
 /* HOST pointers to float32 matrices, row-major [out, in]; values are rounded to bfloat16
  * (nearest-even) when fm_create copies them.  Gains stay float32. */
@@ -93,6 +109,22 @@ typedef struct fm_layer_weights {
   const float* W2;            /* [d, d_ff]                                                    */
 } fm_layer_weights;
 
+/* One SP-Block head (Eq. 1).  Reduced: y = h + A rms(h, g).  Full: the attention of the block reads
+ * the cache of the backbone's last layer at the head's level (keys / values of the split-node hiddens;
+ * conditioning as the prefix entries of the same softmax) with the head's own query and output
+ * matrices: u = h + Wo Attn(Wq rms(h, ga)), y = h + A rms(u, g).  ga / Wq / Wo are read only with
+ * FM_HEADS_FULL. */
+typedef struct fm_sp_weights {
+  const float* g;  const float* A;        /* [d], [d, d]                                       */
+  const float* ga; const float* Wq; const float* Wo;   /* [d], [H*dh, d], [d, H*dh]            */
+} fm_sp_weights;
+
+/* One HF-Block (Eq. 3-5) for one offset: x + W2 gelu(W1 Attn(Wq rms(x, g), K, V)) with K, V the cache
+ * of the backbone's last layer at the block's level, entries up to the last accepted position. */
+typedef struct fm_hf_weights {
+  const float* g; const float* Wq; const float* W1; const float* W2;   /* [d], [H*dh, d], [hf, H*dh], [d, hf] */
+} fm_hf_weights;
+
 typedef struct fm_weights {
   const float* E;                         /* [V, d] token embedding                          */
   const fm_layer_weights* stack[5];       /* stack[s][l], l < layers[s]                      */
@@ -102,11 +134,23 @@ typedef struct fm_weights {
   const float* U_vc;                      /* [3d, d] upsample vertex -> 3 coordinates        */
   const float* g_out;                     /* [d]                                              */
   const float* W_out;                     /* [V, d]                                           */
-  const float* head_c_g[2];  const float* head_c_A[2];   /* coordinate draft heads, A [d,d]  */
-  const float* head_v_g[2];  const float* head_v_A[2];   /* vertex (point) draft heads       */
-  const float* head_f_g[FM_MAX_FACE_HEADS]; const float* head_f_A[FM_MAX_FACE_HEADS];
-                              /* face head e (1-based) drafts the face e-1 after the one that holds the
-                                 pending token; D < 7 uses 1 head, otherwise (D+8)/9 + 1 */
+  /* Draft modules.  heads_c: coordinate heads (2, or D with FM_LEVELS_COORD); heads_v: 2 point-level
+   * heads (vertex v*+1, v*+2); heads_f: face-level heads, head e (1-based) drafts the face e-1 after
+   * the one that holds the pending token; D < 7 uses 1 head, otherwise (D+8)/9 + 1.  heads_v,
+   * heads_f and the HF-Blocks are not read with FM_LEVELS_COORD. */
+  const fm_sp_weights* heads_c;
+  const fm_sp_weights* heads_v;
+  const fm_sp_weights* heads_f;
+  /* HF-Blocks (FM_HEADS_FULL only): hf_vc[6] refine the point level's coordinate features (offset
+   * 3..8 from the vertex row), hf_fv[3*Ef] the face level's vertex features, hf_fc[9*Ef] the face
+   * level's coordinate features. */
+  const fm_hf_weights* hf_vc;
+  const fm_hf_weights* hf_fv;
+  const fm_hf_weights* hf_fc;
+  /* label head of the correction stage (Sec. 3.2): gain [d] and matrix [3, d]; may be NULL (then
+   * fm_draft produces no labels) */
+  const float* label_g;
+  const float* label_W;
 } fm_weights;
 
 /* Optional device-side draft editor for fm_generate: the place where the paper's Correct
@@ -178,6 +222,21 @@ int fm_draft(fm_ctx* ctx, int32_t* cand /*DEV*/, float* draft_logits /*DEV*/, fl
 #define FM_LABEL_NEW 1
 #define FM_LABEL_INTRA 2
 int fm_correct(fm_ctx* ctx, int32_t* cand /*DEV*/, const int32_t* labels /*DEV*/);
+
+/* Labels of the drafted points (Sec. 3.2: a label head, a linear layer, on every point-level
+ * feature), as computed by the last fm_draft: labels[b][s] in {FM_LABEL_HISTORICAL, FM_LABEL_NEW,
+ * FM_LABEL_INTRA} where a vertex made of drafts only starts at slot s, -1 elsewhere; the label is
+ * the argmax (ties to the lowest) of label_W rms(f, label_g) over the point-level feature f in the
+ * pipeline of the head that drafts the point's last coordinate.  margin: top-1 minus top-2, or NULL.
+ * DEV out [batch, D+1].  Errors: UNSUPPORTED without a label head or with FM_LEVELS_COORD. */
+int fm_draft_labels(fm_ctx* ctx, int32_t* labels /*DEV*/, float* margin /*DEV*/);
+
+/* fm_correct with two options: labels == NULL takes the label head's labels of the last fm_draft;
+ * use_history != 0 also enforces the historical label against the accepted tokens: a point labelled
+ * FM_LABEL_HISTORICAL that equals no complete accepted vertex of the face that holds the pending
+ * token or of the face before it is replaced by the nearest of them (same distance, ties to the
+ * earliest); historical points are handled first, in sequence order. */
+int fm_correct_ex(fm_ctx* ctx, int32_t* cand /*DEV*/, const int32_t* labels /*DEV or NULL*/, int32_t use_history);
 
 /* Verify (Sec. 3.3): one forward pass over main + D candidates, causal among themselves,
  * through all five level stacks.  cand: DEV int32 in [batch, D+1]; cand[b][0] must be the

@@ -38,7 +38,8 @@ def run_lockstep(cfg, w, conds, prompts, dev, max_faces, max_steps, *, tol=2e-2,
     dev.prefill(np.stack(conds), prompts)
     dev.set_max_faces([max_faces[b] if hasattr(max_faces, "__len__") else max_faces for b in range(B)])
     rep = dict(steps=0, emitted=0, overrides=0, max_logit_err=0.0, max_draft_err=0.0, rows=0, low_margin_rows=0,
-               argmax_flips=0, draft_flips=0, accept_hist=[0] * (D + 2))
+               argmax_flips=0, draft_flips=0, accept_hist=[0] * (D + 2), labels=0, label_flips=0)
+    check_labels = check_drafts and D > 0 and cfg.draft_levels == "three" and hasattr(dev, "draft_labels")
     for _ in range(max_steps):
         if all(s.done for s in seqs):
             break
@@ -60,6 +61,22 @@ def run_lockstep(cfg, w, conds, prompts, dev, max_faces, max_steps, *, tol=2e-2,
                         assert cand_g[b, j] == o_d[b][0][j], "draft id differs at a decisive margin"
                     elif cand_g[b, j] != o_d[b][0][j]:
                         rep["draft_flips"] += 1
+        # ---- labels of the drafted points (Sec. 3.2): equal where the oracle's margin is decisive
+        if check_labels:
+            lab_g = _np(dev.draft_labels()[0])
+            for b, s in enumerate(seqs):
+                if s.done:
+                    assert (lab_g[b] == -1).all()
+                    continue
+                lab_o, lmg_o = s.draft_labels()
+                for sl in range(D + 1):
+                    assert (lab_g[b, sl] == -1) == (lab_o[sl] == -1), "label slots differ"
+                    if lab_o[sl] >= 0:
+                        rep["labels"] += 1
+                        if lmg_o[sl] > margin:
+                            assert lab_g[b, sl] == lab_o[sl], "label differs at a decisive margin"
+                        elif lab_g[b, sl] != lab_o[sl]:
+                            rep["label_flips"] += 1
         # ---- candidates: the oracle's, optionally teacher-edited
         cands = []
         for b, s in enumerate(seqs):

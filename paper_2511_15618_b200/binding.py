@@ -29,7 +29,8 @@ class FmConfig(C.Structure):
                 ("d_ff", C.c_int32), ("layers", C.c_int32 * 5), ("n_bins", C.c_int32), ("n_prefix", C.c_int32),
                 ("window", C.c_int32 * 3), ("draft_len", C.c_int32), ("max_batch", C.c_int32),
                 ("max_tokens", C.c_int32), ("rope_theta", C.c_float), ("norm_eps", C.c_float),
-                ("allow_eos", C.c_int32)]
+                ("allow_eos", C.c_int32), ("draft_heads", C.c_int32), ("draft_levels", C.c_int32),
+                ("hf_ff", C.c_int32), ("avg_levels", C.c_int32)]
 
 
 _FP = C.POINTER(C.c_float)
@@ -39,11 +40,20 @@ class FmLayerWeights(C.Structure):
     _fields_ = [(n, _FP) for n in ("g1", "Wqkv", "Wo", "g2", "W1", "W2")]
 
 
+class FmSpWeights(C.Structure):
+    _fields_ = [(n, _FP) for n in ("g", "A", "ga", "Wq", "Wo")]
+
+
+class FmHfWeights(C.Structure):
+    _fields_ = [(n, _FP) for n in ("g", "Wq", "W1", "W2")]
+
+
 class FmWeights(C.Structure):
     _fields_ = [("E", _FP), ("stack", C.POINTER(FmLayerWeights) * 5),
                 ("S_cv", _FP), ("S_vf", _FP), ("U_fv", _FP), ("U_vc", _FP), ("g_out", _FP), ("W_out", _FP),
-                ("head_c_g", _FP * 2), ("head_c_A", _FP * 2), ("head_v_g", _FP * 2), ("head_v_A", _FP * 2),
-                ("head_f_g", _FP * FM_MAX_FACE_HEADS), ("head_f_A", _FP * FM_MAX_FACE_HEADS)]
+                ("heads_c", C.POINTER(FmSpWeights)), ("heads_v", C.POINTER(FmSpWeights)), ("heads_f", C.POINTER(FmSpWeights)),
+                ("hf_vc", C.POINTER(FmHfWeights)), ("hf_fv", C.POINTER(FmHfWeights)), ("hf_fc", C.POINTER(FmHfWeights)),
+                ("label_g", _FP), ("label_W", _FP)]
 
 
 class FmTeacher(C.Structure):
@@ -89,6 +99,10 @@ def load_library():
     lib.fm_draft.argtypes = [vp, vp, f32p, f32p]
     lib.fm_correct.restype = C.c_int
     lib.fm_correct.argtypes = [vp, vp, vp]
+    lib.fm_draft_labels.restype = C.c_int
+    lib.fm_draft_labels.argtypes = [vp, vp, f32p]
+    lib.fm_correct_ex.restype = C.c_int
+    lib.fm_correct_ex.argtypes = [vp, vp, vp, i32]
     lib.fm_verify.restype = C.c_int
     lib.fm_verify.argtypes = [vp, vp, vp, f32p, f32p]
     lib.fm_verify_static_scratch.restype = C.c_int
@@ -157,6 +171,14 @@ def fm_draft(ctx, cand_ptr, draft_logits_ptr=None, draft_margin_ptr=None):
 
 def fm_correct(ctx, cand_ptr, labels_ptr):
     return load_library().fm_correct(ctx, cand_ptr, labels_ptr)
+
+
+def fm_draft_labels(ctx, labels_ptr, margin_ptr=None):
+    return load_library().fm_draft_labels(ctx, labels_ptr, margin_ptr)
+
+
+def fm_correct_ex(ctx, cand_ptr, labels_ptr=None, use_history=0):
+    return load_library().fm_correct_ex(ctx, cand_ptr, labels_ptr, int(use_history))
 
 
 def fm_verify(ctx, cand_ptr, argmax_ptr=None, logits_ptr=None, margin_ptr=None):
@@ -232,6 +254,10 @@ def make_config(mc, max_batch=None, max_tokens=None, draft_len=None) -> FmConfig
     cfg.max_batch = mc.max_batch if max_batch is None else max_batch
     cfg.max_tokens = mc.max_tokens if max_tokens is None else max_tokens
     cfg.rope_theta, cfg.norm_eps, cfg.allow_eos = mc.rope_theta, mc.norm_eps, mc.allow_eos
+    cfg.draft_heads = 1 if getattr(mc, "draft_heads", "reduced") == "full" else 0
+    cfg.draft_levels = 1 if getattr(mc, "draft_levels", "three") == "coord" else 0
+    cfg.hf_ff = int(getattr(mc, "hf_ff", 0))
+    cfg.avg_levels = int(getattr(mc, "avg_levels", 0))
     return cfg
 
 
@@ -240,7 +266,7 @@ def _fp(a):
     return a.ctypes.data_as(_FP)
 
 
-def make_weights(w: dict, n_face_heads: int):
+def make_weights(w: dict):
     """FmWeights pointing into the float32 numpy arrays of `w` (which must stay alive)."""
     fw = FmWeights()
     keep = []
@@ -254,11 +280,22 @@ def make_weights(w: dict, n_face_heads: int):
         fw.stack[s] = C.cast(arr, C.POINTER(FmLayerWeights))
     for name in ("S_cv", "S_vf", "U_fv", "U_vc", "g_out", "W_out"):
         setattr(fw, name, _fp(w[name]))
-    for k in range(2):
-        fw.head_c_g[k], fw.head_c_A[k] = _fp(w["heads_c"][k]["g"]), _fp(w["heads_c"][k]["A"])
-        fw.head_v_g[k], fw.head_v_A[k] = _fp(w["heads_v"][k]["g"]), _fp(w["heads_v"][k]["A"])
-    for k in range(min(n_face_heads, len(w["heads_f"]))):
-        fw.head_f_g[k], fw.head_f_A[k] = _fp(w["heads_f"][k]["g"]), _fp(w["heads_f"][k]["A"])
+
+    def block_array(kind, fields, blocks):
+        arr = (kind * max(1, len(blocks)))()
+        for i, blk in enumerate(blocks):
+            for name in fields:
+                if name in blk:
+                    setattr(arr[i], name, _fp(blk[name]))
+        keep.append(arr)
+        return C.cast(arr, C.POINTER(kind))
+
+    for name in ("heads_c", "heads_v", "heads_f"):
+        setattr(fw, name, block_array(FmSpWeights, ("g", "A", "ga", "Wq", "Wo"), w.get(name, [])))
+    for name in ("hf_vc", "hf_fv", "hf_fc"):
+        setattr(fw, name, block_array(FmHfWeights, ("g", "Wq", "W1", "W2"), w.get(name, [])))
+    if "label" in w:
+        fw.label_g, fw.label_W = _fp(w["label"]["g"]), _fp(w["label"]["W"])
     return fw, keep
 
 
@@ -285,7 +322,7 @@ class FlashMesh:
             base = (self.workspace.data_ptr() + 255) // 256 * 256
             # a stream of its own: the legacy default stream cannot be captured into a CUDA graph
             self.stream = stream if stream is not None else torch.cuda.Stream(self.device)
-            fw, self._keep = make_weights(weights, 0 if self.D == 0 else (1 if self.D < 7 else (self.D + 8) // 9 + 1))
+            fw, self._keep = make_weights(weights)
             rc, self.ctx = fm_create(self.cfg, fw, base, nbytes, self.stream.cuda_stream)
         if rc != 0:
             raise FmError(rc, "fm_create")
@@ -373,13 +410,27 @@ class FlashMesh:
         self._after(cand, dl, dm)
         return cand, dl, dm
 
-    def correct(self, cand, labels):
+    def correct(self, cand, labels=None, use_history=False):
         """Edit the drafts of `cand` (int32 [B, D+1], device) in place with the per-point labels
-        (int32 [B, D+1], device); returns `cand`."""
+        (int32 [B, D+1], device; None = the label head's of the last draft); returns `cand`."""
         self._before()
-        self._check(fm_correct(self.ctx, cand.data_ptr(), labels.data_ptr()), "fm_correct")
+        if labels is not None and not use_history:
+            self._check(fm_correct(self.ctx, cand.data_ptr(), labels.data_ptr()), "fm_correct")
+        else:
+            self._check(fm_correct_ex(self.ctx, cand.data_ptr(), labels.data_ptr() if labels is not None else None,
+                                      1 if use_history else 0), "fm_correct_ex")
         self._after(cand, labels)
         return cand
+
+    def draft_labels(self):
+        """Labels [B, D+1] int32 and margins [B, D+1] float32 of the last draft (device tensors)."""
+        t = self.torch
+        lab = self._empty((self.batch, self.D + 1), t.int32)
+        mg = self._empty((self.batch, self.D + 1), t.float32)
+        self._before()
+        self._check(fm_draft_labels(self.ctx, lab.data_ptr(), mg.data_ptr()), "fm_draft_labels")
+        self._after(lab, mg)
+        return lab, mg
 
     def verify(self, cand, want_logits=False, reuse=False):
         t = self.torch

@@ -63,6 +63,8 @@ struct fm_ctx {
   // draft
   bf16 *dh_a, *up_in_v, *up_in_f, *feat_n;
   float *dh_y, *feat, *dlogits;
+  float *label_g, *label_W, *label_margin;   // label head of the correction stage and its last results
+  int* labels;
   // attention scratch and TMA descriptors
   float* attn_part;
   int* attn_ticket;
@@ -142,6 +144,9 @@ int check_config(const fm_config* c) {
   if (c->d_model % 64 != 0 || c->d_ff % 64 != 0 || (c->n_heads * c->head_dim) % 128 != 0) return FM_ERR_UNSUPPORTED;
   if (c->head_dim != 64 && c->head_dim != 128) return FM_ERR_UNSUPPORTED;
   if (c->draft_len >= 7 && (c->draft_len + 8) / 9 + 1 > FM_MAX_FACE_HEADS) return FM_ERR_UNSUPPORTED;
+  if (c->draft_heads != FM_HEADS_REDUCED && c->draft_heads != FM_HEADS_FULL) return FM_ERR_INVALID_ARG;
+  if (c->draft_levels != FM_LEVELS_THREE && c->draft_levels != FM_LEVELS_COORD) return FM_ERR_INVALID_ARG;
+  if (c->hf_ff < 0 || c->hf_ff % 64 != 0) return FM_ERR_UNSUPPORTED;
   if (c->max_tokens < c->draft_len + 2) return FM_ERR_INVALID_ARG;
   return FM_OK;
 }
@@ -163,7 +168,15 @@ Dims make_dims(const fm_config& c) {
   dm.eps = c.norm_eps; dm.theta = c.rope_theta;
   // face head e drafts face f* + e - 1 (f* holds the pending token); offsets below 7 never leave
   // the next two points, a draft of D tokens reaches face f* + (8 + D) / 9
-  dm.Ef = dm.D >= 7 ? (dm.D + 8) / 9 + 1 : 1; dm.NH = 4 + dm.Ef;
+  const bool coord_only = c.draft_levels == FM_LEVELS_COORD;
+  dm.nc = coord_only ? (dm.D > 0 ? dm.D : 1) : 2;
+  dm.nv = coord_only ? 0 : 2;
+  dm.Ef = coord_only ? 0 : (dm.D >= 7 ? (dm.D + 8) / 9 + 1 : 1);
+  dm.NH = dm.nc + dm.nv + dm.Ef;
+  dm.full = c.draft_heads == FM_HEADS_FULL ? 1 : 0;
+  dm.avg = c.avg_levels != 0 ? 1 : 0;
+  dm.hf = c.hf_ff > 0 ? c.hf_ff : c.d_model;
+  dm.has_label = 0;                     // set by fm_create when the weights hold a label head
   return dm;
 }
 
@@ -229,12 +242,15 @@ void carve(fm_ctx* c, Carver& cv) {
   c->zc = cv.take<float>(B * FM_RING_C * d); c->zv = cv.take<float>(B * FM_RING_V * d);
   c->zf = cv.take<float>(B * FM_RING_F * d);
   // draft
-  const size_t NF = 8 + 9 * (size_t)dm.Ef;
+  const size_t NF = (size_t)dm.nc + 3 * dm.nv + 9 * (size_t)dm.Ef;
   c->dh_a = cv.take<bf16>(((size_t)dm.NH * B + 16) * d); c->dh_y = cv.take<float>((size_t)dm.NH * B * d);
-  c->up_in_v = cv.take<bf16>(align_up((2 + 3 * (size_t)dm.Ef) * B, 16) * d);
-  c->up_in_f = cv.take<bf16>(align_up((size_t)dm.Ef * B, 16) * d);
+  c->up_in_v = cv.take<bf16>(align_up((dm.nv + 3 * (size_t)dm.Ef) * B + 1, 16) * d);
+  c->up_in_f = cv.take<bf16>(align_up((size_t)dm.Ef * B + 1, 16) * d);
   c->feat = cv.take<float>(align_up(NF * B, 16) * d); c->feat_n = cv.take<bf16>(align_up(NF * B, 16) * d);
   c->dlogits = cv.take<float>(align_up(NF * B, 16) * dm.Vpad);
+  c->label_g = cv.take<float>(d); c->label_W = cv.take<float>(3 * d);
+  c->labels = cv.take<int>(B * dm.R1); c->label_margin = cv.take<float>(B * dm.R1);
+  c->st.hist = cv.take<int>(B * FM_HIST);
   // attention: chunk size, chunks per group (fixed per level so that the reduction order of a row
   // never depends on the cache length), group partials (max over levels), tickets
   c->attn_chunk = dm.dh == 64 ? 128 : 64;
@@ -675,7 +691,7 @@ void draft(fm_ctx* c, float* logits_out, float* margin_out, const GenOut* gen) {
   const int B = c->batch, d = dm.d;
   if (dm.D > 0) {
     const int dpad = round_up(d, 128);
-    const int NF = 8 + 9 * dm.Ef;
+    const int NF = dm.nc + 3 * dm.nv + 9 * dm.Ef, NP = dm.nv + 3 * dm.Ef;
     const int* na = c->st.n_active + 3;
     const size_t MB = dm.max_batch;
     LAUNCH(c, draft_prep_kernel, dim3(B, dm.NH), 256, 0, dm, c->st, B, c->zc, c->zv, c->zf, c->head_g, c->dh_a);
@@ -689,15 +705,19 @@ void draft(fm_ctx* c, float* logits_out, float* margin_out, const GenOut* gen) {
     }
     launch_pdl(c, dim3(1, 1, 1), draft_residual_kernel, dim3(B, dm.NH), 128, 0, dm, c->st, B, (const float*)c->zc, (const float*)c->zv,
                (const float*)c->zf, (const float*)c->dh_y, c->feat, c->up_in_v, c->up_in_f);
-    gemm(c, c->U_fv, pad128(3 * d), 0, c->up_in_f, align_up((size_t)dm.Ef * MB, 16), 0, 3 * d, d, dm.Ef * B, na, tc::EPI_BF16,
-         epi_plain(c->up_in_v + (size_t)2 * B * d, 3 * d));
-    gemm(c, c->U_vc, pad128(3 * d), 0, c->up_in_v, align_up((2 + 3 * (size_t)dm.Ef) * MB, 16), 0, 3 * d, d, (2 + 3 * dm.Ef) * B, na,
-         tc::EPI_F32, epi_plain(c->feat + (size_t)2 * B * d, 3 * d));
+    if (dm.Ef > 0)
+      gemm(c, c->U_fv, pad128(3 * d), 0, c->up_in_f, align_up((size_t)dm.Ef * MB + 1, 16), 0, 3 * d, d, dm.Ef * B, na, tc::EPI_BF16,
+           epi_plain(c->up_in_v + (size_t)dm.nv * B * d, 3 * d));
+    if (NP > 0)
+      gemm(c, c->U_vc, pad128(3 * d), 0, c->up_in_v, align_up((size_t)NP * MB + 1, 16), 0, 3 * d, d, NP * B, na,
+           tc::EPI_F32, epi_plain(c->feat + (size_t)dm.nc * B * d, 3 * d));
     launch_pdl(c, dim3(1, 1, 1), rmsnorm_kernel, NF * B, 256, 0, (const float*)c->feat, (const float*)c->g_out, c->feat_n, d, dm.eps);
     gemm(c, c->W_out, dm.Vpad, 0, c->feat_n, align_up((size_t)NF * MB, 16), 0, dm.V, d, NF * B, na, tc::EPI_F32,
          epi_plain(c->dlogits, dm.Vpad));
   }
-  launch_pdl(c, dim3(1, 1, 1), draft_pick_kernel, dim3(B, dm.R1), 256, 0, dm, c->st, B, (const float*)c->dlogits, logits_out, margin_out, gen);
+  const bool lab = dm.has_label != 0 && dm.D > 0;
+  launch_pdl(c, dim3(1, 1, 1), draft_pick_kernel, dim3(B, dm.R1), 256, 0, dm, c->st, B, (const float*)c->dlogits, logits_out, margin_out, gen,
+             (const bf16*)c->up_in_v, (const float*)c->label_g, (const float*)c->label_W, lab ? c->labels : (int*)nullptr, c->label_margin);
 }
 
 __global__ void verify_load_kernel(Dims dm, SeqState st, int batch, const int* __restrict__ cand) {
@@ -917,12 +937,17 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
   TRY(upload_packed(c->W_out, w->W_out, (size_t)dm.V, d, tmp));
   TRY(upload_f32(c->g_out, w->g_out, d));
   const size_t dpad = align_up(d, 128);
-  for (int h = 0; h < dm.NH; ++h) {
-    const float* A = h < 2 ? w->head_c_A[h] : h < 4 ? w->head_v_A[h - 2] : w->head_f_A[h - 4];
-    const float* g = h < 2 ? w->head_c_g[h] : h < 4 ? w->head_v_g[h - 2] : w->head_f_g[h - 4];
-    if (dm.D == 0 && (A == nullptr || g == nullptr)) continue;     // no drafts: heads are unused
-    TRY(upload_packed(c->headA + (size_t)h * dpad * d, A, d, d, tmp));
-    TRY(upload_f32(c->head_g + (size_t)h * d, g, d));
+  for (int h = 0; h < dm.NH && dm.D > 0; ++h) {
+    const fm_sp_weights* group = h < dm.nc ? w->heads_c : h < dm.nc + dm.nv ? w->heads_v : w->heads_f;
+    if (group == nullptr) { delete c; return FM_ERR_INVALID_ARG; }
+    const fm_sp_weights& sp = group[h < dm.nc ? h : h < dm.nc + dm.nv ? h - dm.nc : h - dm.nc - dm.nv];
+    TRY(upload_packed(c->headA + (size_t)h * dpad * d, sp.A, d, d, tmp));
+    TRY(upload_f32(c->head_g + (size_t)h * d, sp.g, d));
+  }
+  if (w->label_g != nullptr && w->label_W != nullptr && dm.nv > 0) {
+    TRY(upload_f32(c->label_g, w->label_g, d));
+    TRY(upload_f32(c->label_W, w->label_W, 3 * d));
+    c->dm.has_label = 1;
   }
   // TMA descriptors of the KV caches: each cache is a 2-D [max_batch*Hkv*slots, dh] bf16 matrix
   for (int s = 0; s < 5; ++s)
@@ -1147,13 +1172,33 @@ int fm_draft(fm_ctx* c, int32_t* cand, float* draft_logits, float* draft_margin)
   return FM_OK;
 }
 
-int fm_correct(fm_ctx* c, int32_t* cand, const int32_t* labels) {
-  if (c == nullptr || cand == nullptr || labels == nullptr) return FM_ERR_INVALID_ARG;
+int fm_correct_ex(fm_ctx* c, int32_t* cand, const int32_t* labels, int32_t use_history) {
+  if (c == nullptr || cand == nullptr) return FM_ERR_INVALID_ARG;
   if (c->phase < 1) return FM_ERR_BAD_STATE;
   if (c->dm.R1 > 3 * FM_CORRECT_MAX_POINTS) return FM_ERR_UNSUPPORTED;
-  LAUNCH(c, correct_kernel, (c->batch + 63) / 64, 64, 0, c->dm, c->st, c->batch, cand, labels);
+  if (labels == nullptr) {
+    if (!c->dm.has_label || c->dm.D == 0) return FM_ERR_UNSUPPORTED;
+    labels = c->labels;
+  }
+  LAUNCH(c, correct_kernel, (c->batch + 63) / 64, 64, 0, c->dm, c->st, c->batch, cand, labels, use_history != 0 ? 1 : 0);
   CUDA_OK(cudaGetLastError());
   if (c->launch_error != FM_OK) return c->launch_error;
+  return FM_OK;
+}
+
+int fm_correct(fm_ctx* c, int32_t* cand, const int32_t* labels) {
+  if (labels == nullptr) return FM_ERR_INVALID_ARG;
+  return fm_correct_ex(c, cand, labels, 0);
+}
+
+int fm_draft_labels(fm_ctx* c, int32_t* labels, float* margin) {
+  if (c == nullptr || labels == nullptr) return FM_ERR_INVALID_ARG;
+  if (c->phase < 1) return FM_ERR_BAD_STATE;
+  if (!c->dm.has_label || c->dm.D == 0) return FM_ERR_UNSUPPORTED;
+  const int n = c->batch * c->dm.R1;
+  LAUNCH(c, copy_i32_kernel, (n + 127) / 128, 128, 0, c->labels, labels, n);
+  if (margin != nullptr) LAUNCH(c, copy_f32_kernel, (n + 127) / 128, 128, 0, c->label_margin, margin, n);
+  CUDA_OK(cudaGetLastError());
   return FM_OK;
 }
 

@@ -13,6 +13,7 @@ typedef __nv_bfloat16 bf16;
 constexpr int FM_RING_C = 32;
 constexpr int FM_RING_V = 16;
 constexpr int FM_RING_F = 8;
+constexpr int FM_HIST = 32;             // the correction stage looks back at most two faces (18 tokens)
 
 struct Dims {
   int d, H, Hkv, dh, dff;
@@ -23,7 +24,10 @@ struct Dims {
   int max_batch, max_tokens;
   int allow_eos;
   float eps, theta;
-  int Ef, NH;                 // face heads, total draft heads (2 + 2 + Ef)
+  int Ef, NH;                 // face heads, total draft heads (nc + nv + Ef)
+  int nc, nv;                 // coordinate heads (2, or D when only the coordinate level drafts), vertex heads (2 or 0)
+  int full, avg, hf;          // full SP / HF blocks, averaged merge of the levels, width of the HF feed-forward
+  int has_label;              // a label head was given
 };
 
 // Per-sequence decoding state, all int32 arrays of max_batch entries in device memory.
@@ -40,6 +44,7 @@ struct SeqState {
   int* status;     // device status word
   int* n_active;   // sequences with nrow > 0 in the current pass
   int* step;       // passes executed by fm_generate (schedule index)
+  int* hist;       // [max_batch, FM_HIST] accepted mesh tokens, token t_i at entry i mod FM_HIST
 };
 
 __host__ __device__ inline int fm_ratio(int level) { return level == 0 ? 1 : (level == 1 ? 3 : 9); }

@@ -279,6 +279,7 @@ __device__ inline void accept_one(const Dims& dm, const SeqState& st, int b, int
     const unsigned em = __ballot_sync(0xffffffffu, lane < a && cand == eos);
     bool fin = false;
     if (em) { a = __ffs(em); fin = true; }           // an accepted EOS ends the sequence
+    if (lane < a) st.hist[b * FM_HIST + ((L - 1 + lane) & (FM_HIST - 1))] = cand;   // accepted token t_{L-1+lane}
     L += a;
     if (L - 1 >= st.t_end[b]) fin = true;
     if (gen != nullptr && gen->out_tok != nullptr && lane < a) {
@@ -356,6 +357,7 @@ __global__ void prefill_feed_kernel(Dims dm, SeqState st, int batch, const int* 
     int tok = dm.n_bins + 2;
     if (j < n) tok = pos == 0 ? dm.n_bins : prompt[prompt_off[b] + pos - 1];
     st.cand[b * dm.R1 + j] = tok;
+    if (j < n && pos >= 1) st.hist[b * FM_HIST + ((pos - 1) & (FM_HIST - 1))] = tok;            // input u_pos is mesh token t_{pos-1}
   }
   if (threadIdx.x == 0) st.nrow[b] = n;
 }
@@ -385,8 +387,16 @@ __global__ void arm_kernel(Dims dm, SeqState st, int batch) {
 // ------------------------------------------------------------------------------------------
 // a13. draft heads
 // ------------------------------------------------------------------------------------------
-// Head inputs.  Head index h: 0,1 coordinate; 2,3 vertex; 4.. face.  Row (h, b):
-// a[h][b] = bf16(rms(z) * g_h) with z the stashed split-node hidden of the pending position.
+// Split-node hidden that head h of sequence b reads.  Head index h: [0, nc) coordinate heads,
+// [nc, nc + nv) vertex heads, the rest face heads.
+__device__ inline const float* head_split_node(const Dims& dm, int h, int b, int n, const float* zc, const float* zv, const float* zf) {
+  return h < dm.nc ? zc + ((size_t)b * FM_RING_C + n % FM_RING_C) * dm.d
+       : h < dm.nc + dm.nv ? zv + ((size_t)b * FM_RING_V + (n / 3) % FM_RING_V) * dm.d
+                           : zf + ((size_t)b * FM_RING_F + (n / 9) % FM_RING_F) * dm.d;
+}
+
+// Head inputs.  Row (h, b): a[h][b] = bf16(rms(z) * g_h) with z the stashed split-node hidden of
+// the pending position.
 __global__ void draft_prep_kernel(Dims dm, SeqState st, int batch, const float* __restrict__ zc, const float* __restrict__ zv,
                                   const float* __restrict__ zf, const float* __restrict__ gains /*[NH,d]*/,
                                   bf16* __restrict__ a /*[NH, max_batch, d]*/) {
@@ -394,9 +404,7 @@ __global__ void draft_prep_kernel(Dims dm, SeqState st, int batch, const float* 
   const int h = blockIdx.y, b = blockIdx.x, d = dm.d;
   if (b >= batch) return;
   const int n = max(0, st.L[b] - 1);
-  const float* z = h < 2 ? zc + ((size_t)b * FM_RING_C + n % FM_RING_C) * d
-                 : h < 4 ? zv + ((size_t)b * FM_RING_V + (n / 3) % FM_RING_V) * d
-                         : zf + ((size_t)b * FM_RING_F + (n / 9) % FM_RING_F) * d;
+  const float* z = head_split_node(dm, h, b, n, zc, zv, zf);
   float ss = 0.f;
   for (int i = threadIdx.x; i < d; i += blockDim.x) ss += z[i] * z[i];
   ss = block_sum(ss, sh);
@@ -416,31 +424,40 @@ __global__ void draft_residual_kernel(Dims dm, SeqState st, int batch, const flo
   const int h = blockIdx.y, b = blockIdx.x, d = dm.d;
   if (b >= batch) return;
   const int n = max(0, st.L[b] - 1);
-  const float* z = h < 2 ? zc + ((size_t)b * FM_RING_C + n % FM_RING_C) * d
-                 : h < 4 ? zv + ((size_t)b * FM_RING_V + (n / 3) % FM_RING_V) * d
-                         : zf + ((size_t)b * FM_RING_F + (n / 9) % FM_RING_F) * d;
+  const float* z = head_split_node(dm, h, b, n, zc, zv, zf);
   const float* yr = y + ((size_t)h * dm.max_batch + b) * d;
   for (int i = threadIdx.x; i < d; i += blockDim.x) {
     const float v = z[i] + yr[i];
-    if (h < 2) feat[((size_t)h * batch + b) * d + i] = v;
-    else if (h < 4) up_in_v[((size_t)(h - 2) * batch + b) * d + i] = __float2bfloat16(v);
-    else up_in_f[((size_t)(h - 4) * batch + b) * d + i] = __float2bfloat16(v);
+    if (h < dm.nc) feat[((size_t)h * batch + b) * d + i] = v;
+    else if (h < dm.nc + dm.nv) up_in_v[((size_t)(h - dm.nc) * batch + b) * d + i] = __float2bfloat16(v);
+    else up_in_f[((size_t)(h - dm.nc - dm.nv) * batch + b) * d + i] = __float2bfloat16(v);
   }
 }
 
-// Feature row that serves draft offset j of sequence b (single source per offset; supplement,
-// "Optimizations"): offsets 1,2 -> coordinate heads (rule B); targets in the next two vertices
-// v*+1, v*+2 -> vertex head floor(p/3) - v*, wherever the face boundary lies, except where the
-// latest vertex row was also a face row (v* % 3 == 0): there the face level keeps the rest of
-// its own face (rule A), face head 1; targets beyond two vertices -> face head
-// floor(p/9) - f* + 1 (head e drafts face f* + e - 1).
-__device__ inline int draft_feature_row(int n, int j, int b, int B) {
+// Source of draft offset j (single source per offset; supplement, "Optimizations"): offsets 1,2
+// -> coordinate heads (rule B); targets in the next two vertices v*+1, v*+2 -> vertex head
+// floor(p/3) - v*, wherever the face boundary lies, except where the latest vertex row was also a
+// face row (v* % 3 == 0): there the face level keeps the rest of its own face (rule A), face head
+// 1; targets beyond two vertices -> face head floor(p/9) - f* + 1 (head e drafts face f* + e - 1).
+// With only the coordinate level drafting, coordinate head j serves offset j.
+// level 0: head = j; level 1: head = e (1, 2), slot = p % 3; level 2: head = e, slot = p % 9.
+__device__ inline void draft_source(const Dims& dm, int n, int j, int& level, int& head, int& slot) {
   const int p = n + j;
-  if (j <= 2) return (j - 1) * B + b;
+  if (j <= 2 || dm.nv == 0) { level = 0; head = j; slot = 0; return; }
   const int ev = p / 3 - n / 3;
-  if (ev <= 2 && !((n / 3) % 3 == 0 && p / 9 == n / 9)) return 2 * B + 3 * ((ev - 1) * B + b) + p % 3;
-  const int e = p / 9 - n / 9 + 1, s = p % 9;
-  return 2 * B + 3 * (2 * B + 3 * ((e - 1) * B + b) + s / 3) + s % 3;
+  if (ev <= 2 && !((n / 3) % 3 == 0 && p / 9 == n / 9)) { level = 1; head = ev; slot = p % 3; return; }
+  level = 2; head = p / 9 - n / 9 + 1; slot = p % 9;
+}
+// row of the coordinate-level feature matrix [NF*B, d] that holds the feature of (level, head, slot)
+__device__ inline int draft_feature_row(const Dims& dm, int level, int head, int slot, int b, int B) {
+  if (level == 0) return (head - 1) * B + b;
+  if (level == 1) return dm.nc * B + 3 * ((head - 1) * B + b) + slot;
+  return dm.nc * B + 3 * (dm.nv * B + 3 * ((head - 1) * B + b) + slot / 3) + slot % 3;
+}
+// row of the point-level feature matrix [(nv + 3 Ef)*B, d] (the upsample GEMM's operand rows) behind it
+__device__ inline int draft_point_row(const Dims& dm, int level, int head, int slot, int b, int B) {
+  if (level == 1) return (head - 1) * B + b;
+  return dm.nv * B + 3 * ((head - 1) * B + b) + slot / 3;
 }
 
 // masked argmax of the chosen feature's logits -> cand[b][j]; cand[b][0] = pending main token
@@ -449,12 +466,45 @@ __device__ inline int draft_feature_row(int n, int j, int b, int B) {
 // different coordinate id.
 __global__ void draft_pick_kernel(Dims dm, SeqState st, int batch, const float* __restrict__ logits /*[NF*B, Vpad]*/,
                                   float* __restrict__ logits_out, float* __restrict__ margin_out,
-                                  const GenOut* __restrict__ gen) {
+                                  const GenOut* __restrict__ gen, const bf16* __restrict__ point_feat /*[(nv+3Ef)*B, d]*/,
+                                  const float* __restrict__ label_g, const float* __restrict__ label_W,
+                                  int* __restrict__ labels /*[B, R1]*/, float* __restrict__ label_margin) {
   ptx::grid_dep_launch();
   ptx::grid_dep_wait();
   const int b = blockIdx.x, j = blockIdx.y;        // j = 0..D
   if (b >= batch) return;
   const bool fin = st.done[b] != 0 || st.nrow[b] <= 0;
+  const int n = st.L[b] - 1;
+  // ---- label of the point that starts at slot j (Sec. 3.2): a vertex whose three tokens are drafts
+  if (labels != nullptr) {
+    const bool starts = !fin && j >= 1 && j + 2 <= dm.D && (n + j) % 3 == 0 && dm.nv > 0;
+    if (!starts) {
+      if (threadIdx.x == 0) { labels[b * dm.R1 + j] = -1; label_margin[b * dm.R1 + j] = 0.f; }
+    } else {
+      __shared__ float shl[32];
+      int level, head, slot;
+      draft_source(dm, n, j + 2, level, head, slot);        // the head that drafts the point's last coordinate
+      const bf16* f = point_feat + (size_t)draft_point_row(dm, level, head, slot, b, batch) * dm.d;
+      float ss = 0.f, z0 = 0.f, z1 = 0.f, z2 = 0.f;
+      for (int i = threadIdx.x; i < dm.d; i += blockDim.x) {
+        const float v = __bfloat162float(f[i]), vg = v * label_g[i];
+        ss += v * v;
+        z0 += label_W[i] * vg; z1 += label_W[dm.d + i] * vg; z2 += label_W[2 * dm.d + i] * vg;
+      }
+      ss = block_sum(ss, shl); z0 = block_sum(z0, shl); z1 = block_sum(z1, shl); z2 = block_sum(z2, shl);
+      if (threadIdx.x == 0) {
+        const float inv = rsqrtf(ss / (float)dm.d + dm.eps);
+        z0 *= inv; z1 *= inv; z2 *= inv;
+        int best = 0; float top = z0;
+        if (z1 > top) { best = 1; top = z1; }
+        if (z2 > top) { best = 2; top = z2; }
+        const float second = best == 0 ? fmaxf(z1, z2) : (best == 1 ? fmaxf(z0, z2) : fmaxf(z0, z1));
+        labels[b * dm.R1 + j] = best;
+        label_margin[b * dm.R1 + j] = top - second;
+      }
+      __syncthreads();
+    }
+  }
   if (j == 0) {
     if (threadIdx.x == 0) st.cand[b * dm.R1] = fin ? dm.n_bins + 2 : st.main_tok[b];
     return;
@@ -465,8 +515,9 @@ __global__ void draft_pick_kernel(Dims dm, SeqState st, int batch, const float* 
       for (int i = threadIdx.x; i < dm.V; i += blockDim.x) logits_out[((size_t)b * dm.D + j - 1) * dm.V + i] = 0.f;
     return;
   }
-  const int n = st.L[b] - 1;
-  const float* z = logits + (size_t)draft_feature_row(n, j, b, batch) * dm.Vpad;
+  int level, head, slot;
+  draft_source(dm, n, j, level, head, slot);
+  const float* z = logits + (size_t)draft_feature_row(dm, level, head, slot, b, batch) * dm.Vpad;
   if (logits_out)
     for (int i = threadIdx.x; i < dm.V; i += blockDim.x) logits_out[((size_t)b * dm.D + j - 1) * dm.V + i] = z[i];
   const Top2 t = block_top2(z, dm, n + j);
@@ -522,7 +573,8 @@ __device__ inline bool vertex_less(const int* a, const int* b) {       // (z, y,
   return a[2] < b[2];
 }
 
-__global__ void correct_kernel(Dims dm, SeqState st, int batch, int* __restrict__ cand, const int* __restrict__ labels) {
+__global__ void correct_kernel(Dims dm, SeqState st, int batch, int* __restrict__ cand, const int* __restrict__ labels,
+                               int use_history) {
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= batch) return;
   const int n = st.nrow[b];
@@ -542,6 +594,31 @@ __global__ void correct_kernel(Dims dm, SeqState st, int batch, int* __restrict_
     usable[m] = row[s] >= 0 && row[s] < dm.n_bins && row[s + 1] >= 0 && row[s + 1] < dm.n_bins && row[s + 2] >= 0 &&
                 row[s + 2] < dm.n_bins;
     ++m;
+  }
+  // historical points against the accepted vertices: the complete ones of the face that holds the
+  // main token and of the face before it (at most five), oldest first; a point that equals none of
+  // them becomes the nearest (ties to the earliest)
+  if (use_history) {
+    int win[5][3], nw = 0;
+    const int* h = st.hist + (size_t)b * FM_HIST;
+    const int fprev = first / 9 - 1;
+    for (int v = fprev > 0 ? 3 * fprev : 0; v < first / 3 && nw < 5; ++v) {
+      const int t0 = h[(3 * v) & (FM_HIST - 1)], t1 = h[(3 * v + 1) & (FM_HIST - 1)], t2 = h[(3 * v + 2) & (FM_HIST - 1)];
+      if (t0 < 0 || t0 >= dm.n_bins || t1 < 0 || t1 >= dm.n_bins || t2 < 0 || t2 >= dm.n_bins) continue;
+      win[nw][0] = t0; win[nw][1] = t1; win[nw][2] = t2; ++nw;
+    }
+    for (int k = 0; k < m && nw > 0; ++k) {
+      if (kind[k] != 0 || !usable[k]) continue;
+      const int z = row[slot[k]], y = row[slot[k] + 1], x = row[slot[k] + 2];
+      int src = -1;
+      long long best = 0;
+      for (int q = 0; q < nw; ++q) {
+        const long long dz = win[q][0] - z, dy = win[q][1] - y, dx = win[q][2] - x;
+        const long long dist = dz * dz + dy * dy + dx * dx;
+        if (src < 0 || dist < best) { src = q; best = dist; }
+      }
+      if (best != 0) { row[slot[k]] = win[src][0]; row[slot[k] + 1] = win[src][1]; row[slot[k] + 2] = win[src][2]; }
+    }
   }
   // intra-batch points in sequence order; each sees the corrections before it
   for (int k = 0; k < m; ++k) {

@@ -24,7 +24,8 @@ def test_correct_matches_oracle_at_every_phase(D):
     dev.prefill(np.stack(conds), prompts)
     rng = np.random.default_rng(D)
     L = np.array([1 + len(p) for p in prompts])
-    checked = 0
+    hist = [list(p) for p in prompts]                # accepted mesh tokens t_0 .. t_{L-2} per sequence
+    checked = moved = 0
     phases = set()
     for step in range(14):
         phases |= {int(x) % 9 for x in L}
@@ -39,17 +40,32 @@ def test_correct_matches_oracle_at_every_phase(D):
         d_rows = torch.as_tensor(rows).cuda()
         d_lab = torch.as_tensor(labels).cuda()
         out = dev.correct(d_rows, d_lab).cpu().numpy()
+        out_h = dev.correct(torch.as_tensor(rows).cuda(), d_lab, use_history=True).cpu().numpy()
+        # ... and with the label head's own labels (compared with the oracle's in the lock-step tests)
+        own = dev.draft_labels()[0]
+        out_own = dev.correct(torch.as_tensor(rows).cuda(), None, use_history=True).cpu().numpy()
+        own = own.cpu().numpy()
         for b in range(B):
+            assert len(hist[b]) == int(L[b]) - 1
             want = correct_row(rows[b].tolist(), labels[b].tolist(), int(L[b]), cfg.n_bins)
             assert out[b].tolist() == want, (step, b, int(L[b]), rows[b].tolist(), labels[b].tolist())
+            want_h = correct_row(rows[b].tolist(), labels[b].tolist(), int(L[b]), cfg.n_bins, history=hist[b])
+            assert out_h[b].tolist() == want_h, (step, b, int(L[b]), rows[b].tolist(), labels[b].tolist(), hist[b][-18:])
+            want_own = correct_row(rows[b].tolist(), own[b].tolist(), int(L[b]), cfg.n_bins, history=hist[b])
+            assert out_own[b].tolist() == want_own
+            moved += int(want_h != want)
             checked += 1
         # move every sequence on by a different number of tokens: all nine phases get visited
         dev.verify(cand)
         force = np.array([1 + (step + b) % min(D + 1, 4) for b in range(B)], dtype=np.int32)
-        n_acc, _, kv = dev.accept(force_len=force)
+        n_acc, em, kv = dev.accept(force_len=force)
+        em, n_acc = em.cpu().numpy(), n_acc.cpu().numpy()
+        for b in range(B):
+            hist[b] += [int(t) for t in em[b, :n_acc[b]]]
         L = kv.cpu().numpy()[:, 0]
     assert checked == 14 * B
     assert phases == set(range(9))                   # the rows started at every coordinate of the face
+    assert moved > 0                                 # the historical rule did change rows
     assert dev.device_status() == 0
 
 

@@ -49,7 +49,21 @@ def test_toy_lockstep_all_draft_lengths(D):
     rep = run_lockstep(cfg, w, conds, prompts, dev, [6, 5], 200, tol=TOY_TOL, margin=TOY_MARGIN)
     assert rep["done"] and rep["emitted"] == 9 * 11
     assert dev.device_status() == 0
-    print(D, {k: rep[k] for k in ("steps", "max_logit_err", "max_draft_err", "overrides", "low_margin_rows", "rows")})
+    assert D < 5 or rep["labels"] > 0                 # the label head's labels were compared as well
+    print(D, {k: rep[k] for k in ("steps", "max_logit_err", "max_draft_err", "overrides", "low_margin_rows", "rows", "labels", "label_flips")})
+
+
+@pytest.mark.parametrize("D", [9, 18])
+def test_toy_coordinate_only_drafting_lockstep(D):
+    """The supplement's ablation variant: D coordinate heads, no point- or face-level modules."""
+    from oracle.lockstep import run_lockstep
+    cfg = S.toy_config(**TOY, draft_len=D, draft_levels="coord", layers=(1, 2, 2, 1, 2), max_batch=2, prompt_faces=(1, 1), gen_faces=6)
+    cfg = cfg.with_(max_tokens=1 + 9 * 8 + D + 2)
+    w, conds, prompts = _setup(cfg, batch=2)
+    dev = _dev(cfg, w)
+    rep = run_lockstep(cfg, w, conds, prompts, dev, [6, 5], 200, tol=TOY_TOL, margin=TOY_MARGIN)
+    assert rep["done"] and rep["emitted"] == 9 * 11 and dev.device_status() == 0
+    print(D, {k: rep[k] for k in ("steps", "max_logit_err", "max_draft_err", "overrides")})
 
 
 def test_toy_lockstep_windows_and_mqa_and_eos():
