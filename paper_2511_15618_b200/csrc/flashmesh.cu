@@ -24,6 +24,7 @@ namespace {
 
 constexpr int STACK_LEVEL[5] = {0, 1, 2, 1, 0};
 constexpr int PREFILL_CHUNK = 256;      // conditioning rows projected per launch group
+constexpr int FM_ROPE_SLACK = 64;       // the HF-Blocks of the face level query positions up to 4 faces ahead
 
 struct LayerDev {
   bf16 *Wqkv, *Wo, *W1, *W2;
@@ -65,6 +66,15 @@ struct fm_ctx {
   float *dh_y, *feat, *dlogits;
   float *label_g, *label_W, *label_margin;   // label head of the correction stage and its last results
   int* labels;
+  float* avg_rows;                           // [B*R1, Vpad] rows of the averaged merge
+  // full draft modules: SP-Block attention (per head) and HF-Blocks (per offset), stacked per stage
+  bf16 *spWq, *spWo; float* sp_ga;
+  bf16 *hfWq[2], *hfW1[2], *hfW2[2]; float* hf_g[2];       // [0] vertex-level blocks (3 Ef), [1] coordinate-level blocks (3 nv + 9 Ef)
+  int hf_T[2];
+  float *d_qf, *d_out, *xv_pre;              // projections' fp32 results [sets*max_batch, .], face level's upsampled triples
+  bf16 *d_q, *d_attn, *d_a, *d_h1;           // rotated queries, attention output [hi | lo], block inputs, FFN hidden [hi | lo]
+  int draft_sets;                            // rows reserved per stage: max number of sets
+  int attn_mt_draft[3];                      // query tiles of the draft modules' attention launches per level
   // attention scratch and TMA descriptors
   float* attn_part;
   int* attn_ticket;
@@ -220,7 +230,7 @@ void carve(fm_ctx* c, Carver& cv) {
   c->g_out = cv.take<float>(d);
   c->head_g = cv.take<float>((size_t)dm.NH * d);
   c->inv_freq = cv.take<double>(dm.dh / 2);
-  c->rope_tab = cv.take<float2>((size_t)(dm.max_tokens + 1) * (dm.dh / 2));
+  c->rope_tab = cv.take<float2>((size_t)(dm.max_tokens + 1 + FM_ROPE_SLACK) * (dm.dh / 2));
   // state
   c->st.L = cv.take<int>(B); c->st.nrow = cv.take<int>(B); c->st.main_tok = cv.take<int>(B);
   c->st.done = cv.take<int>(B); c->st.t_end = cv.take<int>(B); c->st.plen = cv.take<int>(B);
@@ -251,6 +261,24 @@ void carve(fm_ctx* c, Carver& cv) {
   c->label_g = cv.take<float>(d); c->label_W = cv.take<float>(3 * d);
   c->labels = cv.take<int>(B * dm.R1); c->label_margin = cv.take<float>(B * dm.R1);
   c->st.hist = cv.take<int>(B * FM_HIST);
+  c->avg_rows = dm.avg ? cv.take<float>(B * dm.R1 * (size_t)dm.Vpad) : nullptr;
+  c->hf_T[0] = 3 * dm.Ef; c->hf_T[1] = 3 * dm.nv + 9 * dm.Ef;
+  c->draft_sets = dm.NH > c->hf_T[1] ? dm.NH : c->hf_T[1];
+  if (dm.full) {
+    const size_t hdp = align_up(hd, 128), dp = align_up(d, 128), hfp = align_up((size_t)dm.hf, 128), S = c->draft_sets;
+    c->spWq = cv.take<bf16>((size_t)dm.NH * hdp * d); c->spWo = cv.take<bf16>((size_t)dm.NH * dp * hd);
+    c->sp_ga = cv.take<float>((size_t)dm.NH * d);
+    for (int k = 0; k < 2; ++k) {
+      const size_t T = c->hf_T[k] > 0 ? c->hf_T[k] : 1;
+      c->hfWq[k] = cv.take<bf16>(T * hdp * d); c->hfW1[k] = cv.take<bf16>(T * hfp * hd); c->hfW2[k] = cv.take<bf16>(T * dp * dm.hf);
+      c->hf_g[k] = cv.take<float>(T * d);
+    }
+    const size_t rows = S * B + 16;
+    c->d_qf = cv.take<float>(rows * hd); c->d_out = cv.take<float>(rows * d);
+    c->xv_pre = cv.take<float>(((size_t)dm.Ef * B + 16) * 3 * d);
+    c->d_q = cv.take<bf16>(rows * hd); c->d_attn = cv.take<bf16>(rows * 2 * hd); c->d_a = cv.take<bf16>(rows * d);
+    c->d_h1 = cv.take<bf16>(rows * 2 * dm.hf);
+  }
   // attention: chunk size, chunks per group (fixed per level so that the reduction order of a row
   // never depends on the cache length), group partials (max over levels), tickets
   c->attn_chunk = dm.dh == 64 ? 128 : 64;
@@ -258,13 +286,17 @@ void carve(fm_ctx* c, Carver& cv) {
   for (int l = 0; l < 3; ++l) {
     const int max_chunks = (dm.P + dm.cap[l] + c->attn_chunk - 1) / c->attn_chunk;
     c->attn_mt[l] = (fm_rows_per_seq(dm, l) * (dm.H / dm.Hkv) + 15) / 16;
+    // query rows of the draft modules at this level: SP heads and HF offsets, whichever launch has more
+    const int dq = !dm.full ? 0 : (l == 0 ? (dm.nc > 3 * dm.nv + 9 * dm.Ef ? dm.nc : 3 * dm.nv + 9 * dm.Ef) : (l == 1 ? (dm.nv > 3 * dm.Ef ? dm.nv : 3 * dm.Ef) : dm.Ef));
+    c->attn_mt_draft[l] = (dq * (dm.H / dm.Hkv) + 15) / 16;
+    const int mt_max = c->attn_mt[l] > c->attn_mt_draft[l] ? c->attn_mt[l] : c->attn_mt_draft[l];
     // Chunks per group: the number of groups (1 .. what the merge can stage: 24, fewer for wide
     // heads) that minimises waves x (chunks per CTA + a CTA's fixed cost), with the cache full.
     // The fixed cost (pipeline start, merge of the warps, and with several groups the partials,
     // the ticket and the last CTA's merge) was measured at batch 16 as about 5 chunk times:
     // 87 / 70 / 63 / 61 us per launch with at most 8 / 16 / 32 / 64 chunks per group.
     const int g_cap = dm.dh == 64 ? AttnCfg<64, 128, 8>::MAX_GROUPS : AttnCfg<128, 64, 4>::MAX_GROUPS;
-    const size_t tiles_l = (size_t)dm.Hkv * B * c->attn_mt[l];
+    const size_t tiles_l = (size_t)dm.Hkv * B * c->attn_mt[l];      // the verify pass decides the grouping
     int G = max_chunks;
     double best = 0.0;
     for (int ng = 1; ng <= g_cap && ng <= max_chunks; ++ng) {
@@ -280,9 +312,9 @@ void carve(fm_ctx* c, Carver& cv) {
     }
     c->attn_G[l] = G;
     c->attn_max_groups[l] = (max_chunks + G - 1) / G;
-    const size_t need = B * dm.Hkv * (size_t)c->attn_mt[l] * c->attn_max_groups[l] * 16 * (dm.dh + 2);
+    const size_t need = B * dm.Hkv * (size_t)mt_max * c->attn_max_groups[l] * 16 * (dm.dh + 2);
     part_max = need > part_max ? need : part_max;
-    const size_t tk = B * dm.Hkv * (size_t)c->attn_mt[l];
+    const size_t tk = B * dm.Hkv * (size_t)mt_max;
     ticket_max = tk > ticket_max ? tk : ticket_max;
   }
   c->attn_part = cv.take<float>(part_max);
@@ -685,16 +717,100 @@ void forward(fm_ctx* c, float* logits_out) {
   launch_pdl(c, dim3(1, 1, 1), verify_top2_kernel, Rc, 256, 0, dm, c->st, B, (const float*)c->logits, logits_out);
 }
 
-// a13: draft heads on the stashed split-node hiddens
+// T problems of the same shape in one launch (grid.z): set t multiplies weight matrix t of the stacked
+// buffer W (Mpad rows each) with operand rows [t*max_batch, t*max_batch + batch) and writes the same
+// rows of the output.  More than 32 sequences: one launch per set.
+void gemm_sets(fm_ctx* c, const bf16* W, int Mpad, int M, int K, const bf16* A, int a_parts, int T, int mode, tc::Epi e) {
+  const Dims& dm = c->dm;
+  const int B = c->batch, MB = dm.max_batch;
+  const size_t a_rows = (size_t)c->draft_sets * MB + 16;
+  const int* na = c->st.n_active + 3;
+  const size_t esz = (mode == tc::EPI_F32) ? 4 : 2;
+  if (T <= 0) return;
+  if (B <= 32) {
+    gemm(c, W, (size_t)T * Mpad, 0, A, a_rows, 0, M, K, B, na, mode, e, a_parts, T, MB, Mpad);
+    return;
+  }
+  for (int t = 0; t < T; ++t) {
+    tc::Epi et = e;
+    et.out = static_cast<char*>(e.out) + (size_t)t * MB * e.ldo * esz;
+    gemm(c, W, (size_t)T * Mpad, t * Mpad, A, a_rows, t * MB, M, K, B, na, mode, et, a_parts);
+  }
+}
+
+// attention of nq draft queries per sequence over the cache of the last layer of stack s; the
+// result of query r of sequence b goes to row r * max_batch + b of `out`
+void attention_draft(fm_ctx* c, int s, int nq, const bf16* q, bf16* out) {
+  const Dims& dm = c->dm;
+  const int level = STACK_LEVEL[s];
+  const LayerDev& L = c->layers[s].back();
+  const int groups = c->attn_max_groups[level];
+  const int MT = (nq * (dm.H / dm.Hkv) + 15) / 16;
+  if (MT > c->attn_mt_draft[level] && MT > c->attn_mt[level]) { c->launch_error = FM_ERR_CAPACITY; return; }
+  AttnArgs a{dm, c->st, c->batch, level, q, c->tmaps + L.tmK, c->tmaps + L.tmV, c->attn_part, c->attn_ticket,
+             out, c->attn_G[level], groups, MT, nq, dm.max_batch};
+  const dim3 grid(groups, dm.Hkv * MT, c->batch);
+  c->cur_class = PROF_ATTN;
+  if (dm.dh == 64) launch_pdl(c, dim3(1, 1, 1), attn_stream_kernel<64, 128, 8>, grid, AttnCfg<64, 128, 8>::THREADS, AttnCfg<64, 128, 8>::BYTES, a);
+  else launch_pdl(c, dim3(1, 1, 1), attn_stream_kernel<128, 64, 4>, grid, AttnCfg<128, 64, 4>::THREADS, AttnCfg<128, 64, 4>::BYTES, a);
+  c->cur_class = PROF_OTHER;
+}
+
+// One stage of HF-Blocks (Eq. 3-5) on the fp32 features hf_feature() names: T offsets, each with its
+// own W_q, FFN and gain; k = 0: vertex level (cache of the vertex-up stack), 1: coordinate level.
+void hf_stage(fm_ctx* c, int k) {
+  const Dims& dm = c->dm;
+  const int B = c->batch, d = dm.d, hd = dm.H * dm.dh, T = c->hf_T[k];
+  if (T <= 0) return;
+  const int stage = k == 0 ? DS_HF_V : DS_HF_C, s = k == 0 ? 3 : 4;
+  const int hdp = round_up(hd, 128), dp = round_up(d, 128), hfp = round_up(dm.hf, 128);
+  const float qscale = (float)(1.4426950408889634 / sqrt((double)dm.dh));
+  launch_pdl(c, dim3(1, 1, 1), hf_prep_kernel, dim3(B, T), 256, 0, dm, c->st, B, stage, c->xv_pre, c->feat, (const float*)c->hf_g[k], c->d_a);
+  gemm_sets(c, c->hfWq[k], hdp, hd, d, c->d_a, 1, T, tc::EPI_F32, epi_plain(c->d_qf, hd));
+  launch_pdl(c, dim3(1, 1, 1), draft_q_kernel, dim3(B, T), 256, 0, dm, c->st, B, stage, STACK_LEVEL[s], 0, T, (const float*)c->d_qf,
+             (const float2*)c->rope_tab, qscale, c->d_q);
+  attention_draft(c, s, T, c->d_q, c->d_attn);
+  tc::Epi e1 = epi_plain(c->d_h1, 2 * dm.hf);
+  e1.lo_off = dm.hf;
+  gemm_sets(c, c->hfW1[k], hfp, dm.hf, hd, c->d_attn, 2, T, tc::EPI_GELU, e1);
+  gemm_sets(c, c->hfW2[k], dp, d, dm.hf, c->d_h1, 2, T, tc::EPI_F32, epi_plain(c->d_out, d));
+  launch_pdl(c, dim3(1, 1, 1), hf_finish_kernel, dim3(B, T), 256, 0, dm, c->st, B, stage, c->xv_pre, c->feat, (const float*)c->d_out, c->up_in_v);
+}
+
+// a13: draft modules on the stashed split-node hiddens.  Reduced heads: SP = h + A rms(h), the
+// upsample matrices alone.  Full: the SP-Blocks' attention before the linear layer and an HF-Block
+// after every upsample (Sec. 3.1, Eq. 1-5; supplement "Three-Level Speculative Decoding").
 void draft(fm_ctx* c, float* logits_out, float* margin_out, const GenOut* gen) {
   const Dims& dm = c->dm;
   const int B = c->batch, d = dm.d;
   if (dm.D > 0) {
-    const int dpad = round_up(d, 128);
+    const int dpad = round_up(d, 128), hd = dm.H * dm.dh;
     const int NF = dm.nc + 3 * dm.nv + 9 * dm.Ef, NP = dm.nv + 3 * dm.Ef;
     const int* na = c->st.n_active + 3;
     const size_t MB = dm.max_batch;
-    LAUNCH(c, draft_prep_kernel, dim3(B, dm.NH), 256, 0, dm, c->st, B, c->zc, c->zv, c->zf, c->head_g, c->dh_a);
+    if (dm.full) {
+      // SP-Block attention: a = rms(z, ga); q = Wq a at the split node's position; o over the cache of
+      // the level's last layer; u = Wo o; then the head's input is rms(z + u, g) instead of rms(z, g)
+      const float qscale = (float)(1.4426950408889634 / sqrt((double)dm.dh));
+      LAUNCH(c, draft_prep_kernel, dim3(B, dm.NH), 256, 0, dm, c->st, B, c->zc, c->zv, c->zf, c->sp_ga, c->d_a);
+      gemm_sets(c, c->spWq, round_up(hd, 128), hd, d, c->d_a, 1, dm.NH, tc::EPI_F32, epi_plain(c->d_qf, hd));
+      const int cnt[3] = {dm.nc, dm.nv, dm.Ef}, stack_of[3] = {4, 3, 2};
+      int h0 = 0;
+      for (int l = 0; l < 3; ++l) {
+        if (cnt[l] > 0) {
+          bf16* ql = c->d_q + (size_t)h0 * MB * hd;           // this level's queries, rows (b * cnt + r)
+          launch_pdl(c, dim3(1, 1, 1), draft_q_kernel, dim3(B, cnt[l]), 256, 0, dm, c->st, B, (int)DS_SP, l, h0, cnt[l], (const float*)c->d_qf,
+                     (const float2*)c->rope_tab, qscale, ql);
+          attention_draft(c, stack_of[l], cnt[l], ql, c->d_attn + (size_t)h0 * MB * 2 * hd);
+        }
+        h0 += cnt[l];
+      }
+      gemm_sets(c, c->spWo, dpad, d, hd, c->d_attn, 2, dm.NH, tc::EPI_F32, epi_plain(c->d_out, d));
+      launch_pdl(c, dim3(1, 1, 1), sp_mid_kernel, dim3(B, dm.NH), 256, 0, dm, c->st, B, (const float*)c->zc, (const float*)c->zv,
+                 (const float*)c->zf, (const float*)c->d_out, (const float*)c->head_g, c->dh_a);
+    } else {
+      LAUNCH(c, draft_prep_kernel, dim3(B, dm.NH), 256, 0, dm, c->st, B, c->zc, c->zv, c->zf, c->head_g, c->dh_a);
+    }
     if (B <= 32) {                                               // the NH head matrices as one launch
       gemm(c, c->headA, (size_t)dm.NH * dpad, 0, c->dh_a, (size_t)dm.NH * MB + 16, 0, d, d, B, na, tc::EPI_F32, epi_plain(c->dh_y, d), 1,
            dm.NH, (int)MB, dpad);
@@ -705,19 +821,29 @@ void draft(fm_ctx* c, float* logits_out, float* margin_out, const GenOut* gen) {
     }
     launch_pdl(c, dim3(1, 1, 1), draft_residual_kernel, dim3(B, dm.NH), 128, 0, dm, c->st, B, (const float*)c->zc, (const float*)c->zv,
                (const float*)c->zf, (const float*)c->dh_y, c->feat, c->up_in_v, c->up_in_f);
-    if (dm.Ef > 0)
-      gemm(c, c->U_fv, pad128(3 * d), 0, c->up_in_f, align_up((size_t)dm.Ef * MB + 1, 16), 0, 3 * d, d, dm.Ef * B, na, tc::EPI_BF16,
-           epi_plain(c->up_in_v + (size_t)dm.nv * B * d, 3 * d));
-    if (NP > 0)
+    if (dm.Ef > 0) {
+      if (dm.full) {                                             // face -> 3 vertices, each refined at the vertex level
+        gemm(c, c->U_fv, pad128(3 * d), 0, c->up_in_f, align_up((size_t)dm.Ef * MB + 1, 16), 0, 3 * d, d, dm.Ef * B, na, tc::EPI_F32,
+             epi_plain(c->xv_pre, 3 * d));
+        hf_stage(c, 0);
+      } else {
+        gemm(c, c->U_fv, pad128(3 * d), 0, c->up_in_f, align_up((size_t)dm.Ef * MB + 1, 16), 0, 3 * d, d, dm.Ef * B, na, tc::EPI_BF16,
+             epi_plain(c->up_in_v + (size_t)dm.nv * B * d, 3 * d));
+      }
+    }
+    if (NP > 0) {
       gemm(c, c->U_vc, pad128(3 * d), 0, c->up_in_v, align_up((size_t)NP * MB + 1, 16), 0, 3 * d, d, NP * B, na,
            tc::EPI_F32, epi_plain(c->feat + (size_t)dm.nc * B * d, 3 * d));
+      if (dm.full) hf_stage(c, 1);                               // every upsampled coordinate feature refined at the coordinate level
+    }
     launch_pdl(c, dim3(1, 1, 1), rmsnorm_kernel, NF * B, 256, 0, (const float*)c->feat, (const float*)c->g_out, c->feat_n, d, dm.eps);
     gemm(c, c->W_out, dm.Vpad, 0, c->feat_n, align_up((size_t)NF * MB, 16), 0, dm.V, d, NF * B, na, tc::EPI_F32,
          epi_plain(c->dlogits, dm.Vpad));
   }
   const bool lab = dm.has_label != 0 && dm.D > 0;
   launch_pdl(c, dim3(1, 1, 1), draft_pick_kernel, dim3(B, dm.R1), 256, 0, dm, c->st, B, (const float*)c->dlogits, logits_out, margin_out, gen,
-             (const bf16*)c->up_in_v, (const float*)c->label_g, (const float*)c->label_W, lab ? c->labels : (int*)nullptr, c->label_margin);
+             (const bf16*)c->up_in_v, (const float*)c->label_g, (const float*)c->label_W, lab ? c->labels : (int*)nullptr, c->label_margin,
+             c->avg_rows);
 }
 
 __global__ void verify_load_kernel(Dims dm, SeqState st, int batch, const int* __restrict__ cand) {
@@ -944,6 +1070,26 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
     TRY(upload_packed(c->headA + (size_t)h * dpad * d, sp.A, d, d, tmp));
     TRY(upload_f32(c->head_g + (size_t)h * d, sp.g, d));
   }
+  if (dm.full && dm.D > 0) {
+    const size_t hdp = align_up(hd, 128), hfp = align_up((size_t)dm.hf, 128);
+    for (int h = 0; h < dm.NH; ++h) {
+      const fm_sp_weights* group = h < dm.nc ? w->heads_c : h < dm.nc + dm.nv ? w->heads_v : w->heads_f;
+      const fm_sp_weights& sp = group[h < dm.nc ? h : h < dm.nc + dm.nv ? h - dm.nc : h - dm.nc - dm.nv];
+      TRY(upload_packed(c->spWq + (size_t)h * hdp * d, sp.Wq, hd, d, tmp));
+      TRY(upload_packed(c->spWo + (size_t)h * dpad * hd, sp.Wo, d, hd, tmp));
+      TRY(upload_f32(c->sp_ga + (size_t)h * d, sp.ga, d));
+    }
+    for (int k = 0; k < 2; ++k)
+      for (int t = 0; t < c->hf_T[k]; ++t) {
+        const fm_hf_weights* arr = k == 0 ? w->hf_fv : (t < 3 * dm.nv ? w->hf_vc : w->hf_fc);
+        if (arr == nullptr) { delete c; return FM_ERR_INVALID_ARG; }
+        const fm_hf_weights& hb = arr[k == 0 ? t : (t < 3 * dm.nv ? t : t - 3 * dm.nv)];
+        TRY(upload_packed(c->hfWq[k] + (size_t)t * hdp * d, hb.Wq, hd, d, tmp));
+        TRY(upload_packed(c->hfW1[k] + (size_t)t * hfp * hd, hb.W1, (size_t)dm.hf, hd, tmp));
+        TRY(upload_packed(c->hfW2[k] + (size_t)t * dpad * dm.hf, hb.W2, d, (size_t)dm.hf, tmp));
+        TRY(upload_f32(c->hf_g[k] + (size_t)t * d, hb.g, d));
+      }
+  }
   if (w->label_g != nullptr && w->label_W != nullptr && dm.nv > 0) {
     TRY(upload_f32(c->label_g, w->label_g, d));
     TRY(upload_f32(c->label_W, w->label_W, 3 * d));
@@ -975,8 +1121,8 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
     freq[i] = dm.theta != 0.f ? pow((double)dm.theta, -2.0 * (double)i / (double)dm.dh) : 0.0;
   TRYCUDA(cudaMemcpy(c->inv_freq, freq.data(), freq.size() * sizeof(double), cudaMemcpyHostToDevice));
   {
-    const size_t n = (size_t)(dm.max_tokens + 1) * (dm.dh / 2);
-    rope_table_kernel<<<(unsigned)((n + 255) / 256), 256, 0, c->stream>>>(c->rope_tab, c->inv_freq, dm.max_tokens + 1, dm.dh / 2);
+    const size_t n = (size_t)(dm.max_tokens + 1 + FM_ROPE_SLACK) * (dm.dh / 2);
+    rope_table_kernel<<<(unsigned)((n + 255) / 256), 256, 0, c->stream>>>(c->rope_tab, c->inv_freq, dm.max_tokens + 1 + FM_ROPE_SLACK, dm.dh / 2);
     TRYCUDA(cudaGetLastError());
   }
   TRYCUDA(cudaHostAlloc(reinterpret_cast<void**>(&c->host_done), 64, cudaHostAllocMapped));

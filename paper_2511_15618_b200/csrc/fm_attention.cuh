@@ -36,6 +36,12 @@ struct AttnArgs {
   int G;                      // chunks per group
   int max_groups;             // groups the cache of this level can hold (= gridDim.x)
   int MT;                     // 16-row query tiles per (sequence, kv-head)
+  // Draft mode (SP-Block / HF-Block queries, Sec. 3.1): draft_nq > 0 query rows per sequence, none of
+  // them in the cache; every row sees what the last accepted position of the level sees (the prefix
+  // and positions max(0, p - W + 1) .. p with p = floor((L - 1) / ratio)).  Row r of sequence b is
+  // read at q[(b * draft_nq + r)] and written to out row r * out_row_stride + b.
+  int draft_nq;
+  int out_row_stride;
 };
 
 template <int DH, int C, int NW>
@@ -82,9 +88,10 @@ __global__ void __launch_bounds__((NW + 1) * 32) attn_stream_kernel(const AttnAr
   const int n = b < a.batch ? a.st.nrow[b] : 0;
   const int Lb = b < a.batch ? a.st.L[b] : 0;
   const int ratio = fm_ratio(level);
-  const int p0 = attn::div_ratio(Lb + ratio - 1, level);
-  const int nq = n > 0 ? attn::div_ratio(Lb + n - 1, level) - p0 + 1 : 0;
-  const int p_max = p0 + nq - 1;
+  const bool dmode = a.draft_nq > 0;
+  const int p0 = dmode ? attn::div_ratio(Lb - 1, level) : attn::div_ratio(Lb + ratio - 1, level);
+  const int nq = n > 0 ? (dmode ? a.draft_nq : attn::div_ratio(Lb + n - 1, level) - p0 + 1) : 0;
+  const int p_max = dmode ? p0 : p0 + nq - 1;
   const int P = dm.P, cap = dm.cap[level], W = dm.window[level];
   const int slots = P + cap;
   const int used = P + min(cap, p_max + 1);
@@ -100,7 +107,7 @@ __global__ void __launch_bounds__((NW + 1) * 32) attn_stream_kernel(const AttnAr
     return;
   }
   const int c_lo = u * a.G, n_my = min(a.G, n_chunks - c_lo);
-  const int m_rows = fm_rows_per_seq(dm, level);
+  const int m_rows = dmode ? a.draft_nq : fm_rows_per_seq(dm, level);
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -111,10 +118,11 @@ __global__ void __launch_bounds__((NW + 1) * 32) attn_stream_kernel(const AttnAr
   // slots written by this pass: P + (p mod cap), p = p0..p_max: one run of nq slots from new_lo,
   // which may wrap around the end of the ring once
   const int new_lo = P + p0 % cap;
+  const int n_new = dmode ? 0 : nq;                          // draft queries append nothing
   auto has_new = [&](int c) {
     const int lo = c * C, hi = lo + C;                       // [lo, hi)
-    const int e1 = min(new_lo + nq, slots);                  // first part [new_lo, e1)
-    const int n2 = new_lo + nq - e1;                         // wrapped part [P, P + n2)
+    const int e1 = min(new_lo + n_new, slots);               // first part [new_lo, e1)
+    const int n2 = new_lo + n_new - e1;                      // wrapped part [P, P + n2)
     return (new_lo < hi && e1 > lo) || (n2 > 0 && P < hi && P + n2 > lo);
   };
   const int row_base = (b * dm.Hkv + hk) * slots;
@@ -169,7 +177,7 @@ __global__ void __launch_bounds__((NW + 1) * 32) attn_stream_kernel(const AttnAr
       const int idx = mt * 16 + g + hrow * 8;
       const bool ok = idx < M;
       const int r = ok ? (group == 1 ? idx : idx / group) : 0, gh = ok ? idx - r * group : 0;
-      prow[hrow] = ok ? p0 + r : -100;
+      prow[hrow] = ok ? (dmode ? p0 : p0 + r) : -100;
       const bf16* qp = a.q + ((size_t)(b * m_rows + r) * dm.H + hk * group + gh) * DH;
 #pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
@@ -351,7 +359,8 @@ __global__ void __launch_bounds__((NW + 1) * 32) attn_stream_kernel(const AttnAr
       const int idx = mt * 16 + i;
       if (idx >= M) continue;
       const int r = group == 1 ? idx : idx / group, gh = idx - r * group;
-      attn::store_out(a.out, ((size_t)(b * m_rows + r) * 2 * dm.H + hk * group + gh) * DH + c, res[e] / res[16 * DH + i], dm.H * DH);
+      const size_t orow = a.out_row_stride > 0 ? (size_t)r * a.out_row_stride + b : (size_t)(b * m_rows + r);
+      attn::store_out(a.out, (orow * 2 * dm.H + hk * group + gh) * DH + c, res[e] / res[16 * DH + i], dm.H * DH);
     }
     return;
   }
@@ -420,7 +429,8 @@ __global__ void __launch_bounds__((NW + 1) * 32) attn_stream_kernel(const AttnAr
     }
     const int idx = mt * 16 + i;
     const int r = group == 1 ? idx : idx / group, gh = idx - r * group;
-    const size_t at = ((size_t)(b * m_rows + r) * 2 * dm.H + hk * group + gh) * DH + c;
+    const size_t orow = a.out_row_stride > 0 ? (size_t)r * a.out_row_stride + b : (size_t)(b * m_rows + r);
+    const size_t at = (orow * 2 * dm.H + hk * group + gh) * DH + c;
     const float o0 = acc0 / wr[n_groups], o1 = acc1 / wr[n_groups];
     const __nv_bfloat162 hi = __floats2bfloat162_rn(o0, o1);
     *reinterpret_cast<__nv_bfloat162*>(a.out + at) = hi;

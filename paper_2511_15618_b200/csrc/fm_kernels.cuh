@@ -17,6 +17,17 @@ __device__ inline float block_sum(float v, float* sh) {
   return t;
 }
 
+__device__ inline float block_max(float v, float* sh) {
+  v = warp_max(v);
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31, nw = blockDim.x >> 5;
+  __syncthreads();
+  if (l == 0) sh[w] = v;
+  __syncthreads();
+  float t = -INFINITY;
+  for (int i = 0; i < nw; ++i) t = fmaxf(t, sh[i]);
+  return t;
+}
+
 // ------------------------------------------------------------------------------------------
 // A GEMM operand value as two bfloat16 terms: hi = bf16(v) at p[0], lo = bf16(v - hi) at p[lo_off].
 __device__ inline void store_hi_lo(bf16* p, float v, int lo_off) {
@@ -434,6 +445,109 @@ __global__ void draft_residual_kernel(Dims dm, SeqState st, int batch, const flo
   }
 }
 
+// ---- full draft modules (Sec. 3.1 Eq. 1-5): row-wise pieces around the stacked GEMMs and the
+// attention launches.  A "set" is one SP head (set = head index h) or one HF-Block (set = offset
+// index t); operand and result rows of set t and sequence b sit at row t * max_batch + b.
+enum DraftStage { DS_SP = 0, DS_HF_V = 1, DS_HF_C = 2 };
+
+// the fp32 feature that HF-Block t of sequence b refines
+//   DS_HF_V: vertex rv = t % 3 of face head e = 1 + t / 3, in the face level's upsampled triples [Ef*B, 3d]
+//   DS_HF_C: t < 3 nv: coordinate r = t % 3 of vertex head e = 1 + t / 3; else slot s of face head e,
+//            both in the coordinate-level feature matrix (rows as in draft_feature_row)
+__device__ inline float* hf_feature(const Dims& dm, int stage, int t, int b, int B, float* xv_pre, float* feat) {
+  if (stage == DS_HF_V) return xv_pre + ((size_t)(t / 3) * B + b) * 3 * dm.d + (size_t)(t % 3) * dm.d;
+  const int tv = 3 * dm.nv;
+  if (t < tv) return feat + ((size_t)dm.nc * B + 3 * ((size_t)(t / 3) * B + b) + t % 3) * dm.d;
+  const int tt = t - tv, e0 = tt / 9, s = tt % 9;
+  return feat + ((size_t)dm.nc * B + 3 * ((size_t)dm.nv * B + 3 * ((size_t)e0 * B + b) + s / 3) + s % 3) * dm.d;
+}
+// level-local position of the query of set t (SP: the split node's own position)
+__device__ inline int draft_query_pos(const Dims& dm, int stage, int level, int t, int n) {
+  if (stage == DS_SP) return level == 0 ? n : (level == 1 ? n / 3 : n / 9);
+  if (stage == DS_HF_V) return 3 * (n / 9) + t;
+  const int tv = 3 * dm.nv;
+  if (t < tv) return 3 * (n / 3 + 1 + t / 3) + t % 3;
+  return 9 * (n / 9) + (t - tv);
+}
+
+// a[t][b] = bf16(rms(x) * g_t) for the HF-Blocks' inputs
+__global__ void hf_prep_kernel(Dims dm, SeqState st, int batch, int stage, float* xv_pre, float* feat,
+                               const float* __restrict__ gains /*[T, d]*/, bf16* __restrict__ a /*[T*max_batch, d]*/) {
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
+  __shared__ float sh[32];
+  const int b = blockIdx.x, t = blockIdx.y, d = dm.d;
+  if (b >= batch) return;
+  const float* x = hf_feature(dm, stage, t, b, batch, xv_pre, feat);
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) ss += x[i] * x[i];
+  ss = block_sum(ss, sh);
+  const float inv = rsqrtf(ss / (float)d + dm.eps);
+  bf16* dst = a + ((size_t)t * dm.max_batch + b) * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = __float2bfloat16(x[i] * inv * gains[(size_t)t * d + i]);
+}
+
+// queries of the draft modules: rotate to the query's level position, scale, round; rows
+// [t0, t0 + T) of the projection's output become rows (b * T + (t - t0)) of the attention's q
+__global__ void draft_q_kernel(Dims dm, SeqState st, int batch, int stage, int level, int t0, int T,
+                               const float* __restrict__ qf /*[sets*max_batch, H*dh]*/, const float2* __restrict__ rope_tab,
+                               float qscale, bf16* __restrict__ q /*[B*T, H*dh]*/) {
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
+  const int b = blockIdx.x, t = blockIdx.y;        // t counts from t0
+  if (b >= batch) return;
+  const int n = max(0, st.L[b] - 1), half = dm.dh >> 1, hd = dm.H * dm.dh;
+  const int pos = draft_query_pos(dm, stage, level, t0 + t, n);
+  const float* src = qf + ((size_t)(t0 + t) * dm.max_batch + b) * hd;
+  bf16* dst = q + ((size_t)b * T + t) * hd;
+  for (int i = threadIdx.x; i < dm.H * half; i += blockDim.x) {
+    const int head = i / half, k = i - head * half;
+    float2 cs = make_float2(1.f, 0.f);
+    if (dm.theta != 0.f) cs = rope_tab[(size_t)pos * half + k];
+    const float x1 = src[head * dm.dh + k], x2 = src[head * dm.dh + half + k];
+    dst[head * dm.dh + k] = __float2bfloat16((x1 * cs.x - x2 * cs.y) * qscale);
+    dst[head * dm.dh + half + k] = __float2bfloat16((x2 * cs.x + x1 * cs.y) * qscale);
+  }
+}
+
+// SP-Block, between its attention and its linear layer: y = z + Wo o, a[h][b] = bf16(rms(y) * g_h)
+__global__ void sp_mid_kernel(Dims dm, SeqState st, int batch, const float* __restrict__ zc, const float* __restrict__ zv,
+                              const float* __restrict__ zf, const float* __restrict__ u /*[NH*max_batch, d]*/,
+                              const float* __restrict__ gains, bf16* __restrict__ a) {
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
+  __shared__ float sh[32];
+  const int h = blockIdx.y, b = blockIdx.x, d = dm.d;
+  if (b >= batch) return;
+  const int n = max(0, st.L[b] - 1);
+  const float* z = head_split_node(dm, h, b, n, zc, zv, zf);
+  const float* ur = u + ((size_t)h * dm.max_batch + b) * d;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) { const float y = z[i] + ur[i]; ss += y * y; }
+  ss = block_sum(ss, sh);
+  const float inv = rsqrtf(ss / (float)d + dm.eps);
+  bf16* dst = a + ((size_t)h * dm.max_batch + b) * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = __float2bfloat16((z[i] + ur[i]) * inv * gains[(size_t)h * d + i]);
+}
+
+// HF-Block, last step: x += FFN output; the vertex-level blocks also hand the refined vertex
+// feature to the next upsample GEMM (bf16 operand row)
+__global__ void hf_finish_kernel(Dims dm, SeqState st, int batch, int stage, float* xv_pre, float* feat,
+                                 const float* __restrict__ y /*[T*max_batch, d]*/, bf16* __restrict__ up_in_v) {
+  ptx::grid_dep_launch();
+  ptx::grid_dep_wait();
+  const int b = blockIdx.x, t = blockIdx.y, d = dm.d;
+  if (b >= batch) return;
+  float* x = hf_feature(dm, stage, t, b, batch, xv_pre, feat);
+  const float* yr = y + ((size_t)t * dm.max_batch + b) * d;
+  bf16* up = stage == DS_HF_V ? up_in_v + ((size_t)dm.nv * batch + 3 * ((size_t)(t / 3) * batch + b) + t % 3) * d : nullptr;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    const float v = x[i] + yr[i];
+    x[i] = v;
+    if (up != nullptr) up[i] = __float2bfloat16(v);
+  }
+}
+
 // Source of draft offset j (single source per offset; supplement, "Optimizations"): offsets 1,2
 // -> coordinate heads (rule B); targets in the next two vertices v*+1, v*+2 -> vertex head
 // floor(p/3) - v*, wherever the face boundary lies, except where the latest vertex row was also a
@@ -468,7 +582,8 @@ __global__ void draft_pick_kernel(Dims dm, SeqState st, int batch, const float* 
                                   float* __restrict__ logits_out, float* __restrict__ margin_out,
                                   const GenOut* __restrict__ gen, const bf16* __restrict__ point_feat /*[(nv+3Ef)*B, d]*/,
                                   const float* __restrict__ label_g, const float* __restrict__ label_W,
-                                  int* __restrict__ labels /*[B, R1]*/, float* __restrict__ label_margin) {
+                                  int* __restrict__ labels /*[B, R1]*/, float* __restrict__ label_margin,
+                                  float* __restrict__ avg_rows /*[B*R1, Vpad] scratch of the averaged merge*/) {
   ptx::grid_dep_launch();
   ptx::grid_dep_wait();
   const int b = blockIdx.x, j = blockIdx.y;        // j = 0..D
@@ -518,6 +633,36 @@ __global__ void draft_pick_kernel(Dims dm, SeqState st, int batch, const float* 
   int level, head, slot;
   draft_source(dm, n, j, level, head, slot);
   const float* z = logits + (size_t)draft_feature_row(dm, level, head, slot, b, batch) * dm.Vpad;
+  if (dm.avg) {
+    // every level that predicts this position (supplement, "Integrating the three levels"): the
+    // coordinate head of the offset if there is one, the point level for the next two vertices,
+    // the face level for the faces its heads draft; the row becomes log(mean of the softmaxes)
+    __shared__ float sha[32];
+    const float* zs[3];
+    int ns = 0;
+    const int p = n + j, ev = p / 3 - n / 3, ef = p / 9 - n / 9 + 1;
+    if (j <= dm.nc) zs[ns++] = logits + (size_t)draft_feature_row(dm, 0, j, 0, b, batch) * dm.Vpad;
+    if (dm.nv > 0 && ev >= 1 && ev <= 2) zs[ns++] = logits + (size_t)draft_feature_row(dm, 1, ev, p % 3, b, batch) * dm.Vpad;
+    if (dm.nv > 0 && ev >= 1 && ef >= 1 && ef <= dm.Ef) zs[ns++] = logits + (size_t)draft_feature_row(dm, 2, ef, p % 9, b, batch) * dm.Vpad;
+    float mx[3], inv_sum[3];
+    for (int k = 0; k < ns; ++k) {
+      float m = -INFINITY;
+      for (int i = threadIdx.x; i < dm.V; i += blockDim.x) m = fmaxf(m, zs[k][i]);
+      m = block_max(m, sha);
+      float e = 0.f;
+      for (int i = threadIdx.x; i < dm.V; i += blockDim.x) e += expf(zs[k][i] - m);
+      e = block_sum(e, sha);
+      mx[k] = m; inv_sum[k] = 1.f / e;
+    }
+    float* row = avg_rows + (size_t)(b * dm.R1 + j) * dm.Vpad;
+    for (int i = threadIdx.x; i < dm.V; i += blockDim.x) {
+      float pr = 0.f;
+      for (int k = 0; k < ns; ++k) pr += expf(zs[k][i] - mx[k]) * inv_sum[k];
+      row[i] = logf(pr / (float)ns);
+    }
+    __syncthreads();
+    z = row;
+  }
   if (logits_out)
     for (int i = threadIdx.x; i < dm.V; i += blockDim.x) logits_out[((size_t)b * dm.D + j - 1) * dm.V + i] = z[i];
   const Top2 t = block_top2(z, dm, n + j);

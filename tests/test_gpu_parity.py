@@ -66,6 +66,32 @@ def test_toy_coordinate_only_drafting_lockstep(D):
     print(D, {k: rep[k] for k in ("steps", "max_logit_err", "max_draft_err", "overrides")})
 
 
+@pytest.mark.parametrize("D,avg,window,kv", [(9, 0, (0, 0, 0), 2), (12, 0, (11, 5, 2), 2), (9, 1, (0, 0, 0), 2), (27, 0, (0, 0, 0), 1), (3, 1, (0, 0, 0), 2)])
+def test_toy_full_sp_and_hf_blocks_lockstep(D, avg, window, kv):
+    """The paper's draft path (Sec. 3.1 Eq. 1-5): SP-Blocks with attention over the backbone's cache,
+    an HF-Block after every upsample; single-source and averaged merge; windows; shared KV head."""
+    from oracle.lockstep import run_lockstep
+    cfg = S.toy_config(**TOY, draft_len=D, draft_heads="full", avg_levels=avg, window=window, n_kv_heads=kv, hf_ff=192,
+                       layers=(1, 2, 2, 1, 2), max_batch=2, prompt_faces=(1, 1), gen_faces=6)
+    cfg = cfg.with_(max_tokens=1 + 9 * 8 + D + 2)
+    w, conds, prompts = _setup(cfg, batch=2)
+    prompts[1] = prompts[1] + prompts[0]
+    dev = _dev(cfg, w)
+    rep = run_lockstep(cfg, w, conds, prompts, dev, [6, 5], 200, tol=TOY_TOL, margin=TOY_MARGIN)
+    assert rep["done"] and rep["emitted"] == 9 * 11 and dev.device_status() == 0
+    print(D, avg, {k: rep[k] for k in ("steps", "max_logit_err", "max_draft_err", "overrides", "labels", "label_flips")})
+
+
+def test_toy_averaged_merge_of_reduced_heads_lockstep():
+    from oracle.lockstep import run_lockstep
+    cfg = S.toy_config(**TOY, draft_len=12, avg_levels=1, layers=(1, 1, 2, 1, 1), max_batch=2, gen_faces=6, max_tokens=1 + 9 * 8 + 12 + 2)
+    w, conds, prompts = _setup(cfg, batch=2)
+    dev = _dev(cfg, w)
+    rep = run_lockstep(cfg, w, conds, prompts, dev, 6, 200, tol=TOY_TOL, margin=TOY_MARGIN)
+    assert rep["done"] and dev.device_status() == 0
+    print({k: rep[k] for k in ("steps", "max_logit_err", "max_draft_err", "overrides")})
+
+
 def test_toy_lockstep_windows_and_mqa_and_eos():
     from oracle.lockstep import run_lockstep
     cfg = S.toy_config(**TOY, draft_len=9, layers=(2, 1, 2, 2, 1), window=(11, 5, 2), n_kv_heads=1, allow_eos=1,
@@ -115,6 +141,17 @@ def test_tiny_full_length_lockstep():
     rep = run_lockstep(cfg, w, conds, prompts, dev, cfg.gen_faces, 400)
     assert rep["done"] and rep["emitted"] == 288 and rep["max_logit_err"] <= 2e-2
     print(rep)
+
+
+def test_tiny_and_small_full_draft_modules_lockstep():
+    from oracle.lockstep import run_lockstep
+    for name, faces in (("tiny", 8), ("small", 6)):
+        cfg = S.get_config(name).with_(draft_heads="full")
+        w, conds, prompts = _setup(cfg)
+        dev = _dev(cfg, w)
+        rep = run_lockstep(cfg, w, conds, prompts, dev, faces, 100)
+        assert rep["done"] and rep["emitted"] == 9 * faces and rep["max_draft_err"] <= 2e-2 and dev.device_status() == 0
+        print(name, {k: rep[k] for k in ("steps", "max_logit_err", "max_draft_err", "overrides", "labels", "label_flips")})
 
 
 def test_small_lockstep_with_teacher_drafts():

@@ -40,6 +40,22 @@ def test_medium_model_lockstep_with_teacher_drafts():
     print(rep)
 
 
+def test_medium_model_full_draft_modules_lockstep():
+    """Medium with the full SP-Blocks and HF-Blocks: draft logits of all three pipelines against the
+    oracle for a few passes behind a 40-face prefix."""
+    from oracle.lockstep import run_lockstep
+    fill, faces = 40, 2
+    cfg = S.get_config("medium").with_(draft_heads="full", gen_faces=faces, max_tokens=1 + 9 * (fill + faces) + 9 + 2)
+    w = S.make_weights(cfg)
+    conds = [S.make_condition(cfg)]
+    prompts = [S.fill_prompt(cfg, 0, fill)]
+    dev = _dev(cfg, w)
+    rep = run_lockstep(cfg, w, conds, prompts, dev, faces, 6, prefill_chunk=512)
+    assert rep["steps"] == 6 and rep["max_logit_err"] <= 2e-2 and rep["max_draft_err"] <= 2e-2
+    assert dev.device_status() == 0
+    print(rep)
+
+
 def test_batched_ragged_lockstep():
     from oracle.lockstep import run_lockstep
     B = 4
