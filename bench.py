@@ -137,6 +137,11 @@ def run_ours(args):
     cfg = S.get_config(args.workload)
     if args.draft_len >= 0:               # cost curve of the pass against the number of drafts
         cfg = cfg.with_(draft_len=args.draft_len)
+    cfg = cfg.with_(draft_heads=args.draft_heads, draft_levels=args.draft_levels)
+    if args.kv_heads > 0:
+        cfg = cfg.with_(n_kv_heads=args.kv_heads)
+    if args.full_run:
+        return run_full_length(args, cfg, rank, local)
     B, D = cfg.batch, cfg.draft_len
     K, W = args.steps, args.warmup
     start_faces = int(cfg.gen_faces * args.start_frac)
@@ -337,6 +342,67 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_full_length(args, cfg, rank, local):
+    """The workload as configured: its own prompts, generation to gen_faces faces per sequence (or to
+    per-sequence stop lengths), teacher drafts from a plain run on the same kernels.  Reports
+    tokens/s over the whole run and the verify-step fraction of the HBM peak in three windows."""
+    import torch
+    from paper_2511_15618_b200 import FlashMesh
+    B, D = cfg.batch, cfg.draft_len
+    w = S.make_weights(cfg)
+    conds = np.stack([S.make_condition(cfg, b) for b in range(B)])
+    prompts = [[int(t) for t in S.make_prompt(cfg, b)] for b in range(B)]
+    faces = cfg.gen_faces
+    stops = S.stop_lengths(cfg.seed, B, faces).tolist() if args.stop_lengths else [faces] * B
+    dev = FlashMesh(cfg, w, device=f"cuda:{local}")
+    del w
+    stride = 9 * faces
+    dev.prefill(conds, prompts)
+    dev.set_max_faces(stops)
+    plain_tok, plain_len, st_plain = dev.generate(-1, plain=True, stride=stride)
+    pt, pl = plain_tok.cpu().numpy(), plain_len.cpu().numpy()
+    truth = np.zeros((B, max(len(p) for p in prompts) + stride), dtype=np.int32)
+    for b in range(B):
+        seq = np.concatenate([np.asarray(prompts[b], np.int32), pt[b, :pl[b]]])
+        truth[b, :len(seq)] = seq
+    keep = (S.accept_schedule(cfg.seed + rank, B, 4096, D, MEAN_DRAFTS) - 1).astype(np.int32)
+    truth_d, keep_d = torch.as_tensor(truth).cuda(), torch.as_tensor(keep).cuda()
+    dev.prefill(conds, prompts)
+    dev.set_max_faces(stops)
+    peak, peak_kind = _peaks()
+    est_steps = max(1, int(sum(stops) * 9 / B / (1 + MEAN_DRAFTS)))
+    seg = max(20, est_steps // 40)
+    out, windows, total_ms, total_tok, total_steps = None, [], 0.0, 0, 0
+    for _ in range(100000):
+        tok, ln, st = dev.generate(-1, truth=truth_d, keep=keep_d, max_steps=seg, out=out, stride=stride)
+        out = (tok, ln)
+        total_ms += float(st.ms); total_tok += int(st.emitted); total_steps += int(st.steps)
+        cand, _, _ = dev.draft()
+        o, _, _ = dev.verify(cand)
+        act = (o[:, 0] >= 0).cpu().numpy()
+        active = int(act.sum())
+        lens = ln.cpu().numpy()
+        kv = [[int(1 + len(prompts[b]) + lens[b]), -(-int(1 + len(prompts[b]) + lens[b]) // 3), -(-int(1 + len(prompts[b]) + lens[b]) // 9)]
+              for b in range(B) if act[b]]
+        ms_step = float(st.ms) / max(1, int(st.steps))
+        frac = dev.verify_bytes(kv) / (ms_step * 1e-3) / 1e9 / peak if kv else 0.0
+        windows.append((total_steps, ms_step, int(st.emitted), active, frac))
+        if active == 0 or int(st.emitted) == 0:
+            break
+    got, n = tok.cpu().numpy(), ln.cpu().numpy()
+    for b in range(B):
+        assert n[b] == pl[b] and (got[b, :n[b]] == pt[b, :n[b]]).all(), "speculative output differs from plain decoding"
+    line = {"metric": METRIC, "mode": "full_run", "value": total_tok / (total_ms * 1e-3), "unit": "tokens/s", "workload": cfg.name,
+            "batch": B, "draft_len": D, "draft_heads": cfg.draft_heads, "n_kv_heads": cfg.n_kv_heads,
+            "faces_per_sequence": stops, "steps": total_steps, "emitted": total_tok, "ms_total": total_ms,
+            "tokens_per_pass": total_tok / max(1, total_steps),
+            "plain_run": {"tokens_per_s": float(pl.sum()) / (st_plain.ms * 1e-3), "ms_per_pass": st_plain.ms / max(1, st_plain.steps)},
+            "windows": [{"after_steps": a, "ms_per_step": m, "emitted": e, "active_sequences": act, "verify_step_frac_of_hbm_peak": fr}
+                        for a, m, e, act, fr in (windows[0], windows[len(windows) // 2], windows[-2] if len(windows) > 1 else windows[-1])],
+            "peak_GBps": peak, "peak_kind": peak_kind}
+    print(json.dumps(line), flush=True)
+
+
 def run_e2e(dev, cfg, truth, keep, prompts, steps):
     """Host-in-the-loop decode through the stepwise C ABI: per pass the host builds the edited
     candidates from the transcript (it knows L from the previous pass), copies them in from pinned
@@ -450,6 +516,11 @@ def main():
     ap.add_argument("--no-batched", action="store_true", help="skip the batch-16 add-on of the default run")
     ap.add_argument("--timed-only", action="store_true", help="stop after the timed passes (for profiler captures)")
     ap.add_argument("--draft-len", type=int, default=-1, help="override the workload's number of drafts D (0 = plain decoding)")
+    ap.add_argument("--draft-heads", default="reduced", choices=["reduced", "full"], help="draft modules: reduced heads or the full SP / HF blocks")
+    ap.add_argument("--draft-levels", default="three", choices=["three", "coord"], help="coord: D coordinate heads only (the supplement's ablation)")
+    ap.add_argument("--kv-heads", type=int, default=0, help="override n_kv_heads (1 = one shared KV head)")
+    ap.add_argument("--full-run", action="store_true", help="decode the workload's whole length from its own prompt; report tokens/s over the run and the verify-step fraction at the start, middle and end")
+    ap.add_argument("--stop-lengths", action="store_true", help="with --full-run: per-sequence stop lengths from the face-count split of the paper's data")
     ap.add_argument("--pin-accept", type=int, default=0,
                     help="teacher drafts with the true acceptance pinned to this many tokens per pass (1 .. D+1); 0 = seeded schedule")
     args = ap.parse_args()

@@ -287,7 +287,8 @@ int fm_accept(fm_ctx* ctx, const int32_t* force_len /*DEV*/, const int32_t* forc
  * receives the emitted tokens (prompt not included), out_len: DEV int32 [batch], zeroed by the
  * first call after fm_prefill and advanced by every call; both may be NULL.  teacher and stats may
  * be NULL.  plain != 0 accepts only the main token every pass (the one-token-at-a-time baseline
- * on the same kernels).  Synchronous (returns after the last pass).
+ * on the same kernels).  max_faces == -1 keeps the per-sequence limits set with fm_set_max_faces
+ * (tokens beyond out_stride are then not stored).  Synchronous (returns after the last pass).
  * Errors: BAD_STATE, CAPACITY (prompt + 9*max_faces + D + 2 > max_tokens, or out_stride too small). */
 int fm_generate(fm_ctx* ctx, int32_t max_faces, int32_t* out_tok /*DEV*/, int32_t out_stride,
                 int32_t* out_len /*DEV*/, const fm_teacher* teacher /*HOST struct, DEV arrays*/,

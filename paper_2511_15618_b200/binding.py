@@ -460,12 +460,13 @@ class FlashMesh:
         self._after(fl, ft, n_acc, em, kv)
         return n_acc, em, kv
 
-    def generate(self, max_faces, truth=None, keep=None, plain=False, out=None, max_steps=0):
+    def generate(self, max_faces, truth=None, keep=None, plain=False, out=None, max_steps=0, stride=None):
         """Run the decode loop; returns (tokens [B, 9*max_faces] int32, lengths [B], FmStats).
-        `out` = (tokens, lengths) of an earlier call continues appending to them."""
+        `out` = (tokens, lengths) of an earlier call continues appending to them.  max_faces = -1
+        keeps the limits of set_max_faces (give `stride`, the row length of the token buffer)."""
         t = self.torch
         B = self.batch
-        stride = 9 * max_faces
+        stride = 9 * max_faces if stride is None else int(stride)
         out_tok = out[0] if out is not None else self.torch.full((B, max(stride, 1)), -1, dtype=t.int32, device=self.device)
         out_len = out[1] if out is not None else self._empty((B,), t.int32)
         teacher = None

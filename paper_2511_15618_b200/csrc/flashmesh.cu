@@ -1427,17 +1427,22 @@ int fm_accept(fm_ctx* c, const int32_t* force_len, const int32_t* force_tok, int
 
 int fm_generate(fm_ctx* c, int32_t max_faces, int32_t* out_tok, int32_t out_stride, int32_t* out_len,
                 const fm_teacher* teacher, int32_t plain, int64_t max_steps, fm_stats* stats) {
-  if (c == nullptr || max_faces < 0) return FM_ERR_INVALID_ARG;
+  if (c == nullptr || max_faces < -1) return FM_ERR_INVALID_ARG;
   if (c->phase < 1) return FM_ERR_BAD_STATE;
   const Dims& dm = c->dm;
-  if (out_tok != nullptr && (out_len == nullptr || out_stride < 9 * max_faces)) return FM_ERR_CAPACITY;
+  const bool keep_limits = max_faces == -1;          // per-sequence limits of fm_set_max_faces stay
+  if (keep_limits) max_faces = (dm.max_tokens + 8) / 9;
+  if (out_tok != nullptr && (out_len == nullptr || (!keep_limits && out_stride < 9 * max_faces))) return FM_ERR_CAPACITY;
   if (teacher != nullptr && (teacher->truth == nullptr || teacher->truth_stride <= 0 ||
                              (teacher->keep != nullptr && teacher->n_sched <= 0))) return FM_ERR_INVALID_ARG;
-  for (int b = 0; b < c->batch; ++b)
-    if ((long long)c->plen_host[b] + 9ll * max_faces + dm.D + 2 > dm.max_tokens) return FM_ERR_CAPACITY;
-  std::vector<int> lim(c->batch, max_faces);
-  int rc = fm_set_max_faces(c, lim.data());
-  if (rc != FM_OK) return rc;
+  int rc = FM_OK;
+  if (!keep_limits) {
+    for (int b = 0; b < c->batch; ++b)
+      if ((long long)c->plen_host[b] + 9ll * max_faces + dm.D + 2 > dm.max_tokens) return FM_ERR_CAPACITY;
+    std::vector<int> lim(c->batch, max_faces);
+    rc = fm_set_max_faces(c, lim.data());
+    if (rc != FM_OK) return rc;
+  }
   GenOut g{};
   g.out_tok = out_tok; g.out_stride = out_stride; g.out_len = out_len;
   if (teacher != nullptr) { g.truth = teacher->truth; g.truth_stride = teacher->truth_stride; g.keep = teacher->keep; g.n_sched = teacher->n_sched; }
