@@ -281,6 +281,16 @@ int fm_verify_static_scratch(fm_ctx* ctx, const int32_t* cand /*DEV*/, int32_t* 
 int fm_accept(fm_ctx* ctx, const int32_t* force_len /*DEV*/, const int32_t* force_tok /*DEV*/,
               int32_t* n_acc /*DEV*/, int32_t* emitted /*DEV*/, int32_t* kv_len /*DEV*/);
 
+/* One pass of the loop for a host that sits in it (Sec. 3: predict, edit, verify, accept), with HOST
+ * buffers: runs the draft modules; copies `cand` in (HOST int32 [batch, D+1], pinned memory makes
+ * the copy asynchronous; an entry >= 0 replaces the draft modules' candidate at that slot, an entry
+ * < 0 keeps it, slot 0 always stays the pending main token; NULL keeps all); verifies; accepts;
+ * copies n_acc [batch], emitted [batch, D+1] (may be NULL) and kv_len [batch, 3] (may be NULL) back to
+ * HOST memory and waits for the stream.  Equivalent to fm_draft, fm_verify, fm_accept with the
+ * copies in between, in one call.  Errors as those calls. */
+int fm_step_host(fm_ctx* ctx, const int32_t* cand /*HOST*/, int32_t* n_acc /*HOST*/, int32_t* emitted /*HOST*/,
+                 int32_t* kv_len /*HOST*/);
+
 /* The whole loop (Sec. 3): draft -> (optional teacher edit) -> verify -> accept, until every
  * sequence has emitted 9*max_faces tokens or EOS, or, when max_steps > 0, for exactly max_steps
  * passes (a later call continues where this one stopped).  out_tok: DEV int32 [batch, out_stride]

@@ -107,6 +107,8 @@ def load_library():
     lib.fm_verify.argtypes = [vp, vp, vp, f32p, f32p]
     lib.fm_verify_static_scratch.restype = C.c_int
     lib.fm_verify_static_scratch.argtypes = [vp, vp, vp, f32p, f32p]
+    lib.fm_step_host.restype = C.c_int
+    lib.fm_step_host.argtypes = [vp, vp, vp, vp, vp]
     lib.fm_accept.restype = C.c_int
     lib.fm_accept.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.fm_generate.restype = C.c_int
@@ -189,6 +191,11 @@ def fm_verify_static_scratch(ctx, cand_ptr, argmax_ptr=None, logits_ptr=None, ma
     """fm_verify with the attention kernel's scratch in the library's own fixed array: for hosts
     that may not allocate device memory for it (see include/flashmesh.h)."""
     return load_library().fm_verify_static_scratch(ctx, cand_ptr, argmax_ptr, logits_ptr, margin_ptr)
+
+
+def fm_step_host(ctx, cand_host_ptr, n_acc_host_ptr, emitted_host_ptr=None, kv_len_host_ptr=None):
+    """One pass with host buffers (addresses of host memory; see include/flashmesh.h)."""
+    return load_library().fm_step_host(ctx, cand_host_ptr, n_acc_host_ptr, emitted_host_ptr, kv_len_host_ptr)
 
 
 def fm_accept(ctx, force_len_ptr=None, force_tok_ptr=None, n_acc_ptr=None, emitted_ptr=None, kv_len_ptr=None):
@@ -459,6 +466,13 @@ class FlashMesh:
                               kv.data_ptr()), "fm_accept")
         self._after(fl, ft, n_acc, em, kv)
         return n_acc, em, kv
+
+    def step_host(self, cand_h, n_acc_h, emitted_h=None, kv_len_h=None):
+        """One pass through fm_step_host; the arguments are host tensors (pinned for asynchronous
+        copies), int32: cand_h [B, D+1] or None, n_acc_h [B], emitted_h [B, D+1], kv_len_h [B, 3]."""
+        self._before()
+        ptr = lambda x: x.data_ptr() if x is not None else None
+        self._check(fm_step_host(self.ctx, ptr(cand_h), ptr(n_acc_h), ptr(emitted_h), ptr(kv_len_h)), "fm_step_host")
 
     def generate(self, max_faces, truth=None, keep=None, plain=False, out=None, max_steps=0, stride=None):
         """Run the decode loop; returns (tokens [B, 9*max_faces] int32, lengths [B], FmStats).

@@ -66,6 +66,7 @@ struct fm_ctx {
   float *dh_y, *feat, *dlogits;
   float *label_g, *label_W, *label_margin;   // label head of the correction stage and its last results
   int* labels;
+  int *step_in, *step_cand, *step_nacc, *step_em, *step_kv;     // device side of fm_step_host
   float* avg_rows;                           // [B*R1, Vpad] rows of the averaged merge
   // full draft modules: SP-Block attention (per head) and HF-Blocks (per offset), stacked per stage
   bf16 *spWq, *spWo; float* sp_ga;
@@ -261,6 +262,8 @@ void carve(fm_ctx* c, Carver& cv) {
   c->label_g = cv.take<float>(d); c->label_W = cv.take<float>(3 * d);
   c->labels = cv.take<int>(B * dm.R1); c->label_margin = cv.take<float>(B * dm.R1);
   c->st.hist = cv.take<int>(B * FM_HIST);
+  c->step_in = cv.take<int>(B * dm.R1); c->step_cand = cv.take<int>(B * dm.R1); c->step_nacc = cv.take<int>(B);
+  c->step_em = cv.take<int>(B * dm.R1); c->step_kv = cv.take<int>(B * 3);
   c->avg_rows = dm.avg ? cv.take<float>(B * dm.R1 * (size_t)dm.Vpad) : nullptr;
   c->hf_T[0] = 3 * dm.Ef; c->hf_T[1] = 3 * dm.nv + 9 * dm.Ef;
   c->draft_sets = dm.NH > c->hf_T[1] ? dm.NH : c->hf_T[1];
@@ -855,6 +858,14 @@ __global__ void verify_load_kernel(Dims dm, SeqState st, int batch, const int* _
   st.cand[i] = t;
 }
 
+// candidates of a host-driven pass: the host's entry where it gave one (>= 0), else the draft modules'
+__global__ void step_merge_kernel(Dims dm, SeqState st, int batch, const int* __restrict__ host_cand, int* __restrict__ out) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= batch * dm.R1) return;
+  const int h = host_cand != nullptr ? host_cand[i] : -1;
+  out[i] = (h >= 0 && i % dm.R1 != 0) ? h : st.cand[i];          // slot 0 is always the pending main token
+}
+
 __global__ void init_state_kernel(Dims dm, SeqState st, int batch, const int* __restrict__ prompt_off) {
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= dm.max_batch) return;
@@ -1411,6 +1422,26 @@ int fm_verify_static_scratch(fm_ctx* c, const int32_t* cand, int32_t* argmax, fl
   c->attn_part = saved_part;
   c->attn_ticket = saved_ticket;
   return rc;
+}
+
+int fm_step_host(fm_ctx* c, const int32_t* cand, int32_t* n_acc, int32_t* emitted, int32_t* kv_len) {
+  if (c == nullptr || n_acc == nullptr) return FM_ERR_INVALID_ARG;
+  if (c->phase < 1) return FM_ERR_BAD_STATE;
+  const Dims& dm = c->dm;
+  const int n = c->batch * dm.R1;
+  int rc = fm_draft(c, nullptr, nullptr, nullptr);
+  if (rc != FM_OK) return rc;
+  if (cand != nullptr) CUDA_OK(cudaMemcpyAsync(c->step_in, cand, n * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+  LAUNCH(c, step_merge_kernel, (n + 127) / 128, 128, 0, dm, c->st, c->batch, cand != nullptr ? (const int*)c->step_in : (const int*)nullptr, c->step_cand);
+  rc = fm_verify(c, c->step_cand, nullptr, nullptr, nullptr);
+  if (rc != FM_OK) return rc;
+  rc = fm_accept(c, nullptr, nullptr, c->step_nacc, c->step_em, c->step_kv);
+  if (rc != FM_OK) return rc;
+  CUDA_OK(cudaMemcpyAsync(n_acc, c->step_nacc, c->batch * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  if (emitted != nullptr) CUDA_OK(cudaMemcpyAsync(emitted, c->step_em, n * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  if (kv_len != nullptr) CUDA_OK(cudaMemcpyAsync(kv_len, c->step_kv, c->batch * 3 * sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_OK(cudaStreamSynchronize(c->stream));
+  return FM_OK;
 }
 
 int fm_accept(fm_ctx* c, const int32_t* force_len, const int32_t* force_tok, int32_t* n_acc, int32_t* emitted,

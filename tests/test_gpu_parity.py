@@ -257,3 +257,37 @@ def test_bounded_wait_gives_up_and_prefill_recovers():
     assert fm_selftest_wait_timeout(dev.ctx, 0) == -1              # limit out of range: nothing is launched
     rep = run_lockstep(cfg, w, conds, prompts, dev, 2, 40)         # starts with fm_prefill
     assert rep["done"] and rep["emitted"] == 18 and dev.device_status() == 0
+
+
+def test_step_host_equals_the_stepwise_calls():
+    """fm_step_host (one call per pass, host buffers) gives what fm_draft / fm_verify / fm_accept
+    give, with the host's candidates where it supplies them and the draft modules' elsewhere."""
+    import torch
+    cfg = S.get_config("tiny")
+    w, conds, prompts = _setup(cfg)
+    D = cfg.draft_len
+    a, b = _dev(cfg, w), _dev(cfg, w)
+    a.prefill(np.stack(conds), prompts)
+    b.prefill(np.stack(conds), prompts)
+    truth = _oracle_greedy(cfg, w, conds[0], prompts[0], 6)
+    cand_h = torch.full((1, D + 1), -1, dtype=torch.int32).pin_memory()
+    nacc_h = torch.zeros((1,), dtype=torch.int32).pin_memory()
+    em_h = torch.zeros((1, D + 1), dtype=torch.int32).pin_memory()
+    kv_h = torch.zeros((1, 3), dtype=torch.int32).pin_memory()
+    L = 1 + len(prompts[0])
+    for step in range(12):
+        cand, _, _ = a.draft()
+        c = cand.cpu().numpy()
+        edit = np.full((1, D + 1), -1, dtype=np.int32)
+        if step % 3 != 2:                                 # some passes keep the draft modules' own candidates
+            k = step % (D + 1)
+            for j in range(1, k + 1):
+                edit[0, j] = truth[L - 1 + j]
+            c[edit >= 0] = edit[edit >= 0]
+        a.verify(c)
+        n_a, em_a, kv_a = a.accept()
+        cand_h.copy_(torch.as_tensor(edit))
+        b.step_host(cand_h if step % 3 != 2 else None, nacc_h, em_h, kv_h)
+        assert int(n_a[0]) == int(nacc_h[0]) and em_a.cpu().tolist() == em_h.tolist() and kv_a.cpu().tolist() == kv_h.tolist()
+        L += int(nacc_h[0])
+    assert a.device_status() == 0 and b.device_status() == 0
