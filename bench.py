@@ -65,7 +65,7 @@ def rank_sequences(rank, batch_per_rank):
 # DRAM traffic of the dominant kernel per launch from ncu (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by workload, each with the summary under profiles/ that holds the
 # capture; None where the kernel changed since the capture or none was taken.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {"medium": {"bytes_per_launch": 6.46e6, "summary": "profiles/gemm_and_attention_dram_traffic_medium.md"}}
 
 
 class ClockSampler:
