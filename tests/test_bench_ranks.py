@@ -44,3 +44,13 @@ def test_report_is_reduced_over_two_gloo_ranks_and_sequences_are_disjoint():
 def test_single_process_passes_through():
     import bench
     assert bench.reduce_over_ranks([1.5], [2.0, 3.0], "cpu") == ([1.5], [2.0, 3.0])
+
+
+def test_gpus_flag_must_agree_with_the_launcher():
+    """Started by a launcher (RANK set) with a world size that differs from --gpus, the benchmark
+    stops with a message instead of silently timing one replica."""
+    import subprocess
+    env = dict(os.environ, RANK="0", WORLD_SIZE="1", LOCAL_RANK="0")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "1"], env=env,
+                       capture_output=True, text=True, timeout=120)
+    assert r.returncode != 0 and "--gpus 2 but WORLD_SIZE is 1" in r.stderr
