@@ -334,6 +334,17 @@ def run_ours(args):
                                           "note": "S = T_ori * m / T_ours (Sec. 4.1) with T_ori from this run"}
             except Exception:
                 line["plain_decoding"] = {"error": (r.stderr or r.stdout)[-300:]}
+        if world == 1 and args.workload == "medium" and args.draft_len < 0 and not args.no_batched:
+            # the small workloads, timed passes only (the Large line, which needs minutes of prefill,
+            # is in profiles/workload_lines_and_draft_variants.md with its command)
+            line["other_workloads"] = {}
+            for wl, st_ in (("tiny", "50"), ("small", "100")):
+                r = subprocess.run([sys.executable, os.path.abspath(__file__), "--workload", wl, "--steps", st_, "--warmup", "5",
+                                    "--timed-only", "--no-cpu"], capture_output=True, text=True)
+                try:
+                    line["other_workloads"][wl] = json.loads(r.stdout.strip().splitlines()[-1])
+                except Exception:
+                    line["other_workloads"][wl] = {"error": (r.stderr or r.stdout)[-300:]}
         if world == 1 and not args.no_cpu:
             line["cpu_baseline"] = cpu_baseline(args.workload, budget_s=args.cpu_seconds)
         print(json.dumps(line), flush=True)
