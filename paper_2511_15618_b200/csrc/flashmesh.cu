@@ -59,7 +59,8 @@ struct fm_ctx {
   SeqState st;
   // activations
   float *xc, *xv, *xf, *logits, *tmp3d;
-  bf16 *qbuf, *a_norm, *a_cat, *a_attn, *a_ff;
+  bf16 *qbuf, *a_norm, *a_cat, *a_cat2, *a_attn, *a_ff;
+  bool fuse_hourglass;                     // shorten gather and upsample add inside the adjacent GEMM epilogues
   float *hc_ring, *hv_ring, *trif_ring, *triv_ring, *zc, *zv, *zf;
   // draft
   bf16 *dh_a, *up_in_v, *up_in_f, *feat_n;
@@ -246,7 +247,7 @@ void carve(fm_ctx* c, Carver& cv) {
   c->ssq = cv.take<float>((size_t)((d + 127) / 128) * tc::MAX_SPLIT * Rc);
   c->logits = cv.take<float>(Rc * dm.Vpad); c->tmp3d = cv.take<float>(Rv * 3 * d);
   // GEMM operand rows of the backbone hold two bfloat16 terms per value: [hi | lo]
-  c->a_norm = cv.take<bf16>(Rc * 2 * d); c->a_cat = cv.take<bf16>(Rv * 6 * d);
+  c->a_norm = cv.take<bf16>(Rc * 2 * d); c->a_cat = cv.take<bf16>(Rv * 6 * d); c->a_cat2 = cv.take<bf16>(Rf * 6 * d);
   c->a_attn = cv.take<bf16>(Rc * 2 * hd); c->a_ff = cv.take<bf16>(Rc * 2 * dm.dff);
   c->hc_ring = cv.take<float>(B * FM_RING_C * d); c->hv_ring = cv.take<float>(B * FM_RING_V * d);
   c->trif_ring = cv.take<float>(B * FM_RING_F * 3 * d); c->triv_ring = cv.take<float>(B * FM_RING_V * 3 * d);
@@ -602,6 +603,8 @@ void gemm(fm_ctx* c, const bf16* W, size_t w_rows_alloc, int w_row0, const bf16*
     case tc::EPI_F32: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_F32, false>, grid, 128, smem, g, e); break;
     case tc::EPI_BF16: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_BF16, false>, grid, 128, smem, g, e); break;
     case tc::EPI_GELU: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_GELU, false>, grid, 128, smem, g, e); break;
+    case tc::EPI_RESID_CAT: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_RESID_CAT, false>, grid, 128, smem, g, e); break;
+    case tc::EPI_UP: launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_UP, false>, grid, 128, smem, g, e); break;
     case tc::EPI_RESID:
       if (side) launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_RESID, true>, grid, 128, smem, g, e);
       else launch_pdl(c, cl, tc::gemm_tc_kernel<tc::EPI_RESID, false>, grid, 128, smem, g, e);
@@ -613,7 +616,8 @@ void gemm(fm_ctx* c, const bf16* W, size_t w_rows_alloc, int w_row0, const bf16*
   }
   c->cur_class = PROF_OTHER;
   prof_close(c, pi);
-  if (mode == tc::EPI_RESID && e.ssq_out != nullptr) c->ssq_n = tiles * split * (split == 1 ? 2 : 1);     // slots the next consumer adds
+  if ((mode == tc::EPI_RESID || mode == tc::EPI_RESID_CAT) && e.ssq_out != nullptr) c->ssq_n = tiles * split * (split == 1 ? 2 : 1);     // slots the next consumer adds
+  if (mode == tc::EPI_UP && e.ssq_out != nullptr) c->ssq_n = (c->dm.d / tc::BM) * split * (split == 1 ? 2 : 1);   // tiles within d
 }
 
 // rows fed at each level in this pass (n_active[level]); n_active[3] = unfinished sequences
@@ -645,7 +649,7 @@ inline size_t pad128(size_t v) { return align_up(v, 128); }
 // layer.  On entry c->a_norm holds bf16(x * g1 of the first layer) and c->ssq the rows' sums of
 // squares; on exit, if `want_a`, c->a_norm holds bf16(x * next_gain) (gain 1 when null) and c->ssq
 // the sums of squares of the stack's output rows.
-void run_stack(fm_ctx* c, int s, float* x, float* stash_ring, const float* next_gain, bool want_a) {
+void run_stack(fm_ctx* c, int s, float* x, float* stash_ring, const float* next_gain, bool want_a, const tc::Epi* cat = nullptr) {
   const Dims& dm = c->dm;
   const int level = STACK_LEVEL[s];
   const int rows = c->batch * fm_rows_per_seq(dm, level);
@@ -677,6 +681,12 @@ void run_stack(fm_ctx* c, int s, float* x, float* stash_ring, const float* next_
     const bool last = l == nl - 1;
     e2.gain = last ? next_gain : c->layers[s][l + 1].g1;
     if (last && !want_a) { e2.a_out = nullptr; e2.ssq_out = nullptr; }
+    if (last && cat != nullptr) {                           // the stack below a shortening: hiddens leave through the epilogue
+      e2.dm = dm; e2.st = c->st; e2.batch = c->batch; e2.level = level; e2.d_model = d;
+      e2.cat_out = cat->cat_out; e2.cat_ring = cat->cat_ring; e2.cat_tri = cat->cat_tri;
+      gemm(c, L.W2, pad128(d), 0, c->a_ff, Rc_alloc, 0, d, dm.dff, rows, na, tc::EPI_RESID_CAT, e2, 2);
+      continue;
+    }
     gemm(c, L.W2, pad128(d), 0, c->a_ff, Rc_alloc, 0, d, dm.dff, rows, na, tc::EPI_RESID, e2, 2);
   }
 }
@@ -691,28 +701,63 @@ void forward(fm_ctx* c, float* logits_out) {
   // The launch that opens a pass is a full barrier: the per-pass state (rows, lengths, row counts
   // -- every call that changes them ends with a row count -- and candidates) is final before any
   // later kernel's prologue can run.
-  LAUNCH(c, embed_kernel, Rc, row_threads(d), 0, dm, c->st, B, c->E, c->xc, c->layers[0][0].g1, c->a_norm, c->ssq);
-  c->ssq_n = 1;
-  run_stack(c, 0, c->xc, nullptr, nullptr, false);
-  launch_pdl(c, dim3(1, 1, 1), shorten_gather_kernel, dim3(Rv + Rc, 3), row_threads(d), 0, dm, c->st, B, 1, (const float*)c->xc, c->hc_ring, c->a_cat, Rv);
+  const size_t Rf_alloc = align_up((size_t)dm.max_batch * dm.mf, 16);
   tc::Epi es{};
-  es.x = c->xv; es.ldx = d; es.add = 0; es.gain = c->layers[1][0].g1; es.a_out = c->a_norm; es.lda = 2 * d; es.lo_off = d;
+  es.ldx = d; es.add = 0; es.a_out = c->a_norm; es.lda = 2 * d; es.lo_off = d;
   es.ssq_out = c->ssq; es.ld_ssq_out = c->ssq_ld;
-  gemm(c, c->S_cv, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rv, na + 1, tc::EPI_RESID, es, 2);
-  run_stack(c, 1, c->xv, nullptr, nullptr, false);
-  launch_pdl(c, dim3(1, 1, 1), shorten_gather_kernel, dim3(Rf + Rv, 3), row_threads(d), 0, dm, c->st, B, 2, (const float*)c->xv, c->hv_ring, c->a_cat, Rf);
-  es.x = c->xf; es.gain = c->layers[2][0].g1;
-  gemm(c, c->S_vf, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rf, na + 2, tc::EPI_RESID, es, 2);
-  run_stack(c, 2, c->xf, c->zf, nullptr, true);                    // leaves bf16(xf) in a_norm
-  gemm(c, c->U_fv, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rf, na + 2, tc::EPI_F32, epi_plain(c->tmp3d, 3 * d), 2);
-  launch_pdl(c, dim3(1, 1, 1), upsample_add_kernel, Rv + Rf, row_threads(d), 0, dm, c->st, B, 1, (const float*)c->hv_ring, (const float*)c->tmp3d,
-             c->trif_ring, c->xv, (const float*)c->layers[3][0].g1, c->a_norm, c->ssq, Rv);
-  c->ssq_n = 1;
-  run_stack(c, 3, c->xv, c->zv, nullptr, true);                    // leaves bf16(xv) in a_norm
-  gemm(c, c->U_vc, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rv, na + 1, tc::EPI_F32, epi_plain(c->tmp3d, 3 * d), 2);
-  launch_pdl(c, dim3(1, 1, 1), upsample_add_kernel, Rc + Rv, row_threads(d), 0, dm, c->st, B, 0, (const float*)c->hc_ring, (const float*)c->tmp3d,
-             c->triv_ring, c->xc, (const float*)c->layers[4][0].g1, c->a_norm, c->ssq, Rc);
-  c->ssq_n = 1;
+  if (c->fuse_hourglass) {
+    // Shorten and upsample inside the adjacent GEMMs.  Down: the epilogue of a down-stack's last layer
+    // scatters the new hiddens into the shorten GEMM's concatenated operand rows and the carry ring
+    // (the parts that precede the pass were laid down by the opening launch) and gives rows whose
+    // parent belongs to an earlier pass that parent's stored slot.  Up: the upsampling GEMM's
+    // epilogue adds slot r of parent u to child row 3u + r, whose residual row still holds the
+    // pre-shorten hidden, and hands the child rows to the stack above.
+    LAUNCH(c, embed_kernel, Rc + 3 * (Rv + Rf), row_threads(d), 0, dm, c->st, B, c->E, c->xc, c->layers[0][0].g1, c->a_norm, c->ssq, Rc,
+           (const float*)c->hc_ring, (const float*)c->hv_ring, c->a_cat, c->a_cat2, Rv, Rf);
+    c->ssq_n = 1;
+    tc::Epi cat{};
+    cat.cat_out = c->a_cat; cat.cat_ring = c->hc_ring; cat.cat_tri = c->triv_ring;
+    run_stack(c, 0, c->xc, nullptr, nullptr, false, &cat);
+    es.x = c->xv; es.gain = c->layers[1][0].g1;
+    gemm(c, c->S_cv, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rv, na + 1, tc::EPI_RESID, es, 2);
+    cat.cat_out = c->a_cat2; cat.cat_ring = c->hv_ring; cat.cat_tri = c->trif_ring;
+    run_stack(c, 1, c->xv, nullptr, nullptr, false, &cat);
+    es.x = c->xf; es.gain = c->layers[2][0].g1;
+    gemm(c, c->S_vf, pad128(d), 0, c->a_cat2, Rf_alloc, 0, d, 3 * d, Rf, na + 2, tc::EPI_RESID, es, 2);
+    run_stack(c, 2, c->xf, c->zf, nullptr, true);                  // leaves bf16(xf) in a_norm
+    tc::Epi eu{};
+    eu.dm = dm; eu.st = c->st; eu.batch = B; eu.d_model = d;
+    eu.ldx = d; eu.a_out = c->a_norm; eu.lda = 2 * d; eu.lo_off = d; eu.ssq_out = c->ssq; eu.ld_ssq_out = c->ssq_ld;
+    eu.level = 2; eu.x = c->xv; eu.gain = c->layers[3][0].g1; eu.tri_ring = c->trif_ring;
+    // (skipped only when the CHILD level has no rows: children whose parent is older than the pass
+    // still need their operand rows and sums of squares)
+    gemm(c, c->U_fv, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rf, na + 1, tc::EPI_UP, eu, 2);
+    run_stack(c, 3, c->xv, c->zv, nullptr, true);                  // leaves bf16(xv) in a_norm
+    eu.level = 1; eu.x = c->xc; eu.gain = c->layers[4][0].g1; eu.tri_ring = c->triv_ring;
+    gemm(c, c->U_vc, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rv, na, tc::EPI_UP, eu, 2);
+  } else {
+    LAUNCH(c, embed_kernel, Rc, row_threads(d), 0, dm, c->st, B, c->E, c->xc, c->layers[0][0].g1, c->a_norm, c->ssq, Rc,
+           (const float*)nullptr, (const float*)nullptr, (bf16*)nullptr, (bf16*)nullptr, 0, 0);
+    c->ssq_n = 1;
+    run_stack(c, 0, c->xc, nullptr, nullptr, false);
+    launch_pdl(c, dim3(1, 1, 1), shorten_gather_kernel, dim3(Rv + Rc, 3), row_threads(d), 0, dm, c->st, B, 1, (const float*)c->xc, c->hc_ring, c->a_cat, Rv);
+    es.x = c->xv; es.gain = c->layers[1][0].g1;
+    gemm(c, c->S_cv, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rv, na + 1, tc::EPI_RESID, es, 2);
+    run_stack(c, 1, c->xv, nullptr, nullptr, false);
+    launch_pdl(c, dim3(1, 1, 1), shorten_gather_kernel, dim3(Rf + Rv, 3), row_threads(d), 0, dm, c->st, B, 2, (const float*)c->xv, c->hv_ring, c->a_cat, Rf);
+    es.x = c->xf; es.gain = c->layers[2][0].g1;
+    gemm(c, c->S_vf, pad128(d), 0, c->a_cat, Rv_alloc, 0, d, 3 * d, Rf, na + 2, tc::EPI_RESID, es, 2);
+    run_stack(c, 2, c->xf, c->zf, nullptr, true);                  // leaves bf16(xf) in a_norm
+    gemm(c, c->U_fv, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rf, na + 2, tc::EPI_F32, epi_plain(c->tmp3d, 3 * d), 2);
+    launch_pdl(c, dim3(1, 1, 1), upsample_add_kernel, Rv + Rf, row_threads(d), 0, dm, c->st, B, 1, (const float*)c->hv_ring, (const float*)c->tmp3d,
+               c->trif_ring, c->xv, (const float*)c->layers[3][0].g1, c->a_norm, c->ssq, Rv);
+    c->ssq_n = 1;
+    run_stack(c, 3, c->xv, c->zv, nullptr, true);                  // leaves bf16(xv) in a_norm
+    gemm(c, c->U_vc, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rv, na + 1, tc::EPI_F32, epi_plain(c->tmp3d, 3 * d), 2);
+    launch_pdl(c, dim3(1, 1, 1), upsample_add_kernel, Rc + Rv, row_threads(d), 0, dm, c->st, B, 0, (const float*)c->hc_ring, (const float*)c->tmp3d,
+               c->triv_ring, c->xc, (const float*)c->layers[4][0].g1, c->a_norm, c->ssq, Rc);
+    c->ssq_n = 1;
+  }
   run_stack(c, 4, c->xc, c->zc, c->g_out, true);                   // leaves bf16(xc * g_out) and its sums of squares
   tc::Epi el = epi_plain(c->logits, dm.Vpad);
   el.ssq_in = c->ssq; el.ssq_n = c->ssq_n; el.ld_ssq = c->ssq_ld; el.inv_d_in = 1.f / d; el.eps = dm.eps;
@@ -1124,6 +1169,8 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
   TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_RESID, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
   TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_QKV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
   TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_RESID, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_RESID_CAT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
+  TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_UP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
   TRYCUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<tc::EPI_QKV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::max_smem_bytes()));
   TRYCUDA(cudaFuncSetAttribute(attn_stream_kernel<64, 128, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<64, 128, 8>::BYTES));
   TRYCUDA(cudaFuncSetAttribute(attn_stream_kernel<128, 64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<128, 64, 4>::BYTES));
@@ -1162,6 +1209,8 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
     c->device = dev;
     const char* tt = getenv("FM_SPLIT_TARGET_DEEP");
     c->split_target_deep = tt != nullptr && atoi(tt) > 0 ? atoi(tt) : 296;
+    const char* nf = getenv("FM_NO_FUSE");
+    c->fuse_hourglass = c->dm.d % tc::BM == 0 && !(nf != nullptr && nf[0] == '1');
     const char* sc = getenv("FM_STAGE_CAP");
     c->stage_cap = sc != nullptr ? atoi(sc) : 4;        // measured: deeper rings cost more than they prefetch
   }

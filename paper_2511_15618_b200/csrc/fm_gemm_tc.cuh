@@ -27,7 +27,15 @@
 //   EPI_GELU             bf16(gelu(y))                      (first FFN matrix),
 //   EPI_RESID            x (+)= y; next operand bf16(x * gain); per-tile sums of squares
 //                        (output projection, second FFN matrix, shorten),
-//   EPI_QKV              rotary embedding, queries out, keys / values appended to the cache.
+//   EPI_QKV              rotary embedding, queries out, keys / values appended to the cache,
+//   EPI_RESID_CAT        EPI_RESID of the last layer below a shortening: the new hiddens are also
+//                        scattered into the concatenated operand rows of the shorten GEMM and into
+//                        the level's carry ring, and rows whose parent was computed in an earlier
+//                        pass receive that parent's stored upsampled slot at once,
+//   EPI_UP               the upsampling projection [3d x d]: slot r of parent row u is added to the
+//                        child row 3u + r of the level below (whose residual rows still hold the
+//                        pre-shorten hiddens), with next operand and sums of squares for the child
+//                        rows; the triple is stored for later passes.
 // The kernel is written for programmatic dependent launch: weights do not depend on the
 // previous kernel, so their first stages are requested before griddepcontrol.wait.
 #pragma once
@@ -42,7 +50,7 @@ constexpr int MAX_STAGES = 8;
 constexpr int MAX_SPLIT = 8;     // portable cluster size
 constexpr int MAX_N = 240;       // token rows per launch: two stages + the receive buffer must fit in 227 KB
 
-enum EpiMode { EPI_F32 = 0, EPI_BF16 = 1, EPI_GELU = 2, EPI_RESID = 3, EPI_QKV = 4 };
+enum EpiMode { EPI_F32 = 0, EPI_BF16 = 1, EPI_GELU = 2, EPI_RESID = 3, EPI_QKV = 4, EPI_RESID_CAT = 5, EPI_UP = 6 };
 
 struct Args {
   const bf16* W;                 // packed weight slabs: [M tile][K slab][128 x 64 swizzled image]
@@ -80,6 +88,13 @@ struct Epi {
   const float* stash_x;          //            when stash_ring is set: residual rows [rows, stash_d] that the CTAs
   float* stash_ring;             //            of K split 0 copy, column block by column block, into the carry ring
   int stash_d, stash_rs;         //            [B, stash_rs, stash_d] at entry pos mod stash_rs (split-node hiddens)
+  // EPI_RESID_CAT (dm, st, batch, level = this level): shorten / carry side outputs
+  bf16* cat_out;                 //            operand rows of the shorten GEMM [rows above, 6d] as [hi | lo], part k at k*d
+  float* cat_ring;               //            carry ring of this level's hiddens [B, fm_ring(level), d]
+  const float* cat_tri;          //            stored upsampled triples of the level above [B, fm_ring(level+1), 3d]
+  // EPI_UP (dm, st, batch, level = the parent level; x / gain / a_out / ssq_out describe the child rows)
+  float* tri_ring;               //            where the triples of this pass go [B, fm_ring(level), 3d]
+  int d_model;
 };
 
 __device__ inline uint64_t smem_desc_sw128(uint32_t addr) {
@@ -217,6 +232,8 @@ __device__ inline void pair_cols(int q, bool head128, int& ca, int& cb) {
 // mere presence of that path costs the few-row launches 0.4 us each (measured).
 template <int MODE, bool SIDE>
 __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e) {
+  constexpr int ROWS_AUX = (MODE == EPI_RESID_CAT || MODE == EPI_UP) ? 256 : 1;
+  constexpr int CARRY_MAX = MODE == EPI_UP ? 128 : 1;
   if (g.n_active != nullptr && *g.n_active == 0) {   // the whole grid leaves; keep the launch chain ordered
     ptx::grid_dep_launch();
     ptx::grid_dep_wait();
@@ -239,6 +256,8 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   __shared__ int s_fail;
   __shared__ float s_inv[256];
   __shared__ int s_rb[256], s_rp[256];
+  __shared__ int s_ra[ROWS_AUX], s_rl[ROWS_AUX];             // EPI_RESID_CAT / EPI_UP: see the row maps below
+  __shared__ int s_carry[CARRY_MAX], s_ncarry;               // EPI_UP: child rows whose parent is not in this pass
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tile_m = blockIdx.x;
@@ -295,7 +314,9 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   // angles (EPI_QKV tiles that hold query or key heads)
   // Only when a thread has more than two items: with fewer, loads straight into registers right
   // after the dependency wait are quicker than the round through the copy engine (measured).
-  const bool want_side = (MODE == EPI_RESID && e.add != 0) ||
+  constexpr bool IS_RESID = MODE == EPI_RESID || MODE == EPI_RESID_CAT;
+  constexpr bool ROW_MAPS = MODE == EPI_QKV || MODE == EPI_RESID_CAT || MODE == EPI_UP;
+  const bool want_side = (IS_RESID && e.add != 0) ||
                          (MODE == EPI_QKV && e.dm.theta != 0.f && (tile_m * BM) / e.dm.dh < e.dm.H + e.dm.Hkv);
   const bool use_side = SIDE && want_side;
   if (warp == 0) {
@@ -337,7 +358,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
     // ---- warps 2 and 3, while the operands arrive: operand-row scales (the partial sums of
     // squares of a row are gathered by 8 lanes, each adding its slots in slot order, then combined by
     // a fixed shuffle tree) and row maps
-    if (MODE == EPI_QKV && warp == 3) {
+    if (ROW_MAPS && warp == 3) {
       // row maps, and the rows' rotary angles into the side buffer: positions are per-pass state
       // and the table is constant, so nothing here waits for the previous kernel
       const uint32_t row_bytes = (uint32_t)e.dm.dh * 4u;   // dh/2 (cos, sin) pairs
@@ -347,17 +368,37 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
         int b = 0, p = 0;
         const bool valid = n < ns && fm_row_map(e.dm, e.st, e.batch, e.level, row0 + n, b, p);
         if (n < ns) { s_rb[n] = valid ? b : -1; s_rp[n] = p; }
+        if ((MODE == EPI_RESID_CAT || MODE == EPI_UP) && n < ns && valid) {
+          // first position of the sequence at the other level of the pair, last position at the lower one
+          const int Lb = e.st.L[b], nr = e.st.nrow[b];
+          const int rl = fm_ratio(MODE == EPI_UP ? e.level - 1 : e.level), ru = 3 * rl;
+          s_ra[n] = MODE == EPI_UP ? (Lb + rl - 1) / rl : (Lb + ru - 1) / ru;
+          s_rl[n] = (Lb + nr - 1) / rl;
+        }
         total += (uint32_t)__popc(__ballot_sync(0xffffffffu, valid)) * row_bytes;
       }
-      if (use_side) {
+      if (MODE == EPI_QKV && use_side) {
         if (lane == 0) ptx::mbar_expect_tx(sbar, total);
         __syncwarp();
         for (int n = lane; n < ns; n += 32)
           if (s_rb[n] >= 0) ptx::bulk_load(side + n * 128, e.rope_tab + (size_t)s_rp[n] * (e.dm.dh >> 1), row_bytes, sbar);
       }
     }
+    if (MODE == EPI_UP && warp == 2 && lane == 0) {
+      const int lvl = e.level - 1, rl = fm_ratio(lvl), m_low = fm_rows_per_seq(e.dm, lvl);
+      const int slot = (tile_m * BM) / e.d_model;
+      int cnt = 0;
+      for (int b = 0; b < e.batch; ++b) {
+        const int nr = e.st.nrow[b], Lb = e.st.L[b];
+        if (nr <= 0) continue;
+        const int p0l = (Lb + rl - 1) / rl, plast = (Lb + nr - 1) / rl, p0u = (Lb + 3 * rl - 1) / (3 * rl);
+        for (int p = p0l; p < 3 * p0u && p <= plast; ++p)
+          if (p % 3 == slot && cnt < CARRY_MAX) s_carry[cnt++] = b * m_low + (p - p0l);
+      }
+      s_ncarry = cnt;
+    }
     ptx::grid_dep_wait();
-    if (MODE == EPI_RESID && use_side && warp == 2) {      // residual rows of this tile's columns
+    if (IS_RESID && use_side && warp == 2) {               // residual rows of this tile's columns
       const int cols = min(BM, g.M - tile_m * BM);
       if (lane == 0) ptx::mbar_expect_tx(sbar, (uint32_t)(ns * cols) * 4u);
       __syncwarp();
@@ -419,9 +460,13 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
     int ca, cb;
     pair_cols<MODE == EPI_QKV>(z * PW + (tid & (PW - 1)), head128, ca, cb);
     const int ma = tile_m * BM + ca, mb = tile_m * BM + cb;
-    if (MODE == EPI_RESID && e.gain != nullptr) {
+    if (IS_RESID && e.gain != nullptr) {
       if (ma < g.M) pre_ga = e.gain[ma];
       if (mb < g.M) pre_gb = e.gain[mb];
+    }
+    if (MODE == EPI_UP && e.gain != nullptr) {             // gains of the child rows' next norm: column m mod d
+      if (ma < g.M) pre_ga = e.gain[ma % e.d_model];
+      if (mb < g.M) pre_gb = e.gain[mb % e.d_model];
     }
     if (MODE == EPI_QKV && want_side && !use_side) {
       int b, p;
@@ -448,7 +493,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
   asm volatile("" : "+f"(k_qs), "+r"(k_H), "+r"(k_Hkv), "+r"(k_dh), "+r"(k_P), "+r"(k_cap));
   ptx::grid_dep_wait();                                    // everything below touches activations
   float pre_xa = 0.f, pre_xb = 0.f;                        // first item's residual values, same case
-  if (MODE == EPI_RESID && want_side && !use_side && tid < items) {
+  if (IS_RESID && want_side && !use_side && tid < items) {
     int ca, cb;
     pair_cols<MODE == EPI_QKV>(z * PW + (tid & (PW - 1)), head128, ca, cb);
     const int ma = tile_m * BM + ca, mb = tile_m * BM + cb;
@@ -542,7 +587,7 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
       bf16* o = reinterpret_cast<bf16*>(k_out) + row * k_ldo;
       if (b_ok) store_hi_lo2(o + ma, gelu_erf_f(ya), gelu_erf_f(yb), k_lo);
       else if (a_ok) store_hi_lo(o + ma, gelu_erf_f(ya), k_lo);
-    } else if (MODE == EPI_RESID) {
+    } else if (IS_RESID) {
       float* xr = k_x + row * k_ldx;
       float xa = 0.f, xb = 0.f;
       if (b_ok) {                                          // both columns (M is even wherever the residual is used)
@@ -552,6 +597,22 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
         else if (want_side) x0 = *reinterpret_cast<const float2*>(xr + ma);
         xa = x0.x + ya;
         xb = x0.y + yb;
+        if (MODE == EPI_RESID_CAT && s_rb[n] >= 0) {
+          // (xa, xb) is the level's final hidden of position p: into the carry ring, into the operand
+          // row of the parent that pools it (if that parent is a row of this pass), and, where the
+          // position's own parent p / 3 was computed in an earlier pass, that parent's stored slot
+          // is added at once (the up-stack then finds h + upsampled slot in the residual row)
+          const int b = s_rb[n], p = s_rp[n], dd = e.d_model, rs = fm_ring(e.level), rsu = fm_ring(e.level + 1);
+          *reinterpret_cast<float2*>(e.cat_ring + ((size_t)b * rs + p % rs) * dd + ma) = make_float2(xa, xb);
+          const int u = (p + 2) / 3, part = p - 3 * u + 2;
+          if (3 * u <= s_rl[n])
+            store_hi_lo2(e.cat_out + ((size_t)(b * fm_rows_per_seq(e.dm, e.level + 1) + u - s_ra[n]) * 6 + part) * dd + ma, xa, xb, 3 * dd);
+          if (p < 3 * s_ra[n]) {
+            const float2 t = __ldcg(reinterpret_cast<const float2*>(e.cat_tri + (((size_t)b * rsu + (p / 3) % rsu) * 3 + p % 3) * dd + ma));
+            xa += t.x;
+            xb += t.y;
+          }
+        }
         *reinterpret_cast<float2*>(xr + ma) = make_float2(xa, xb);
         if (k_aout != nullptr) store_hi_lo2(k_aout + row * k_lda + ma, xa * pre_ga, xb * pre_gb, k_lo);
       } else if (a_ok) {
@@ -566,6 +627,33 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
         for (int o = L >> 1; o > 0; o >>= 1) sqv += __shfl_xor_sync(0xffffffffu, sqv, o);
         if (active && (cc & (L - 1)) == 0)
           k_ssqo[(size_t)((((tile_m << lgS) + z) << (lgPW - lgL)) + (cc >> lgL)) * k_ldssq + k_row0 + n] = sqv;
+      }
+    } else if (MODE == EPI_UP) {
+      // (ya, yb): columns (ma, ma + 1) of the triple of parent row n = slot ma / d, column ma % d
+      const int dd = e.d_model;
+      float xa = 0.f, xb = 0.f;
+      bool child = false;
+      size_t crow = 0;
+      if (b_ok && s_rb[n] >= 0) {
+        const int b = s_rb[n], pu = s_rp[n], rsu = fm_ring(e.level);
+        *reinterpret_cast<float2*>(e.tri_ring + ((size_t)b * rsu + pu % rsu) * 3 * dd + ma) = make_float2(ya, yb);
+        const int slot = ma / dd, col = ma - slot * dd, p = 3 * pu + slot;
+        if (p <= s_rl[n]) {                                // the child is a row of this pass
+          child = true;
+          crow = (size_t)b * fm_rows_per_seq(e.dm, e.level - 1) + (p - s_ra[n]);
+          float* xr = k_x + crow * k_ldx + col;
+          const float2 x0 = __ldcg(reinterpret_cast<const float2*>(xr));
+          xa = x0.x + ya;
+          xb = x0.y + yb;
+          *reinterpret_cast<float2*>(xr) = make_float2(xa, xb);
+          if (k_aout != nullptr) store_hi_lo2(k_aout + crow * k_lda + col, xa * pre_ga, xb * pre_gb, k_lo);
+        }
+      }
+      if (k_ssqo != nullptr) {                             // as EPI_RESID, for the child row; tiles count within d
+        float sqv = xa * xa + xb * xb;
+        for (int o = L >> 1; o > 0; o >>= 1) sqv += __shfl_xor_sync(0xffffffffu, sqv, o);
+        if (active && child && (cc & (L - 1)) == 0)
+          k_ssqo[(size_t)(((((tile_m % (dd / BM)) << lgS) + z) << (lgPW - lgL)) + (cc >> lgL)) * k_ldssq + crow] = sqv;
       }
     } else {  // EPI_QKV: (ya, yb) is the rotary pair (i, i + dh/2) of one head
       const int dh = k_dh, half = dh >> 1, H = k_H, Hkv = k_Hkv;
@@ -594,6 +682,33 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
           dst[i] = __float2bfloat16(ya);
           dst[half + i] = __float2bfloat16(yb);
         }
+      }
+    }
+  }
+  if (MODE == EPI_UP) {
+    // child rows of this tile's slot whose parent was computed in an earlier pass: their residual
+    // rows are final already (the last layer below added the stored slot); what is missing is the
+    // next operand and the sums of squares, for this rank's columns
+    const int dd = e.d_model, nci = s_ncarry << lgPW;
+    for (int it0 = 0; it0 < nci; it0 += 128) {
+      const int it = it0 + tid;
+      const bool active = it < nci;
+      const int cc = it & (PW - 1);
+      const size_t crow = active ? (size_t)s_carry[it >> lgPW] : 0;
+      int ca, cb;
+      pair_cols<false>(z * PW + cc, false, ca, cb);
+      const int col = (tile_m * BM + ca) % dd;
+      float2 x0 = make_float2(0.f, 0.f);
+      if (active) x0 = __ldcg(reinterpret_cast<const float2*>(k_x + crow * k_ldx + col));
+      if (active && k_aout != nullptr) {
+        const float ga = e.gain != nullptr ? e.gain[col] : 1.f, gb = e.gain != nullptr ? e.gain[col + 1] : 1.f;
+        store_hi_lo2(k_aout + crow * k_lda + col, x0.x * ga, x0.y * gb, k_lo);
+      }
+      if (k_ssqo != nullptr) {
+        float sqv = x0.x * x0.x + x0.y * x0.y;
+        for (int o = L >> 1; o > 0; o >>= 1) sqv += __shfl_xor_sync(0xffffffffu, sqv, o);
+        if (active && (cc & (L - 1)) == 0)
+          k_ssqo[(size_t)(((((tile_m % (dd / BM)) << lgS) + z) << (lgPW - lgL)) + (cc >> lgL)) * k_ldssq + crow] = sqv;
       }
     }
   }

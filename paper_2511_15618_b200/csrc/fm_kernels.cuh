@@ -54,11 +54,40 @@ __device__ inline void stack_entry_row(const float* xr, int row, int d, const fl
   if (threadIdx.x == 0) ssq[row] = ss;
 }
 
+// first level-local position of sequence b in this pass
+__device__ inline int fm_first_pos(const SeqState& st, int b, int level) {
+  const int r = fm_ratio(level);
+  return (st.L[b] + r - 1) / r;
+}
+
 // ------------------------------------------------------------------------------------------
 // a1. candidate embedding: x[row] = E[cand[b][j]]  (zeros for rows that are not fed)
 // ------------------------------------------------------------------------------------------
 __global__ void embed_kernel(Dims dm, SeqState st, int batch, const bf16* __restrict__ E, float* __restrict__ x,
-                             const float* __restrict__ g, bf16* __restrict__ a_out, float* __restrict__ ssq) {
+                             const float* __restrict__ g, bf16* __restrict__ a_out, float* __restrict__ ssq,
+                             int rows, const float* __restrict__ hc_ring, const float* __restrict__ hv_ring,
+                             bf16* __restrict__ cat_v, bf16* __restrict__ cat_f, int rows_v, int rows_f) {
+  if ((int)blockIdx.x >= rows) {
+    // Blocks behind the coordinate rows prepare the operand rows of the two shorten GEMMs (used when
+    // the gather is fused into the producing GEMM's epilogue): part k of parent row u pools position
+    // 3u - 2 + k of the level below; what lies before this pass comes from the carry ring (zeros
+    // below position 0 and for rows that are not fed), the rest is written by the epilogue of the
+    // last layer below.
+    int j = (int)blockIdx.x - rows;
+    const int level_out = j < 3 * rows_v ? 1 : 2;
+    if (level_out == 2) j -= 3 * rows_v;
+    if (cat_v == nullptr || j >= 3 * (level_out == 1 ? rows_v : rows_f)) return;
+    const int row = j / 3, part = j - 3 * row, lb = level_out - 1, rs = fm_ring(lb), d = dm.d;
+    int b, u;
+    const bool valid = fm_row_map(dm, st, batch, level_out, row, b, u);
+    const int pos = 3 * u - 2 + part, p0 = valid ? fm_first_pos(st, b, lb) : 0;
+    if (valid && pos >= p0) return;                  // a hidden of this pass
+    const bool ok = valid && pos >= 0;
+    const float* src = (lb == 0 ? hc_ring : hv_ring) + ((size_t)b * rs + ((pos + rs) % rs)) * d;
+    bf16* out = (level_out == 1 ? cat_v : cat_f) + (size_t)row * 6 * d + part * d;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) store_hi_lo(out + i, ok ? src[i] : 0.f, 3 * d);
+    return;
+  }
   const int row = blockIdx.x;
   int b, p;
   const bool valid = fm_row_map(dm, st, batch, 0, row, b, p);
@@ -123,11 +152,6 @@ __global__ void prefix_store_kernel(Dims dm, int level, int row0, const float* _
 // ------------------------------------------------------------------------------------------
 // hourglass carry rings
 // ------------------------------------------------------------------------------------------
-// first level-local position of sequence b in this pass
-__device__ inline int fm_first_pos(const SeqState& st, int b, int level) {
-  const int r = fm_ratio(level);
-  return (st.L[b] + r - 1) / r;
-}
 
 // a3/a5 shorten, gather half, fused with the ring store of the level below.  Blocks [0, rows_out):
 // row v of level `level_out` <- [h_{3v-2}; h_{3v-1}; h_{3v}] (zeros for negative positions and for
