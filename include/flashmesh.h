@@ -179,7 +179,7 @@ size_t fm_workspace_bytes(const fm_config* cfg /*HOST*/);
  * default stream); all later work of this context runs on it.  Synchronous.
  * Errors: INVALID_ARG (null, bad config), CAPACITY (workspace too small), UNSUPPORTED
  * (d_model or d_ff not a multiple of 64, n_heads*head_dim not a multiple of 128, head_dim not
- * 64/128, a stack without layers, D > FM_MAX_DRAFT), CUDA. */
+ * 64/128, a stack without layers, D > FM_MAX_DRAFT, hf_ff not a multiple of 64), CUDA. */
 int fm_create(const fm_config* cfg /*HOST*/, const fm_weights* w /*HOST*/, void* dev_workspace /*DEV*/,
               size_t workspace_bytes, void* cuda_stream, fm_ctx** out /*HOST*/);
 int fm_destroy(fm_ctx* ctx);
@@ -197,8 +197,10 @@ int fm_prefill(fm_ctx* ctx, int32_t batch, const float* cond /*DEV*/, const int3
  * its prompt (or at EOS).  HOST int32 [batch].  Default: the cache capacity. */
 int fm_set_max_faces(fm_ctx* ctx, const int32_t* max_faces /*HOST*/);
 
-/* Predict (Sec. 3.1, supplement "Three-Level Speculative Decoding"): run the draft heads on
- * the split-node hiddens stashed at the last accepted position.  cand: DEV int32 out
+/* Predict (Sec. 3.1, supplement "Three-Level Speculative Decoding"): run the draft modules
+ * (reduced heads, or the full SP-Blocks and HF-Blocks; fm_config.draft_heads / draft_levels) on
+ * the split-node hiddens stashed at the last accepted position; with a label head, also the
+ * labels of the drafted points (fm_draft_labels).  cand: DEV int32 out
  * [batch, D+1] = pending main token, then D drafts (PAD for finished sequences).
  * draft_logits: DEV float32 out [batch, D, V] or NULL.  draft_margin: DEV float32 out
  * [batch, D] (top-1 minus top-2 of the masked draft logits) or NULL. */
@@ -210,7 +212,7 @@ int fm_draft(fm_ctx* ctx, int32_t* cand /*DEV*/, float* draft_logits /*DEV*/, fl
  * token and is never touched; vertices that are only partly in the row, or that hold a token that
  * is not a coordinate bin, are left alone).  labels: DEV int32 [batch, D+1]; labels[b][s] is the
  * label of the point that starts at slot s: FM_LABEL_HISTORICAL, FM_LABEL_NEW or FM_LABEL_INTRA
- * (other slots are not read; the label head that would produce them is not part of the library).
+ * (other slots are not read; fm_draft_labels gives the labels of the library's own label head).
  * In sequence order, every FM_LABEL_INTRA point that has no identical point in the row is
  * replaced by the nearest (squared distance between bin indices, ties to the earliest) earlier
  * FM_LABEL_NEW point of another face, if there is one; then the points of every face are sorted
