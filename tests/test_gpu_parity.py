@@ -166,10 +166,12 @@ def test_small_lockstep_with_teacher_drafts():
     print(rep)
 
 
-def test_generate_speculative_equals_plain_on_device():
+@pytest.mark.parametrize("variant", [{}, {"draft_heads": "full"}, {"draft_levels": "coord"}, {"avg_levels": 1}])
+def test_generate_speculative_equals_plain_on_device(variant):
     """Row-invariant numerics: speculative decoding on the GPU emits exactly what one-token-at-a-
-    time decoding on the same kernels emits, whatever the drafts are."""
-    cfg = S.get_config("tiny")
+    time decoding on the same kernels emits, whatever the drafts are (and whichever draft modules
+    produce them)."""
+    cfg = S.get_config("tiny").with_(**variant)
     w, conds, prompts = _setup(cfg)
     dev = _dev(cfg, w)
     dev.prefill(np.stack(conds), prompts)
