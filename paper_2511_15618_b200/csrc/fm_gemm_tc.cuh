@@ -198,10 +198,12 @@ inline int max_smem_bytes() {
   return a > b ? a : b;
 }
 
+// (The differences below use __fsub_rn so that the compiler cannot fold a product that the caller
+// passes in into a fused multiply-subtract: a value must split the same way at every call site.)
 __device__ inline void store_hi_lo(bf16* p, float v, int lo_off) {
   const bf16 hi = __float2bfloat16(v);
   p[0] = hi;
-  if (lo_off > 0) p[lo_off] = __float2bfloat16(v - __bfloat162float(hi));
+  if (lo_off > 0) p[lo_off] = __float2bfloat16(__fsub_rn(v, __bfloat162float(hi)));
 }
 
 // two neighbouring values as [hi, hi] and [lo, lo] pairs: one 4-byte store each
@@ -209,7 +211,7 @@ __device__ inline void store_hi_lo2(bf16* p, float a, float b, int lo_off) {
   const __nv_bfloat162 hi = __floats2bfloat162_rn(a, b);
   *reinterpret_cast<__nv_bfloat162*>(p) = hi;
   if (lo_off > 0)
-    *reinterpret_cast<__nv_bfloat162*>(p + lo_off) = __floats2bfloat162_rn(a - __bfloat162float(hi.x), b - __bfloat162float(hi.y));
+    *reinterpret_cast<__nv_bfloat162*>(p + lo_off) = __floats2bfloat162_rn(__fsub_rn(a, __bfloat162float(hi.x)), __fsub_rn(b, __bfloat162float(hi.y)));
 }
 
 __device__ inline float gelu_erf_f(float x) { return 0.5f * x * (1.f + erff(x * 0.70710678118654752f)); }
@@ -614,16 +616,16 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
           }
         }
         *reinterpret_cast<float2*>(xr + ma) = make_float2(xa, xb);
-        if (k_aout != nullptr) store_hi_lo2(k_aout + row * k_lda + ma, xa * pre_ga, xb * pre_gb, k_lo);
+        if (k_aout != nullptr) store_hi_lo2(k_aout + row * k_lda + ma, __fmul_rn(xa, pre_ga), __fmul_rn(xb, pre_gb), k_lo);
       } else if (a_ok) {
         xa = (use_side ? side[n * 128 + ca] : (first ? pre_xa : (want_side ? xr[ma] : 0.f))) + ya;
         xr[ma] = xa;
-        if (k_aout != nullptr) store_hi_lo(k_aout + row * k_lda + ma, xa * pre_ga, k_lo);
+        if (k_aout != nullptr) store_hi_lo(k_aout + row * k_lda + ma, __fmul_rn(xa, pre_ga), k_lo);
       }
       if (k_ssqo != nullptr) {
         // per-row sums of squares of this rank's columns: a fixed shuffle tree over the L lanes that
         // share the row; the next GEMM adds the (tile, rank, lane group) partials in slot order
-        float sqv = xa * xa + xb * xb;
+        float sqv = __fmaf_rn(xa, xa, __fmul_rn(xb, xb));
         for (int o = L >> 1; o > 0; o >>= 1) sqv += __shfl_xor_sync(0xffffffffu, sqv, o);
         if (active && (cc & (L - 1)) == 0)
           k_ssqo[(size_t)((((tile_m << lgS) + z) << (lgPW - lgL)) + (cc >> lgL)) * k_ldssq + k_row0 + n] = sqv;
@@ -646,11 +648,11 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
           xa = x0.x + ya;
           xb = x0.y + yb;
           *reinterpret_cast<float2*>(xr) = make_float2(xa, xb);
-          if (k_aout != nullptr) store_hi_lo2(k_aout + crow * k_lda + col, xa * pre_ga, xb * pre_gb, k_lo);
+          if (k_aout != nullptr) store_hi_lo2(k_aout + crow * k_lda + col, __fmul_rn(xa, pre_ga), __fmul_rn(xb, pre_gb), k_lo);
         }
       }
       if (k_ssqo != nullptr) {                             // as EPI_RESID, for the child row; tiles count within d
-        float sqv = xa * xa + xb * xb;
+        float sqv = __fmaf_rn(xa, xa, __fmul_rn(xb, xb));
         for (int o = L >> 1; o > 0; o >>= 1) sqv += __shfl_xor_sync(0xffffffffu, sqv, o);
         if (active && child && (cc & (L - 1)) == 0)
           k_ssqo[(size_t)(((((tile_m % (dd / BM)) << lgS) + z) << (lgPW - lgL)) + (cc >> lgL)) * k_ldssq + crow] = sqv;
@@ -702,10 +704,10 @@ __global__ void __launch_bounds__(128) gemm_tc_kernel(const Args g, const Epi e)
       if (active) x0 = __ldcg(reinterpret_cast<const float2*>(k_x + crow * k_ldx + col));
       if (active && k_aout != nullptr) {
         const float ga = e.gain != nullptr ? e.gain[col] : 1.f, gb = e.gain != nullptr ? e.gain[col + 1] : 1.f;
-        store_hi_lo2(k_aout + crow * k_lda + col, x0.x * ga, x0.y * gb, k_lo);
+        store_hi_lo2(k_aout + crow * k_lda + col, __fmul_rn(x0.x, ga), __fmul_rn(x0.y, gb), k_lo);
       }
       if (k_ssqo != nullptr) {
-        float sqv = x0.x * x0.x + x0.y * x0.y;
+        float sqv = __fmaf_rn(x0.x, x0.x, __fmul_rn(x0.y, x0.y));
         for (int o = L >> 1; o > 0; o >>= 1) sqv += __shfl_xor_sync(0xffffffffu, sqv, o);
         if (active && (cc & (L - 1)) == 0)
           k_ssqo[(size_t)(((((tile_m % (dd / BM)) << lgS) + z) << (lgPW - lgL)) + (cc >> lgL)) * k_ldssq + crow] = sqv;

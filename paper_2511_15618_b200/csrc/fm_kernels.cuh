@@ -33,7 +33,7 @@ __device__ inline float block_max(float v, float* sh) {
 __device__ inline void store_hi_lo(bf16* p, float v, int lo_off) {
   const bf16 hi = __float2bfloat16(v);
   p[0] = hi;
-  p[lo_off] = __float2bfloat16(v - __bfloat162float(hi));
+  p[lo_off] = __float2bfloat16(__fsub_rn(v, __bfloat162float(hi)));   // never fused with a product behind v
 }
 
 // Hand a freshly written residual row to the first layer of a stack: the GEMM operand row
@@ -48,7 +48,7 @@ __device__ inline void stack_entry_row(const float* xr, int row, int d, const fl
   for (int i = threadIdx.x; i < d; i += blockDim.x) {
     const float v = xr[i];
     ss += v * v;
-    store_hi_lo(a_out + (size_t)row * 2 * d + i, v * g[i], d);
+    store_hi_lo(a_out + (size_t)row * 2 * d + i, __fmul_rn(v, g[i]), d);
   }
   ss = block_sum(ss, sh);
   if (threadIdx.x == 0) ssq[row] = ss;

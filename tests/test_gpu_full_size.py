@@ -90,3 +90,54 @@ def test_logits_do_not_depend_on_the_row_at_benchmark_size():
     c2[0, 1:] = pt[2:D + 2]
     _, lg_b, _ = dev.verify(torch.as_tensor(c2).cuda(), want_logits=True)
     assert torch.equal(lg_a[0, 1:], lg_b[0, :D])
+
+
+@pytest.mark.parametrize("workload,n_tok", [("medium", 130), ("batched", 70)])
+def test_every_accept_pattern_leaves_the_logits_of_plain_decoding(workload, n_tok):
+    """Bit-exact losslessness (Sec. 3.3) at benchmark size.  A position's hidden states reach the
+    upper stacks along different code paths depending on where the passes happen to start: with its
+    parent vertex or face computed in the same pass, or in an earlier one (stored upsampled slot).
+    Decoding one token per pass takes the second path almost always, accepting whole passes takes
+    the first.  The logits of every position must not depend on that, to the last bit -- a
+    difference of one rounding in an operand row is enough to flip a near-tie thousands of tokens
+    later and let speculative output drift away from plain decoding."""
+    import torch
+    from paper_2511_15618_b200 import FlashMesh
+    cfg = S.get_config(workload)
+    faces = n_tok // 9 + 8
+    cfg = cfg.with_(gen_faces=faces, max_tokens=1 + 9 * (cfg.prompt_faces[1] + faces) + cfg.draft_len + 1)
+    B, D = cfg.batch, cfg.draft_len
+    w = S.make_weights(cfg)
+    conds = np.stack([S.make_condition(cfg, b) for b in range(B)])
+    prompts = [[int(t) for t in S.make_prompt(cfg, b)] for b in range(B)]
+    dev = FlashMesh(cfg, w)
+    del w
+    dev.prefill(conds, prompts)
+    plain, _, _ = dev.generate(faces, plain=True)
+    pt = plain.cpu().numpy()
+
+    def walk(pattern):
+        dev.prefill(conds, prompts)
+        got, n, step = {}, 0, 0
+        while n + D + 1 < n_tok:
+            cand, _, _ = dev.draft()
+            c = cand.cpu().numpy()
+            assert (c[:, 0] == pt[:, n]).all()
+            c[:, 1:] = pt[:, n + 1:n + 1 + D]                  # drafts = the true continuation
+            _, lg, _ = dev.verify(torch.as_tensor(c).cuda(), want_logits=True)
+            a = pattern[step % len(pattern)]
+            for j in range(a):
+                got[n + j] = lg[:, j].clone()
+            dev.accept(force_len=np.full(B, a, dtype=np.int32))
+            n += a
+            step += 1
+        return got
+
+    ref = walk([1])
+    for pattern in ([D + 1], [2], [4, 7, 1, D + 1, 2, 9, 5]):
+        got = walk(pattern)
+        common = [k for k in sorted(got) if k in ref]
+        assert len(common) > n_tok - 2 * (D + 1)
+        bad = [k for k in common if not torch.equal(got[k], ref[k])]
+        assert not bad, (pattern, bad[:5])
+    assert dev.device_status() == 0
