@@ -59,7 +59,7 @@ struct fm_ctx {
   SeqState st;
   // activations
   float *xc, *xv, *xf, *logits, *tmp3d;
-  bf16 *qbuf, *a_norm, *a_cat, *a_cat2, *a_attn, *a_ff;
+  bf16 *qbuf, *a_norm, *a_up, *a_cat, *a_cat2, *a_attn, *a_ff;
   bool fuse_hourglass;                     // shorten gather and upsample add inside the adjacent GEMM epilogues
   float *hc_ring, *hv_ring, *trif_ring, *triv_ring, *zc, *zv, *zf;
   // draft
@@ -247,7 +247,7 @@ void carve(fm_ctx* c, Carver& cv) {
   c->ssq = cv.take<float>((size_t)((d + 127) / 128) * tc::MAX_SPLIT * Rc);
   c->logits = cv.take<float>(Rc * dm.Vpad); c->tmp3d = cv.take<float>(Rv * 3 * d);
   // GEMM operand rows of the backbone hold two bfloat16 terms per value: [hi | lo]
-  c->a_norm = cv.take<bf16>(Rc * 2 * d); c->a_cat = cv.take<bf16>(Rv * 6 * d); c->a_cat2 = cv.take<bf16>(Rf * 6 * d);
+  c->a_norm = cv.take<bf16>(Rc * 2 * d); c->a_up = cv.take<bf16>(Rc * 2 * d); c->a_cat = cv.take<bf16>(Rv * 6 * d); c->a_cat2 = cv.take<bf16>(Rf * 6 * d);
   c->a_attn = cv.take<bf16>(Rc * 2 * hd); c->a_ff = cv.take<bf16>(Rc * 2 * dm.dff);
   c->hc_ring = cv.take<float>(B * FM_RING_C * d); c->hv_ring = cv.take<float>(B * FM_RING_V * d);
   c->trif_ring = cv.take<float>(B * FM_RING_F * 3 * d); c->triv_ring = cv.take<float>(B * FM_RING_V * 3 * d);
@@ -646,10 +646,11 @@ void attention(fm_ctx* c, int level, const LayerDev& L) {
 inline size_t pad128(size_t v) { return align_up(v, 128); }
 
 // One stack of pre-norm blocks on the rows of its level (a2/a4/a6/a8/a10): five launches per
-// layer.  On entry c->a_norm holds bf16(x * g1 of the first layer) and c->ssq the rows' sums of
+// layer.  On entry c->a_norm (or `a_entry`) holds bf16(x * g1 of the first layer) and c->ssq the rows' sums of
 // squares; on exit, if `want_a`, c->a_norm holds bf16(x * next_gain) (gain 1 when null) and c->ssq
 // the sums of squares of the stack's output rows.
-void run_stack(fm_ctx* c, int s, float* x, float* stash_ring, const float* next_gain, bool want_a, const tc::Epi* cat = nullptr) {
+void run_stack(fm_ctx* c, int s, float* x, float* stash_ring, const float* next_gain, bool want_a, const tc::Epi* cat = nullptr,
+               const bf16* a_entry = nullptr) {
   const Dims& dm = c->dm;
   const int level = STACK_LEVEL[s];
   const int rows = c->batch * fm_rows_per_seq(dm, level);
@@ -667,7 +668,7 @@ void run_stack(fm_ctx* c, int s, float* x, float* stash_ring, const float* next_
     eq.dm = dm; eq.st = c->st; eq.batch = c->batch; eq.level = level; eq.rope_tab = c->rope_tab;
     eq.q_out = c->qbuf; eq.Kc = L.K; eq.Vc = L.V;
     eq.qscale = (float)(1.4426950408889634 / sqrt((double)dm.dh));   // 1/sqrt(dh) * log2(e)
-    gemm(c, L.Wqkv, pad128(qkvw), 0, c->a_norm, Rc_alloc, 0, qkvw, d, rows, na, tc::EPI_QKV, eq, 2);
+    gemm(c, L.Wqkv, pad128(qkvw), 0, l == 0 && a_entry != nullptr ? a_entry : c->a_norm, Rc_alloc, 0, qkvw, d, rows, na, tc::EPI_QKV, eq, 2);
     attention(c, level, L);
     tc::Epi eo{};
     eo.x = x; eo.ldx = d; eo.add = 1; eo.gain = L.g2; eo.a_out = c->a_norm; eo.lda = 2 * d; eo.lo_off = d;
@@ -727,12 +728,14 @@ void forward(fm_ctx* c, float* logits_out) {
     run_stack(c, 2, c->xf, c->zf, nullptr, true);                  // leaves bf16(xf) in a_norm
     tc::Epi eu{};
     eu.dm = dm; eu.st = c->st; eu.batch = B; eu.d_model = d;
-    eu.ldx = d; eu.a_out = c->a_norm; eu.lda = 2 * d; eu.lo_off = d; eu.ssq_out = c->ssq; eu.ld_ssq_out = c->ssq_ld;
+    // (the child rows' operand goes to a buffer of its own: the launch is still reading its parent
+    // rows from a_norm while the first epilogues write)
+    eu.ldx = d; eu.a_out = c->a_up; eu.lda = 2 * d; eu.lo_off = d; eu.ssq_out = c->ssq; eu.ld_ssq_out = c->ssq_ld;
     eu.level = 2; eu.x = c->xv; eu.gain = c->layers[3][0].g1; eu.tri_ring = c->trif_ring;
     // (skipped only when the CHILD level has no rows: children whose parent is older than the pass
     // still need their operand rows and sums of squares)
     gemm(c, c->U_fv, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rf, na + 1, tc::EPI_UP, eu, 2);
-    run_stack(c, 3, c->xv, c->zv, nullptr, true);                  // leaves bf16(xv) in a_norm
+    run_stack(c, 3, c->xv, c->zv, nullptr, true, nullptr, c->a_up);   // leaves bf16(xv) in a_norm
     eu.level = 1; eu.x = c->xc; eu.gain = c->layers[4][0].g1; eu.tri_ring = c->triv_ring;
     gemm(c, c->U_vc, pad128(3 * d), 0, c->a_norm, Rc_alloc, 0, 3 * d, d, Rv, na, tc::EPI_UP, eu, 2);
   } else {
@@ -758,7 +761,7 @@ void forward(fm_ctx* c, float* logits_out) {
                c->triv_ring, c->xc, (const float*)c->layers[4][0].g1, c->a_norm, c->ssq, Rc);
     c->ssq_n = 1;
   }
-  run_stack(c, 4, c->xc, c->zc, c->g_out, true);                   // leaves bf16(xc * g_out) and its sums of squares
+  run_stack(c, 4, c->xc, c->zc, c->g_out, true, nullptr, c->fuse_hourglass ? c->a_up : nullptr);   // leaves bf16(xc * g_out) and its sums of squares
   tc::Epi el = epi_plain(c->logits, dm.Vpad);
   el.ssq_in = c->ssq; el.ssq_n = c->ssq_n; el.ld_ssq = c->ssq_ld; el.inv_d_in = 1.f / d; el.eps = dm.eps;
   gemm(c, c->W_out, dm.Vpad, 0, c->a_norm, Rc_alloc, 0, dm.V, d, Rc, na, tc::EPI_F32, el, 2);
