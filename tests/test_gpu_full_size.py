@@ -92,7 +92,7 @@ def test_logits_do_not_depend_on_the_row_at_benchmark_size():
     assert torch.equal(lg_a[0, 1:], lg_b[0, :D])
 
 
-@pytest.mark.parametrize("workload,n_tok", [("medium", 130), ("batched", 70)])
+@pytest.mark.parametrize("workload,n_tok", [("medium", 130), ("batched", 70), ("large", 60)])
 def test_every_accept_pattern_leaves_the_logits_of_plain_decoding(workload, n_tok):
     """Bit-exact losslessness (Sec. 3.3) at benchmark size.  A position's hidden states reach the
     upper stacks along different code paths depending on where the passes happen to start: with its
