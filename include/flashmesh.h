@@ -40,6 +40,13 @@
  *   - Indexing: inputs u_0 = BOS, u_i = t_{i-1}; the row at position i predicts mesh token
  *     t_i.  L = inputs consumed so far; the pending main token is t_{L-1}.  A verify pass
  *     feeds positions L..L+D; accepting a tokens moves L to L+a.
+ *   - Lossless by construction (Sec. 3.3): within one context the logits of a position do not
+ *     depend on the row of the pass it is fed in, on the other rows or sequences of the pass,
+ *     nor on the accept lengths of the passes before it, to the last bit (reduction orders are
+ *     fixed by slot and column index; every value that can be produced at two places of the code
+ *     is rounded explicitly), so the tokens a speculative run emits are those of one-token-per-
+ *     pass decoding with the same context, whatever the drafts were.  Two contexts (another
+ *     batch size, draft count or capacity) may group reductions differently.
  *   - Token ids: [0, n_bins) coordinate bins, BOS = n_bins, EOS = n_bins+1, PAD = n_bins+2.
  *     Emitted ids are always coordinate bins, or EOS at a face boundary when allow_eos != 0;
  *     ties in an argmax go to the lowest id.
