@@ -293,3 +293,32 @@ def test_step_host_equals_the_stepwise_calls():
         assert int(n_a[0]) == int(nacc_h[0]) and em_a.cpu().tolist() == em_h.tolist() and kv_a.cpu().tolist() == kv_h.tolist()
         L += int(nacc_h[0])
     assert a.device_status() == 0 and b.device_status() == 0
+
+
+@pytest.mark.parametrize("switch", ["FM_NO_FUSE", "FM_NO_PDL", "FM_NO_CALL_GRAPH"])
+def test_toy_lockstep_with_a_fallback_switch(switch, monkeypatch):
+    """The environment switches select other launch forms of the same arithmetic (shorten gather
+    and upsample add as row-wise kernels; launches without programmatic dependent launch; stepwise
+    calls never replayed as graphs): each must pass the same lock-step check, with accept lengths
+    that vary so that rows cross passes."""
+    from oracle.lockstep import run_lockstep
+    monkeypatch.setenv(switch, "1")
+    cfg = S.toy_config(**TOY, draft_len=9, layers=(1, 1, 2, 1, 1), max_batch=2, gen_faces=8, max_tokens=1 + 9 * 8 + 9 + 2)
+    w, conds, prompts = _setup(cfg, batch=2)
+    truth = [_oracle_greedy(cfg, w, conds[b], prompts[b], 8) for b in range(2)]
+    dev = _dev(cfg, w)
+    rep = run_lockstep(cfg, w, conds, prompts, dev, 8, 300, truth=truth, keep_rng=np.random.default_rng(5), tol=TOY_TOL, margin=TOY_MARGIN)
+    assert rep["done"] and dev.device_status() == 0
+
+
+def test_toy_lockstep_width_not_a_multiple_of_128():
+    """d = 192 (two heads of 64, d_ff = 320): the last tile of most projections is partly empty and
+    the hourglass steps run as row-wise kernels (the fused epilogues want d to be a multiple of 128)."""
+    from oracle.lockstep import run_lockstep
+    cfg = S.toy_config(d_model=192, n_heads=2, n_kv_heads=2, head_dim=64, d_ff=320, weight_std=0.1, out_std=0.02, draft_len=9,
+                       layers=(1, 1, 2, 1, 1), max_batch=2, gen_faces=6, max_tokens=1 + 9 * 8 + 9 + 2)
+    w, conds, prompts = _setup(cfg, batch=2)
+    truth = [_oracle_greedy(cfg, w, conds[b], prompts[b], 6) for b in range(2)]
+    dev = _dev(cfg, w)
+    rep = run_lockstep(cfg, w, conds, prompts, dev, 6, 300, truth=truth, keep_rng=np.random.default_rng(3), tol=TOY_TOL, margin=TOY_MARGIN)
+    assert rep["done"] and dev.device_status() == 0
