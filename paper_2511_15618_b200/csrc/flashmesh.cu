@@ -1213,7 +1213,8 @@ int fm_create(const fm_config* cfg, const fm_weights* w, void* dev_workspace, si
     const char* tt = getenv("FM_SPLIT_TARGET_DEEP");
     c->split_target_deep = tt != nullptr && atoi(tt) > 0 ? atoi(tt) : 296;
     const char* nf = getenv("FM_NO_FUSE");
-    c->fuse_hourglass = c->dm.d % tc::BM == 0 && !(nf != nullptr && nf[0] == '1');
+    // (the upsampling epilogue lists at most 128 carried rows per slot: one per sequence)
+    c->fuse_hourglass = c->dm.d % tc::BM == 0 && c->dm.max_batch <= 128 && !(nf != nullptr && nf[0] == '1');
     const char* sc = getenv("FM_STAGE_CAP");
     c->stage_cap = sc != nullptr ? atoi(sc) : 4;        // measured: deeper rings cost more than they prefetch
   }

@@ -322,3 +322,21 @@ def test_toy_lockstep_width_not_a_multiple_of_128():
     dev = _dev(cfg, w)
     rep = run_lockstep(cfg, w, conds, prompts, dev, 6, 300, truth=truth, keep_rng=np.random.default_rng(3), tol=TOY_TOL, margin=TOY_MARGIN)
     assert rep["done"] and dev.device_status() == 0
+
+
+@pytest.mark.parametrize("heads", ["reduced", "full"])
+def test_toy_lockstep_forty_sequences(heads):
+    """More than 32 sequences: the stacked draft projections run one launch per head, the verify
+    pass has several row tiles per projection, and accept lengths differ per sequence."""
+    from oracle.lockstep import run_lockstep
+    B = 40
+    cfg = S.toy_config(**TOY, draft_len=3, draft_heads=heads, layers=(1, 1, 1, 1, 1), max_batch=B, batch=B, gen_faces=3,
+                       prompt_faces=(1, 1), max_tokens=1 + 9 * 8 + 3 + 2)
+    w, conds, prompts = _setup(cfg, batch=B)
+    for b in range(0, B, 3):
+        prompts[b] = prompts[b] + prompts[(b + 1) % B]           # ragged: 1 and 2 faces
+    truth = [_oracle_greedy(cfg, w, conds[b], prompts[b], 3) for b in range(B)]
+    dev = _dev(cfg, w)
+    rep = run_lockstep(cfg, w, conds, prompts, dev, 3, 120, truth=truth, keep_rng=np.random.default_rng(11), tol=TOY_TOL, margin=TOY_MARGIN)
+    assert rep["done"] and rep["emitted"] == 27 * B
+    assert dev.device_status() == 0
